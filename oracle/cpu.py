@@ -1,0 +1,208 @@
+"""ctypes front end of the C++ oracle (``dai8_oracle.cpp``).  Test infrastructure only.
+
+All tensors are numpy arrays in plain NCHW / (Cout,Cin,R,S) order.  Every function returns new
+arrays; none of them touches a GPU.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "dai8_oracle.cpp"
+_SO = _HERE / "libdai8_oracle.so"
+_lib = None
+
+
+def build(force: bool = False) -> Path:
+    """Compile the oracle with g++ (no fused multiply-add contraction, OpenMP across channels)."""
+    if force or not _SO.exists() or _SO.stat().st_mtime < _SRC.stat().st_mtime:
+        tmp = _SO.with_suffix(f".tmp{os.getpid()}.so")
+        cmd = ["g++", "-std=c++17", "-O2", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-o", str(tmp), str(_SRC)]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(str(build()))
+        _lib.dai8o_rand_uniform.restype = ctypes.c_float
+        _lib.dai8o_rand_uniform.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64]
+        _lib.dai8o_rand_bits.restype = ctypes.c_uint32
+        _lib.dai8o_rand_bits.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64]
+        _lib.dai8o_num_threads.restype = ctypes.c_int
+        for name in ("dai8o_conv_fwd_acc", "dai8o_conv_bwd_data_acc", "dai8o_conv_bwd_filter_acc"):
+            getattr(_lib, name).restype = ctypes.c_int64
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().dai8o_num_threads())
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def channel_stats(g, std_unbiased: bool = False, center_mean: bool = True):
+    """Algorithm 1 line 2.  Returns (absmax[C], mean[C], sigma[C], gmax_layer) as fp32."""
+    g = _f32(g)
+    N, C, H, W = g.shape
+    absmax = np.empty(C, np.float32)
+    mean = np.empty(C, np.float32)
+    sigma = np.empty(C, np.float32)
+    gl = np.empty(1, np.float32)
+    lib().dai8o_channel_stats(_p(g), N, C, H, W, int(std_unbiased), int(center_mean), _p(absmax),
+                              _p(mean), _p(sigma), _p(gl))
+    return absmax, mean, sigma, float(gl[0])
+
+
+def density_count(g, sigma) -> np.ndarray:
+    """Algorithm 1 line 4: #{|g| > sigma_c} per channel (uint32)."""
+    g = _f32(g)
+    sigma = _f32(sigma)
+    N, C, H, W = g.shape
+    assert sigma.shape == (C,)
+    cnt = np.empty(C, np.uint32)
+    lib().dai8o_density_count(_p(g), N, C, H, W, _p(sigma), _p(cnt))
+    return cnt
+
+
+def classify_clip(cnt, absmax, M: int, s_prev=None, lam: float = 0.3, k: float = 1.0,
+                  A: float = 0.8):
+    """Algorithm 1 lines 5-9.  Returns (s_t[C] fp32, cls[C] uint8 with 1 = bell-shaped)."""
+    cnt = np.ascontiguousarray(cnt, dtype=np.uint32)
+    absmax = _f32(absmax)
+    C = cnt.shape[0]
+    state = _f32(s_prev).copy() if s_prev is not None else np.zeros(C, np.float32)
+    cls = np.empty(C, np.uint8)
+    lib().dai8o_classify_clip(_p(cnt), _p(absmax), C, ctypes.c_int64(M), ctypes.c_float(lam),
+                              ctypes.c_float(k), ctypes.c_float(A), _p(state),
+                              int(s_prev is not None), _p(cls))
+    return state, cls
+
+
+def rand_uniform(seed: int, stream: int, index: int) -> float:
+    return float(lib().dai8o_rand_uniform(seed & 0xFFFFFFFF, stream, index))
+
+
+def rand_bits(seed: int, stream: int, index: int) -> int:
+    return int(lib().dai8o_rand_bits(seed & 0xFFFFFFFF, stream, index))
+
+
+def quantize(x, scale, stochastic: bool = False, seed: int = 0, stream: int = 0) -> np.ndarray:
+    """Eq. 1.  scale: scalar (layer-wide) or array [C] (per channel).  Returns NCHW int8 codes."""
+    x = _f32(x)
+    N, C, H, W = x.shape
+    scale = np.atleast_1d(_f32(scale))
+    per_channel = scale.shape[0] != 1
+    if per_channel:
+        assert scale.shape == (C,)
+    q = np.empty(x.shape, np.int8)
+    lib().dai8o_quantize(_p(x), N, C, H, W, _p(scale), int(per_channel), int(stochastic),
+                         ctypes.c_uint32(seed & 0xFFFFFFFF), ctypes.c_uint32(stream), _p(q))
+    return q
+
+
+def dequantize(q, scale) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    N, C, H, W = q.shape
+    scale = np.atleast_1d(_f32(scale))
+    out = np.empty(q.shape, np.float32)
+    lib().dai8o_dequantize(_p(q), N, C, H, W, _p(scale), int(scale.shape[0] != 1), _p(out))
+    return out
+
+
+def _geom(N, Cin, Cout, H, W, R, S, stride, pad) -> np.ndarray:
+    sh, sw = (stride, stride) if np.isscalar(stride) else stride
+    ph, pw = (pad, pad) if np.isscalar(pad) else pad
+    return np.array([N, Cin, Cout, H, W, R, S, sh, sw, ph, pw], dtype=np.int32)
+
+
+def out_hw(H, W, R, S, stride, pad):
+    sh, sw = (stride, stride) if np.isscalar(stride) else stride
+    ph, pw = (pad, pad) if np.isscalar(pad) else pad
+    return (H + 2 * ph - R) // sh + 1, (W + 2 * pw - S) // sw + 1
+
+
+def _idx(idx):
+    if idx is None:
+        return None, 0
+    idx = np.ascontiguousarray(idx, dtype=np.int64)
+    return idx, idx.shape[0]
+
+
+def conv_fwd_acc(qX, qW, stride=1, pad=0, idx=None):
+    """Integer forward convolution.  Returns (acc int64, n_overflow).  acc is (N,Cout,P,Q), or one
+    value per flat NCHW output index in ``idx``."""
+    qX = np.ascontiguousarray(qX, dtype=np.int8)
+    qW = np.ascontiguousarray(qW, dtype=np.int8)
+    N, Cin, H, W = qX.shape
+    Cout, Cin2, R, S = qW.shape
+    assert Cin == Cin2
+    P, Q = out_hw(H, W, R, S, stride, pad)
+    g = _geom(N, Cin, Cout, H, W, R, S, stride, pad)
+    idx, n = _idx(idx)
+    acc = np.empty(n if n else (N, Cout, P, Q), np.int64)
+    ov = lib().dai8o_conv_fwd_acc(_p(qX), _p(qW), _p(g), _p(idx) if n else None,
+                                  ctypes.c_int64(n), _p(acc))
+    return acc, int(ov)
+
+
+def conv_bwd_data_acc(qG, qW, in_hw, stride=1, pad=0, idx=None):
+    """Integer input gradient (Eq. 3).  qG is (N,Cout,P,Q); returns acc (N,Cin,H,W) or samples."""
+    qG = np.ascontiguousarray(qG, dtype=np.int8)
+    qW = np.ascontiguousarray(qW, dtype=np.int8)
+    N, Cout, P, Q = qG.shape
+    Cout2, Cin, R, S = qW.shape
+    assert Cout == Cout2
+    H, W = in_hw
+    assert (P, Q) == out_hw(H, W, R, S, stride, pad)
+    g = _geom(N, Cin, Cout, H, W, R, S, stride, pad)
+    idx, n = _idx(idx)
+    acc = np.empty(n if n else (N, Cin, H, W), np.int64)
+    ov = lib().dai8o_conv_bwd_data_acc(_p(qG), _p(qW), _p(g), _p(idx) if n else None,
+                                       ctypes.c_int64(n), _p(acc))
+    return acc, int(ov)
+
+
+def conv_bwd_filter_acc(qX, qG, filter_hw, stride=1, pad=0, idx=None):
+    """Integer weight gradient (Eq. 4).  Returns acc (Cout,Cin,R,S) or samples."""
+    qX = np.ascontiguousarray(qX, dtype=np.int8)
+    qG = np.ascontiguousarray(qG, dtype=np.int8)
+    N, Cin, H, W = qX.shape
+    N2, Cout, P, Q = qG.shape
+    R, S = filter_hw
+    assert N == N2 and (P, Q) == out_hw(H, W, R, S, stride, pad)
+    g = _geom(N, Cin, Cout, H, W, R, S, stride, pad)
+    idx, n = _idx(idx)
+    acc = np.empty(n if n else (Cout, Cin, R, S), np.int64)
+    ov = lib().dai8o_conv_bwd_filter_acc(_p(qX), _p(qG), _p(g), _p(idx) if n else None,
+                                         ctypes.c_int64(n), _p(acc))
+    return acc, int(ov)
+
+
+def dequant_acc(acc, sa: float, sb) -> np.ndarray:
+    """out = float(acc) * ((sa/127) * (sb/127)); sb scalar, or one value per leading index of acc."""
+    acc = np.ascontiguousarray(acc, dtype=np.int64)
+    sb = np.atleast_1d(_f32(sb))
+    per_row = sb.shape[0] != 1
+    rows = acc.shape[0] if per_row else 1
+    cols = acc.size // rows
+    if per_row:
+        assert sb.shape[0] == rows
+    out = np.empty(acc.shape, np.float32)
+    lib().dai8o_dequant_acc(_p(acc), ctypes.c_int64(rows), ctypes.c_int64(cols),
+                            ctypes.c_float(sa), _p(sb), int(per_row), _p(out))
+    return out
