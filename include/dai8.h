@@ -1,0 +1,180 @@
+/* dai8 -- Distribution Adaptive INT8 quantization of the convolution backward pass, for B200
+ * (sm_100a).  C ABI of libdai8.so.
+ *
+ * The library implements one training step of one convolution layer as the paper defines it:
+ *
+ *   forward   q(X), q(W) with layer-wide scales and nearest rounding (Sec. 3, Eq. 1; Fig. 2)
+ *             Y = (q(X) * q(W)) . (s_X/127)(s_W/127)                       -> dai8_conv_fwd
+ *   backward  Algorithm 1: per-channel |g|max and sigma of dY, density P(|g| > sigma), the
+ *             discriminator (Eq. 15), the clip rule (Eq. 11 / Eq. 14), per-channel codes vq(dY)
+ *             and layer-wide codes q(dY) with stochastic rounding        -> dai8_quantize_grad
+ *             G_W = q(X') (x) vq(G'), de-quantized per output channel (Eq. 4-7)
+ *                                                                        -> dai8_conv_bwd_filter
+ *             G_X = q(G) (.) q(W), de-quantized with |g|max and s_W (Eq. 3)
+ *                                                                        -> dai8_conv_bwd_data
+ *
+ * General rules
+ *   - Every pointer is DEVICE memory owned by the caller unless its comment says "host".
+ *     All device pointers must be 16-byte aligned.
+ *   - The library allocates nothing, never synchronises the stream (except
+ *     dai8_get_device_status) and never copies a scale to the host: each call only enqueues
+ *     work on `stream` (a cudaStream_t passed as void*; NULL = the legacy default stream).
+ *   - Scratch memory is passed in (`ws`, `ws_bytes`); ask dai8_*_workspace_bytes for the size.
+ *     Its contents are undefined between calls.  Calls that share a workspace must be ordered
+ *     on one stream.
+ *   - Errors are return codes; arguments are checked on the host before anything is enqueued.
+ *     A geometry the kernels do not cover returns DAI8_ERR_UNSUPPORTED: there is no CPU path.
+ *   - Device-side waits are bounded.  A wait that runs out records DAI8_ERR_TIMEOUT in a device
+ *     status word that dai8_get_device_status reads; the affected output is then undefined.
+ *
+ * Code tensors (int8, values in [-127, 127])
+ *   - activations / gradients:  [N][H][W][Cp]       Cp = C rounded up to a multiple of 16
+ *   - weights:                  [Cout][R][S][Cinp]  Cinp = Cin rounded up to a multiple of 16
+ *   The padding channels hold code 0.  dai8_quantize_tensor produces the weight layout when the
+ *   weights are passed as an NCHW tensor with N=Cout, C=Cin, H=R, W=S.
+ */
+#ifndef DAI8_H
+#define DAI8_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  DAI8_OK = 0,
+  DAI8_ERR_INVALID_ARG = 1, /* null / misaligned pointer, non-positive size, bad enum        */
+  DAI8_ERR_UNSUPPORTED = 2, /* valid request outside what the kernels implement               */
+  DAI8_ERR_WORKSPACE = 3,   /* ws_bytes smaller than dai8_*_workspace_bytes reports           */
+  DAI8_ERR_ARCH = 4,        /* current device is not compute capability 10.x                  */
+  DAI8_ERR_CUDA = 5,        /* a CUDA runtime / driver call failed                            */
+  DAI8_ERR_TIMEOUT = 6      /* a bounded device-side wait expired (device status word)        */
+} dai8_status;
+
+typedef enum { DAI8_F32 = 0, DAI8_BF16 = 1, DAI8_I32 = 2 } dai8_dtype; /* I32: raw accumulators */
+typedef enum { DAI8_NCHW = 0, DAI8_NHWC = 1 } dai8_layout;
+typedef enum { DAI8_ROUND_NEAREST_EVEN = 0, DAI8_ROUND_STOCHASTIC = 1 } dai8_round;
+typedef enum { DAI8_SCALE_ABSMAX = 0, DAI8_SCALE_GIVEN = 1 } dai8_scale_mode;
+
+/* Convolution geometry: X (N,Cin,H,W), W (Cout,Cin,R,S), Y (N,Cout,P,Q) with
+ * P = (H + 2*pad_h - R)/stride_h + 1, Q likewise (Sec. 3.2).  Cross-correlation, dilation 1,
+ * one group. */
+typedef struct {
+  int N, Cin, Cout, H, W, R, S, stride_h, stride_w, pad_h, pad_w;
+} dai8_conv_geom;
+
+/* Hyper-parameters of the Magnitude-aware Clipping Strategy.  Paper values: lambda = 0.3
+ * (Eq. 15), k = 1, A = 0.8 (Sec. 4.1).  sigma is the population standard deviation about the
+ * channel mean unless std_unbiased (divide by M-1) or center_mean = 0 (root mean square). */
+typedef struct {
+  float lambda, k, A;
+  int std_unbiased;
+  int center_mean;
+} dai8_mcs_params;
+
+/* Rows of the `stats` output of dai8_quantize_grad: stats[c*4 + i]. */
+enum { DAI8_STAT_ABSMAX = 0, DAI8_STAT_MEAN = 1, DAI8_STAT_SIGMA = 2, DAI8_STAT_P = 3 };
+
+const char* dai8_status_string(dai8_status s);
+
+/* Fills *p with the paper's hyper-parameters (host pointer). */
+void dai8_mcs_defaults(dai8_mcs_params* p);
+
+/* Number of channels of a code tensor holding C logical channels (C rounded up to 16). */
+int dai8_padded_channels(int C);
+
+/* ----------------------------------------------------------------------------------------------
+ * dai8_quantize_tensor -- Eq. 1 with one scale for the whole tensor (forward quantization of X
+ * and W, Fig. 2; also usable for layer-wide gradient codes).
+ *   x          input, N*C*H*W elements of `dtype` (F32 or BF16) in `layout`
+ *   scale_mode ABSMAX: *scale is written with max|x| and then used; GIVEN: *scale is read
+ *   scale      device, 1 float
+ *   round      nearest-even (weights, activations) or stochastic (gradients); the stochastic
+ *              mode draws u from a counter-based hash of (seed, stream 0, NCHW index)
+ *   q          out, int8 [N][H][W][Cp]; padding channels are written with 0
+ * Workspace: none.  q(x) = round(clamp(x*(127/s), -127, 127)); s <= 0 gives all-zero codes.
+ * -------------------------------------------------------------------------------------------- */
+dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout layout, int N, int C,
+                                 int H, int W, dai8_scale_mode scale_mode, float* scale,
+                                 dai8_round round, uint32_t seed, int8_t* q, void* stream);
+
+/* ----------------------------------------------------------------------------------------------
+ * dai8_quantize_grad -- Algorithm 1 lines 1-11: Gradient Vectorized Quantization with the
+ * Magnitude-aware Clipping Strategy.
+ *   dY         gradient of the layer output, (N,C,H,W) elements of `dtype` in `layout`
+ *              (C = Cout, H x W = output extent)
+ *   params     host pointer; NULL = paper defaults
+ *   s_state    device [C]: in  s_{c,t-1} (read only if has_prev != 0; otherwise s_{c,t-1} is
+ *              taken as |g|max,c), out s_{c,t} -- the per-channel clip values used for `vq`
+ *   gmax_layer device [1], out: |g|max of the layer, the scale of `gq`
+ *   stats      device [C][4] or NULL, out: |g|max,c, mean, sigma, P = #{|g|>sigma}/M
+ *   cls        device [C] or NULL, out: 1 = bell-shaped (P > lambda), 0 = Inverted-T
+ *   vq         out, int8 [N][H][W][Cp]: per-channel codes (for dai8_conv_bwd_filter)
+ *   gq         out or NULL, int8 [N][H][W][Cp]: layer-wide codes (for dai8_conv_bwd_data)
+ *   seed       stochastic-rounding seed; vq uses stream 0, gq stream 1 of the generator
+ *   sigma_override  device [C] or NULL: when given, the density count uses these values instead
+ *              of the sigma computed from dY (lets a checker feed identical sigma to both sides)
+ * Workspace: dai8_quantize_grad_workspace_bytes(C).
+ * -------------------------------------------------------------------------------------------- */
+size_t dai8_quantize_grad_workspace_bytes(int C);
+
+dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8_layout layout, int N, int C,
+                               int H, int W, const dai8_mcs_params* params, float* s_state,
+                               int has_prev, float* gmax_layer, float* stats, uint8_t* cls,
+                               int8_t* vq, int8_t* gq, uint32_t seed,
+                               const float* sigma_override, void* ws, size_t ws_bytes,
+                               void* stream);
+
+/* ----------------------------------------------------------------------------------------------
+ * Convolutions on int8 codes with int32 accumulation and a de-quantizing epilogue.
+ *
+ * dai8_conv_fwd        Y[n,co,p,q]   = acc . ((sX/127)(sW/127)),
+ *                      acc = sum_{ci,r,s} qX[n,p*st+r-pad,q*st+s-pad,ci] qW[co,r,s,ci]   (Fig. 2)
+ * dai8_conv_bwd_data   dX[n,ci,h,w]  = acc . ((gmax/127)(sW/127)),
+ *                      acc = sum over (co,r,s,p,q) with h=p*st+r-pad, w=q*st+s-pad of
+ *                      gq[n,p,q,co] qW[co,r,s,ci]                      (Eq. 3, Alg. 1 l. 12, 15)
+ * dai8_conv_bwd_filter dW[co,ci,r,s] = acc . ((sX/127)(s[co]/127)),
+ *                      acc = sum_{n,p,q} vq[n,p,q,co] qX[n,p*st+r-pad,q*st+s-pad,ci]
+ *                                                                      (Eq. 4-7, Alg. 1 l. 11, 14)
+ *   sX, sW, gmax   device, 1 float each;  s: device [Cout] (the s_state of dai8_quantize_grad)
+ *   out_dtype      F32 or BF16 (de-quantized), or I32: the raw accumulators, scales ignored
+ *   out_layout     NCHW or NHWC for Y / dX (C unpadded); dW is always (Cout,Cin,R,S)
+ * Accumulators are int32 and wrap on overflow (possible only for K*127^2 > 2^31, far beyond
+ * what zero-mean gradients reach).  Workspace: dai8_conv_workspace_bytes(op, geom).
+ * -------------------------------------------------------------------------------------------- */
+typedef enum { DAI8_OP_FWD = 0, DAI8_OP_BWD_DATA = 1, DAI8_OP_BWD_FILTER = 2 } dai8_conv_op;
+
+size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geom* geom /* host */);
+
+dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                          const dai8_conv_geom* geom /* host */, void* Y, dai8_dtype out_dtype,
+                          dai8_layout out_layout, void* ws, size_t ws_bytes, void* stream);
+
+dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, const float* gmax,
+                               const float* sW, const dai8_conv_geom* geom /* host */, void* dX,
+                               dai8_dtype out_dtype, dai8_layout out_layout, void* ws,
+                               size_t ws_bytes, void* stream);
+
+dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, const float* sX,
+                                 const float* s, const dai8_conv_geom* geom /* host */, void* dW,
+                                 dai8_dtype out_dtype, void* ws, size_t ws_bytes, void* stream);
+
+/* Kernel family selection for the convolutions (process-wide, host side): 0 = automatic
+ * (tensor-core kernels where the geometry allows, direct kernels otherwise), 1 = direct kernels
+ * only, 2 = tensor-core kernels only (DAI8_ERR_UNSUPPORTED where they do not apply).  Used by
+ * the tests to compare the two families bit for bit. */
+void dai8_set_conv_backend(int mode);
+
+/* Number of kernels the library has launched from this process so far (host counter). */
+uint64_t dai8_launch_count(void);
+
+/* Reads and clears the device status word (DAI8_OK or DAI8_ERR_TIMEOUT).  Synchronises `stream`.
+ * host_status: host pointer. */
+dai8_status dai8_get_device_status(int* host_status, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DAI8_H */

@@ -1,0 +1,204 @@
+"""Thin Python binding of libdai8.so (ctypes).  Same names as ``include/dai8.h``.
+
+Argument marshalling only: tensors are torch CUDA tensors used as device buffers, every step of
+the path runs in the library's kernels.  The shared library must have been built
+(``python -m paper_2102_04782_b200.build``); a missing library is an error, there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+from ctypes import c_int, c_size_t, c_uint32, c_uint64, c_void_p
+from pathlib import Path
+from typing import Optional
+
+import torch
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT = range(7)
+F32, BF16, I32 = 0, 1, 2
+NCHW, NHWC = 0, 1
+ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
+SCALE_ABSMAX, SCALE_GIVEN = 0, 1
+OP_FWD, OP_BWD_DATA, OP_BWD_FILTER = 0, 1, 2
+
+EXPORTS = [
+    "dai8_status_string", "dai8_mcs_defaults", "dai8_padded_channels", "dai8_quantize_tensor",
+    "dai8_quantize_grad_workspace_bytes", "dai8_quantize_grad", "dai8_conv_workspace_bytes",
+    "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
+    "dai8_launch_count", "dai8_get_device_status",
+]
+
+
+class ConvGeom(ctypes.Structure):
+    _fields_ = [(n, c_int) for n in ("N", "Cin", "Cout", "H", "W", "R", "S", "stride_h", "stride_w",
+                                     "pad_h", "pad_w")]
+
+    @property
+    def P(self) -> int:
+        return (self.H + 2 * self.pad_h - self.R) // self.stride_h + 1
+
+    @property
+    def Q(self) -> int:
+        return (self.W + 2 * self.pad_w - self.S) // self.stride_w + 1
+
+
+class McsParams(ctypes.Structure):
+    _fields_ = [("lam", ctypes.c_float), ("k", ctypes.c_float), ("A", ctypes.c_float),
+                ("std_unbiased", c_int), ("center_mean", c_int)]
+
+
+class Dai8Error(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__(f"{where}: {status_string(code)} (status {code})")
+
+
+_LIB_PATH = Path(__file__).resolve().parent / "libdai8.so"
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        if not _LIB_PATH.exists():
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with "
+                               "`python -m paper_2102_04782_b200.build` (there is no CPU fallback)")
+        l = ctypes.CDLL(str(_LIB_PATH))
+        l.dai8_status_string.restype = ctypes.c_char_p
+        l.dai8_status_string.argtypes = [c_int]
+        l.dai8_mcs_defaults.restype = None
+        l.dai8_padded_channels.restype = c_int
+        l.dai8_quantize_grad_workspace_bytes.restype = c_size_t
+        l.dai8_quantize_grad_workspace_bytes.argtypes = [c_int]
+        l.dai8_conv_workspace_bytes.restype = c_size_t
+        l.dai8_conv_workspace_bytes.argtypes = [c_int, ctypes.POINTER(ConvGeom)]
+        l.dai8_launch_count.restype = c_uint64
+        l.dai8_set_conv_backend.restype = None
+        l.dai8_quantize_tensor.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_int,
+                                           c_void_p, c_int, c_uint32, c_void_p, c_void_p]
+        l.dai8_quantize_grad.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int,
+                                         ctypes.POINTER(McsParams), c_void_p, c_int, c_void_p,
+                                         c_void_p, c_void_p, c_void_p, c_void_p, c_uint32, c_void_p,
+                                         c_void_p, c_size_t, c_void_p]
+        conv_args = [c_void_p, c_void_p, c_void_p, c_void_p, ctypes.POINTER(ConvGeom), c_void_p, c_int,
+                     c_int, c_void_p, c_size_t, c_void_p]
+        l.dai8_conv_fwd.argtypes = conv_args
+        l.dai8_conv_bwd_data.argtypes = conv_args
+        l.dai8_conv_bwd_filter.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p,
+                                           ctypes.POINTER(ConvGeom), c_void_p, c_int, c_void_p,
+                                           c_size_t, c_void_p]
+        l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
+        _lib = l
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().dai8_status_string(code).decode()
+
+
+def _check(code: int, where: str) -> None:
+    if code != OK:
+        raise Dai8Error(code, where)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError("dai8 takes CUDA tensors (device buffers)")
+    if not t.is_contiguous():
+        raise ValueError("dai8 takes contiguous buffers")
+    return c_void_p(t.data_ptr())
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    if t.dtype == torch.int32:
+        return I32
+    raise ValueError(f"unsupported dtype {t.dtype}")
+
+
+def padded_channels(C: int) -> int:
+    return int(lib().dai8_padded_channels(C))
+
+
+def mcs_defaults() -> McsParams:
+    p = McsParams()
+    lib().dai8_mcs_defaults(ctypes.byref(p))
+    return p
+
+
+def launch_count() -> int:
+    return int(lib().dai8_launch_count())
+
+
+def set_conv_backend(mode: int) -> None:
+    lib().dai8_set_conv_backend(mode)
+
+
+def get_device_status() -> int:
+    v = c_int(0)
+    _check(lib().dai8_get_device_status(ctypes.byref(v), _stream()), "dai8_get_device_status")
+    return v.value
+
+
+def quantize_tensor(x: torch.Tensor, layout: int, N: int, C: int, H: int, W: int, scale_mode: int,
+                    scale: torch.Tensor, rounding: int, seed: int, q: torch.Tensor) -> None:
+    """dai8_quantize_tensor: x (fp32/bf16, `layout`) -> q int8 [N][H][W][Cp]; scale: 1 float."""
+    _check(lib().dai8_quantize_tensor(_ptr(x), _dtype_code(x), layout, N, C, H, W, scale_mode,
+                                      _ptr(scale), rounding, seed & 0xFFFFFFFF, _ptr(q), _stream()),
+           "dai8_quantize_tensor")
+
+
+def quantize_grad_workspace_bytes(C: int) -> int:
+    return int(lib().dai8_quantize_grad_workspace_bytes(C))
+
+
+def quantize_grad(dY: torch.Tensor, layout: int, N: int, C: int, H: int, W: int,
+                  params: Optional[McsParams], s_state: torch.Tensor, has_prev: bool,
+                  gmax_layer: torch.Tensor, stats: Optional[torch.Tensor],
+                  cls: Optional[torch.Tensor], vq: torch.Tensor, gq: Optional[torch.Tensor],
+                  seed: int, ws: torch.Tensor, sigma_override: Optional[torch.Tensor] = None) -> None:
+    """dai8_quantize_grad (Algorithm 1 lines 1-11)."""
+    _check(lib().dai8_quantize_grad(_ptr(dY), _dtype_code(dY), layout, N, C, H, W,
+                                    ctypes.byref(params) if params is not None else None,
+                                    _ptr(s_state), int(has_prev), _ptr(gmax_layer), _ptr(stats),
+                                    _ptr(cls), _ptr(vq), _ptr(gq), seed & 0xFFFFFFFF,
+                                    _ptr(sigma_override), _ptr(ws), ws.numel() * ws.element_size(),
+                                    _stream()), "dai8_quantize_grad")
+
+
+def conv_workspace_bytes(op: int, geom: ConvGeom) -> int:
+    return int(lib().dai8_conv_workspace_bytes(op, ctypes.byref(geom)))
+
+
+def _ws_args(ws: Optional[torch.Tensor]):
+    if ws is None:
+        return None, 0
+    return _ptr(ws), ws.numel() * ws.element_size()
+
+
+def conv_fwd(qX, qW, sX, sW, geom: ConvGeom, Y: torch.Tensor, out_layout: int, ws=None) -> None:
+    p, n = _ws_args(ws)
+    _check(lib().dai8_conv_fwd(_ptr(qX), _ptr(qW), _ptr(sX), _ptr(sW), ctypes.byref(geom), _ptr(Y),
+                               _dtype_code(Y), out_layout, p, n, _stream()), "dai8_conv_fwd")
+
+
+def conv_bwd_data(gq, qW, gmax, sW, geom: ConvGeom, dX: torch.Tensor, out_layout: int, ws) -> None:
+    p, n = _ws_args(ws)
+    _check(lib().dai8_conv_bwd_data(_ptr(gq), _ptr(qW), _ptr(gmax), _ptr(sW), ctypes.byref(geom),
+                                    _ptr(dX), _dtype_code(dX), out_layout, p, n, _stream()),
+           "dai8_conv_bwd_data")
+
+
+def conv_bwd_filter(qX, vq, sX, s, geom: ConvGeom, dW: torch.Tensor, ws) -> None:
+    p, n = _ws_args(ws)
+    _check(lib().dai8_conv_bwd_filter(_ptr(qX), _ptr(vq), _ptr(sX), _ptr(s), ctypes.byref(geom),
+                                      _ptr(dW), _dtype_code(dW), p, n, _stream()),
+           "dai8_conv_bwd_filter")

@@ -1,0 +1,116 @@
+// C-ABI entry points of the convolutions: argument checks, workspace carving, kernel-family choice.
+#include "conv_internal.cuh"
+
+namespace dai8 {
+namespace {
+
+std::atomic<int> g_backend{0};  // 0 auto, 1 direct only, 2 tensor-core only
+
+dai8_status check_geom(const dai8_conv_geom* g) {
+  if (!g) return DAI8_ERR_INVALID_ARG;
+  if (g->N <= 0 || g->Cin <= 0 || g->Cout <= 0 || g->H <= 0 || g->W <= 0 || g->R <= 0 || g->S <= 0 ||
+      g->stride_h <= 0 || g->stride_w <= 0 || g->pad_h < 0 || g->pad_w < 0)
+    return DAI8_ERR_INVALID_ARG;
+  if (g->H + 2 * g->pad_h < g->R || g->W + 2 * g->pad_w < g->S) return DAI8_ERR_INVALID_ARG;
+  const ConvShape cs = make_shape(*g);
+  const int64_t lim = (int64_t)1 << 31;
+  if ((int64_t)g->N * cs.P * cs.Q >= lim || (int64_t)g->N * g->H * g->W >= lim) return DAI8_ERR_UNSUPPORTED;
+  return DAI8_OK;
+}
+
+bool bad_out(dai8_dtype t) { return t != DAI8_F32 && t != DAI8_BF16 && t != DAI8_I32; }
+bool bad_layout(dai8_layout l) { return l != DAI8_NCHW && l != DAI8_NHWC; }
+
+size_t wt_bytes(const ConvShape& cs) { return (size_t)cs.Cinp * cs.R * cs.S * cs.Coutp; }
+size_t dw_acc_bytes(const ConvShape& cs) { return (size_t)cs.Coutp * cs.R * cs.S * cs.Cinp * sizeof(int); }
+
+}  // namespace
+}  // namespace dai8
+
+using namespace dai8;
+
+extern "C" void dai8_set_conv_backend(int mode) { g_backend.store(mode < 0 || mode > 2 ? 0 : mode); }
+
+extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geom* geom) {
+  if (check_geom(geom) != DAI8_OK) return 0;
+  const ConvShape cs = make_shape(*geom);
+  switch (op) {
+    case DAI8_OP_FWD: return 256;
+    case DAI8_OP_BWD_DATA: return (wt_bytes(cs) + 255) / 256 * 256 + 256;
+    case DAI8_OP_BWD_FILTER: return (dw_acc_bytes(cs) + 255) / 256 * 256 + 256;
+  }
+  return 0;
+}
+
+extern "C" dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                                     const dai8_conv_geom* geom, void* Y, dai8_dtype out_dtype,
+                                     dai8_layout out_layout, void* ws, size_t ws_bytes, void* stream) {
+  (void)ws; (void)ws_bytes;
+  dai8_status g = check_geom(geom);
+  if (g != DAI8_OK) return g;
+  if (!qX || !qW || !Y || bad_out(out_dtype) || bad_layout(out_layout)) return DAI8_ERR_INVALID_ARG;
+  if (out_dtype != DAI8_I32 && (!sX || !sW)) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(qX) || !aligned16(qW) || !aligned16(Y)) return DAI8_ERR_INVALID_ARG;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  const ConvShape cs = make_shape(*geom);
+  const ConvOut out{Y, out_dtype, out_layout};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int mode = g_backend.load();
+  if (mode != 1 && umma_fwd_supported(cs)) return umma_fwd(qX, qW, sX, sW, cs, out, st);
+  if (mode == 2) return DAI8_ERR_UNSUPPORTED;
+  return direct_fwd(qX, qW, sX, sW, cs, out, st);
+}
+
+extern "C" dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, const float* gmax,
+                                          const float* sW, const dai8_conv_geom* geom, void* dX,
+                                          dai8_dtype out_dtype, dai8_layout out_layout, void* ws,
+                                          size_t ws_bytes, void* stream) {
+  dai8_status g = check_geom(geom);
+  if (g != DAI8_OK) return g;
+  if (!gq || !qW || !dX || !ws || bad_out(out_dtype) || bad_layout(out_layout)) return DAI8_ERR_INVALID_ARG;
+  if (out_dtype != DAI8_I32 && (!gmax || !sW)) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(gq) || !aligned16(qW) || !aligned16(dX) || !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (ws_bytes < dai8_conv_workspace_bytes(DAI8_OP_BWD_DATA, geom)) return DAI8_ERR_WORKSPACE;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  const ConvShape cs = make_shape(*geom);
+  const ConvOut out{dX, out_dtype, out_layout};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int8_t* wT = static_cast<int8_t*>(ws);
+  const int mode = g_backend.load();
+  if (mode != 1 && umma_bwd_data_supported(cs)) {
+    dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/1, st);
+    if (r != DAI8_OK) return r;
+    return umma_bwd_data(gq, wT, gmax, sW, cs, out, st);
+  }
+  if (mode == 2) return DAI8_ERR_UNSUPPORTED;
+  dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/0, st);
+  if (r != DAI8_OK) return r;
+  return direct_bwd_data(gq, wT, gmax, sW, cs, out, st);
+}
+
+extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, const float* sX,
+                                            const float* s, const dai8_conv_geom* geom, void* dW,
+                                            dai8_dtype out_dtype, void* ws, size_t ws_bytes,
+                                            void* stream) {
+  dai8_status g = check_geom(geom);
+  if (g != DAI8_OK) return g;
+  if (!qX || !vq || !dW || !ws || bad_out(out_dtype)) return DAI8_ERR_INVALID_ARG;
+  if (out_dtype != DAI8_I32 && (!sX || !s)) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(qX) || !aligned16(vq) || !aligned16(dW) || !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (ws_bytes < dai8_conv_workspace_bytes(DAI8_OP_BWD_FILTER, geom)) return DAI8_ERR_WORKSPACE;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  const ConvShape cs = make_shape(*geom);
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* acc = static_cast<int*>(ws);
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(acc, 0, dw_acc_bytes(cs), st));
+  const int mode = g_backend.load();
+  dai8_status r;
+  if (mode != 1 && umma_bwd_filter_supported(cs)) r = umma_bwd_filter_acc(qX, vq, cs, acc, st);
+  else if (mode == 2) return DAI8_ERR_UNSUPPORTED;
+  else r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
+  if (r != DAI8_OK) return r;
+  return finalize_bwd_filter(acc, sX, s, cs, dW, out_dtype, st);
+}

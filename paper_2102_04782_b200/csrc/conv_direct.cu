@@ -1,0 +1,274 @@
+// Direct int8 convolutions on the CUDA cores (dp4a).  They cover every geometry the boundary
+// accepts (any stride, padding, filter size, channel count) and serve the shapes the tensor-core
+// kernels do not take, e.g. 3-channel stems.  Codes are NHWC with channels padded to 16, so every
+// operand fetch is one 16-byte load and four dp4a.
+#include "conv_internal.cuh"
+
+namespace dai8 {
+namespace {
+
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ int dot16(const uint4& a, const uint4& b, int acc) {
+  acc = __dp4a((int)a.x, (int)b.x, acc);
+  acc = __dp4a((int)a.y, (int)b.y, acc);
+  acc = __dp4a((int)a.z, (int)b.z, acc);
+  acc = __dp4a((int)a.w, (int)b.w, acc);
+  return acc;
+}
+
+// Forward convolution (Fig. 2): thread = (output pixel, output channel), channel fastest.
+__global__ void __launch_bounds__(kThreads)
+direct_fwd_kernel(const int8_t* __restrict__ qX, const int8_t* __restrict__ qW,
+                  const float* __restrict__ sX, const float* __restrict__ sW, ConvShape cs,
+                  ConvOut out) {
+  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * cs.Cout;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int co = (int)(t % cs.Cout);
+  int64_t m = t / cs.Cout;
+  const int q = (int)(m % cs.Q); m /= cs.Q;
+  const int p = (int)(m % cs.P);
+  const int n = (int)(m / cs.P);
+  int acc = 0;
+  for (int r = 0; r < cs.R; ++r) {
+    const int h = p * cs.sh + r - cs.ph;
+    if (h < 0 || h >= cs.H) continue;
+    for (int s = 0; s < cs.S; ++s) {
+      const int w = q * cs.sw + s - cs.pw;
+      if (w < 0 || w >= cs.W) continue;
+      const uint4* xa = reinterpret_cast<const uint4*>(qX + (((int64_t)n * cs.H + h) * cs.W + w) * cs.Cinp);
+      const uint4* wa = reinterpret_cast<const uint4*>(qW + (((int64_t)co * cs.R + r) * cs.S + s) * cs.Cinp);
+      for (int k = 0; k < cs.Cinp / 16; ++k) acc = dot16(__ldg(xa + k), __ldg(wa + k), acc);
+    }
+  }
+  const float scale = out.dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, *sW);
+  const size_t pix = ((size_t)n * cs.P + p) * cs.Q + q;
+  const size_t idx = out.layout == DAI8_NHWC ? pix * cs.Cout + co
+                                             : (((size_t)n * cs.Cout + co) * cs.P + p) * cs.Q + q;
+  store_result(out.ptr, out.dtype, idx, acc, scale);
+}
+
+// Input gradient (Eq. 3): thread = (input pixel, input channel); gathers the output positions
+// (p, q) with h = p*stride + r - pad, w = q*stride + s - pad.
+__global__ void __launch_bounds__(kThreads)
+direct_bwd_data_kernel(const int8_t* __restrict__ gq, const int8_t* __restrict__ wT,
+                       const float* __restrict__ gmax, const float* __restrict__ sW, ConvShape cs,
+                       ConvOut out) {
+  const int64_t total = (int64_t)cs.N * cs.H * cs.W * cs.Cin;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int ci = (int)(t % cs.Cin);
+  int64_t m = t / cs.Cin;
+  const int w = (int)(m % cs.W); m /= cs.W;
+  const int h = (int)(m % cs.H);
+  const int n = (int)(m / cs.H);
+  int acc = 0;
+  for (int r = 0; r < cs.R; ++r) {
+    const int hp = h + cs.ph - r;
+    if (hp < 0 || hp % cs.sh != 0) continue;
+    const int p = hp / cs.sh;
+    if (p >= cs.P) continue;
+    for (int s = 0; s < cs.S; ++s) {
+      const int wq = w + cs.pw - s;
+      if (wq < 0 || wq % cs.sw != 0) continue;
+      const int q = wq / cs.sw;
+      if (q >= cs.Q) continue;
+      const uint4* ga = reinterpret_cast<const uint4*>(gq + (((int64_t)n * cs.P + p) * cs.Q + q) * cs.Coutp);
+      const uint4* wa = reinterpret_cast<const uint4*>(wT + (((int64_t)ci * cs.R + r) * cs.S + s) * cs.Coutp);
+      for (int k = 0; k < cs.Coutp / 16; ++k) acc = dot16(__ldg(ga + k), __ldg(wa + k), acc);
+    }
+  }
+  const float scale = out.dtype == DAI8_I32 ? 0.f : dequant_scale(*gmax, *sW);
+  const size_t pix = ((size_t)n * cs.H + h) * cs.W + w;
+  const size_t idx = out.layout == DAI8_NHWC ? pix * cs.Cin + ci
+                                             : (((size_t)n * cs.Cin + ci) * cs.H + h) * cs.W + w;
+  store_result(out.ptr, out.dtype, idx, acc, scale);
+}
+
+// Weight gradient (Eq. 4).  A warp owns an 8 (co) x 16 (ci) tile of one filter tap and a range of
+// output pixels; each lane takes groups of four consecutive pixels, transposes their codes so that
+// one 32-bit word holds the four pixels of one channel, and accumulates with dp4a.  Partial sums
+// are reduced across the warp and added to acc[Cout][R][S][Cinp] with integer atomics (exact in
+// any order).
+constexpr int kDwCo = 8, kDwCi = 16, kDwWarps = 4;
+
+__device__ __forceinline__ uint32_t gather_byte4(uint32_t p0, uint32_t p1, uint32_t p2, uint32_t p3, int b) {
+  const uint32_t sel = (uint32_t)b | ((uint32_t)(4 + b) << 4);
+  const uint32_t lo = __byte_perm(p0, p1, sel);
+  const uint32_t hi = __byte_perm(p2, p3, sel);
+  return __byte_perm(lo, hi, 0x5410);
+}
+
+__global__ void __launch_bounds__(kDwWarps * 32)
+direct_bwd_filter_kernel(const int8_t* __restrict__ qX, const int8_t* __restrict__ vq, ConvShape cs,
+                         int* __restrict__ acc_out, int ksplit) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int tile = blockIdx.x;
+  const int ci_tiles = cs.Cinp / kDwCi;
+  const int ci0 = (tile % ci_tiles) * kDwCi; tile /= ci_tiles;
+  const int s = tile % cs.S; tile /= cs.S;
+  const int r = tile % cs.R; tile /= cs.R;
+  const int co0 = tile * kDwCo;
+
+  const int64_t npix = (int64_t)cs.N * cs.P * cs.Q;
+  const int64_t nquads = (npix + 3) / 4;
+  const int64_t parts = (int64_t)ksplit * kDwWarps;
+  const int64_t per = (nquads + parts - 1) / parts;
+  const int64_t qbeg = ((int64_t)blockIdx.y * kDwWarps + warp) * per;
+  const int64_t qend = min(nquads, qbeg + per);
+
+  int acc[kDwCo][kDwCi];
+#pragma unroll
+  for (int i = 0; i < kDwCo; ++i)
+#pragma unroll
+    for (int j = 0; j < kDwCi; ++j) acc[i][j] = 0;
+
+  for (int64_t qd = qbeg + lane; qd < qend; qd += 32) {
+    uint2 g[4];   // 8 co codes of each of the 4 pixels
+    uint4 x[4];   // 16 ci codes
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      const int64_t pix = qd * 4 + k;
+      g[k] = make_uint2(0u, 0u);
+      x[k] = make_uint4(0u, 0u, 0u, 0u);
+      if (pix < npix) {
+        const int q = (int)(pix % cs.Q);
+        const int64_t t = pix / cs.Q;
+        const int p = (int)(t % cs.P);
+        const int n = (int)(t / cs.P);
+        const int h = p * cs.sh + r - cs.ph, w = q * cs.sw + s - cs.pw;
+        if (h >= 0 && h < cs.H && w >= 0 && w < cs.W) {
+          g[k] = __ldg(reinterpret_cast<const uint2*>(vq + pix * cs.Coutp + co0));
+          x[k] = __ldg(reinterpret_cast<const uint4*>(qX + (((int64_t)n * cs.H + h) * cs.W + w) * cs.Cinp + ci0));
+        }
+      }
+    }
+    uint32_t gw[kDwCo], xw[kDwCi];
+#pragma unroll
+    for (int b = 0; b < 4; ++b) {
+      gw[b] = gather_byte4(g[0].x, g[1].x, g[2].x, g[3].x, b);
+      gw[4 + b] = gather_byte4(g[0].y, g[1].y, g[2].y, g[3].y, b);
+      xw[b] = gather_byte4(x[0].x, x[1].x, x[2].x, x[3].x, b);
+      xw[4 + b] = gather_byte4(x[0].y, x[1].y, x[2].y, x[3].y, b);
+      xw[8 + b] = gather_byte4(x[0].z, x[1].z, x[2].z, x[3].z, b);
+      xw[12 + b] = gather_byte4(x[0].w, x[1].w, x[2].w, x[3].w, b);
+    }
+#pragma unroll
+    for (int i = 0; i < kDwCo; ++i)
+#pragma unroll
+      for (int j = 0; j < kDwCi; ++j) acc[i][j] = __dp4a((int)gw[i], (int)xw[j], acc[i][j]);
+  }
+
+#pragma unroll
+  for (int i = 0; i < kDwCo; ++i)
+#pragma unroll
+    for (int j = 0; j < kDwCi; ++j) {
+      int v = acc[i][j];
+      for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+      acc[i][j] = v;
+    }
+  if (lane == 0) {
+#pragma unroll
+    for (int i = 0; i < kDwCo; ++i) {
+      const int co = co0 + i;
+      if (co >= cs.Cout) continue;
+#pragma unroll
+      for (int j = 0; j < kDwCi; ++j)
+        if (acc[i][j] != 0)
+          atomicAdd(acc_out + (((int64_t)co * cs.R + r) * cs.S + s) * cs.Cinp + ci0 + j, acc[i][j]);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kThreads)
+repack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int8_t* __restrict__ wT, int flip) {
+  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int co = (int)(t % cs.Coutp);
+  int64_t m = t / cs.Coutp;
+  const int s = (int)(m % cs.S); m /= cs.S;
+  const int r = (int)(m % cs.R);
+  const int ci = (int)(m / cs.R);
+  const int rs = flip ? cs.R - 1 - r : r, ss = flip ? cs.S - 1 - s : s;
+  int8_t v = 0;
+  if (co < cs.Cout) v = qW[(((int64_t)co * cs.R + rs) * cs.S + ss) * cs.Cinp + ci];  // ci >= Cin holds 0
+  wT[t] = v;
+}
+
+__global__ void __launch_bounds__(kThreads)
+finalize_bwd_filter_kernel(const int* __restrict__ acc, const float* __restrict__ sX,
+                           const float* __restrict__ s, ConvShape cs, void* __restrict__ dW,
+                           dai8_dtype dtype) {
+  const int64_t total = (int64_t)cs.Cout * cs.Cin * cs.R * cs.S;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int ss = (int)(t % cs.S);
+  int64_t m = t / cs.S;
+  const int r = (int)(m % cs.R); m /= cs.R;
+  const int ci = (int)(m % cs.Cin);
+  const int co = (int)(m / cs.Cin);
+  const int a = acc[(((int64_t)co * cs.R + r) * cs.S + ss) * cs.Cinp + ci];
+  const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
+  store_result(dW, dtype, (size_t)t, a, scale);
+}
+
+unsigned blocks_for(int64_t total) { return (unsigned)ceil_div64(total, kThreads); }
+
+}  // namespace
+
+dai8_status direct_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                       const ConvShape& cs, const ConvOut& out, cudaStream_t st) {
+  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * cs.Cout;
+  direct_fwd_kernel<<<blocks_for(total), kThreads, 0, st>>>(qX, qW, sX, sW, cs, out);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status direct_bwd_data(const int8_t* gq, const int8_t* wT, const float* gmax, const float* sW,
+                            const ConvShape& cs, const ConvOut& out, cudaStream_t st) {
+  const int64_t total = (int64_t)cs.N * cs.H * cs.W * cs.Cin;
+  direct_bwd_data_kernel<<<blocks_for(total), kThreads, 0, st>>>(gq, wT, gmax, sW, cs, out);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status direct_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc,
+                                  cudaStream_t st) {
+  const int64_t tiles = (int64_t)(cs.Coutp / kDwCo) * cs.R * cs.S * (cs.Cinp / kDwCi);
+  const int64_t nquads = ((int64_t)cs.N * cs.P * cs.Q + 3) / 4;
+  // enough blocks to fill the machine a few times, at least 8 quads per lane
+  int64_t ksplit = ceil_div64(148 * 16, tiles);
+  const int64_t kmax = ceil_div64(nquads, (int64_t)kDwWarps * 32 * 8);
+  if (ksplit > kmax) ksplit = kmax;
+  if (ksplit < 1) ksplit = 1;
+  if (ksplit > 65535) ksplit = 65535;
+  direct_bwd_filter_kernel<<<dim3((unsigned)tiles, (unsigned)ksplit), kDwWarps * 32, 0, st>>>(
+      qX, vq, cs, acc, (int)ksplit);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int8_t* wT, int flip,
+                                      cudaStream_t st) {
+  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;
+  repack_weights_kernel<<<blocks_for(total), kThreads, 0, st>>>(qW, cs, wT, flip);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status finalize_bwd_filter(const int* acc, const float* sX, const float* s, const ConvShape& cs,
+                                void* dW, dai8_dtype dtype, cudaStream_t st) {
+  const int64_t total = (int64_t)cs.Cout * cs.Cin * cs.R * cs.S;
+  finalize_bwd_filter_kernel<<<blocks_for(total), kThreads, 0, st>>>(acc, sX, s, cs, dW, dtype);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+}  // namespace dai8

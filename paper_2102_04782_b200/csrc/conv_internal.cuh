@@ -1,0 +1,81 @@
+// Interfaces shared by the convolution kernel families and the C-ABI dispatch (conv_api.cu).
+#pragma once
+
+#include "dai8_common.cuh"
+
+namespace dai8 {
+
+struct ConvShape {
+  int N, Cin, Cout, H, W, R, S, sh, sw, ph, pw;
+  int P, Q;        // output extent
+  int Cinp, Coutp; // channel counts of the code tensors (multiples of 16)
+};
+
+inline ConvShape make_shape(const dai8_conv_geom& g) {
+  ConvShape s;
+  s.N = g.N; s.Cin = g.Cin; s.Cout = g.Cout; s.H = g.H; s.W = g.W; s.R = g.R; s.S = g.S;
+  s.sh = g.stride_h; s.sw = g.stride_w; s.ph = g.pad_h; s.pw = g.pad_w;
+  s.P = (g.H + 2 * g.pad_h - g.R) / g.stride_h + 1;
+  s.Q = (g.W + 2 * g.pad_w - g.S) / g.stride_w + 1;
+  s.Cinp = round_up(g.Cin, 16);
+  s.Coutp = round_up(g.Cout, 16);
+  return s;
+}
+
+struct ConvOut {
+  void* ptr;
+  dai8_dtype dtype;    // F32, BF16 or I32 (raw accumulators)
+  dai8_layout layout;  // NCHW or NHWC (C unpadded)
+};
+
+// De-quantization scale (Eq. 7 and Algorithm 1 lines 14-15): (a/127)*(b/127), each step rounded.
+__device__ __forceinline__ float dequant_scale(float a, float b) {
+  return __fmul_rn(__fdiv_rn(a, 127.0f), __fdiv_rn(b, 127.0f));
+}
+
+__device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {
+  const uint32_t u = __float_as_uint(f);
+  if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((u >> 16) | 0x40u);  // NaN
+  return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);                  // nearest even
+}
+
+// Writes one output element: the raw accumulator, or float(acc)*scale as fp32 / bf16.
+__device__ __forceinline__ void store_result(void* out, dai8_dtype dtype, size_t idx, int acc, float scale) {
+  if (dtype == DAI8_I32) {
+    static_cast<int*>(out)[idx] = acc;
+  } else {
+    const float v = __fmul_rn(__int2float_rn(acc), scale);
+    if (dtype == DAI8_F32) static_cast<float*>(out)[idx] = v;
+    else static_cast<uint16_t*>(out)[idx] = f32_to_bf16_bits(v);
+  }
+}
+
+// ---- direct (CUDA-core, dp4a) kernels: every geometry --------------------------------------------
+dai8_status direct_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                       const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+// wT: weights repacked as [Cinp][R][S][Coutp] (repack_weights_transposed, flip = 0)
+dai8_status direct_bwd_data(const int8_t* gq, const int8_t* wT, const float* gmax, const float* sW,
+                            const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+// accumulates into acc[Cout][R][S][Cinp] (int32, zeroed by the caller)
+dai8_status direct_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc,
+                                  cudaStream_t st);
+
+// [Cout][R][S][Cinp] -> [Cinp][R][S][Coutp]; flip != 0 also mirrors the taps (r,s) -> (R-1-r,S-1-s).
+dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int8_t* wT, int flip,
+                                      cudaStream_t st);
+// acc[Cout][R][S][Cinp] -> dW (Cout,Cin,R,S), scaled by (sX/127)(s[co]/127) unless dtype is I32.
+dai8_status finalize_bwd_filter(const int* acc, const float* sX, const float* s, const ConvShape& cs,
+                                void* dW, dai8_dtype dtype, cudaStream_t st);
+
+// ---- tensor-core (tcgen05) kernels: see conv_umma.cu for the geometries covered ------------------
+bool umma_fwd_supported(const ConvShape& cs);
+bool umma_bwd_data_supported(const ConvShape& cs);
+bool umma_bwd_filter_supported(const ConvShape& cs);
+dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                     const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* gmax, const float* sW,
+                          const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc,
+                                cudaStream_t st);
+
+}  // namespace dai8

@@ -1,0 +1,104 @@
+// Shared host/device helpers of libdai8 (CUDA side only; the CPU oracle shares nothing with this).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+#include "../../include/dai8.h"
+
+namespace dai8 {
+
+// bfloat16 values travel as their 16-bit patterns; widening to binary32 is exact.
+struct bf16_t {
+  uint16_t bits;
+};
+
+extern std::atomic<uint64_t> g_launch_count;
+inline void note_launch(int n = 1) { g_launch_count.fetch_add((uint64_t)n, std::memory_order_relaxed); }
+
+// Reads and clears the device status word kept beside the tensor-core kernels (conv_umma.cu).
+dai8_status read_clear_device_status(int* host_status, cudaStream_t stream);
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+#define DAI8_RETURN_IF_CUDA(expr)                 \
+  do {                                            \
+    cudaError_t e__ = (expr);                     \
+    if (e__ != cudaSuccess) return DAI8_ERR_CUDA; \
+  } while (0)
+
+// DAI8_OK if the current device is compute capability 10.x, else DAI8_ERR_ARCH / DAI8_ERR_CUDA.
+dai8_status check_device_arch();
+
+__device__ __forceinline__ float to_f32(float v) { return v; }
+__device__ __forceinline__ float to_f32(bf16_t v) { return __uint_as_float((uint32_t)v.bits << 16); }
+
+// Loads VE consecutive elements (VE*sizeof(T) is 16 bytes, or VE == 1) and widens them to fp32.
+template <typename T, int VE>
+__device__ __forceinline__ void load_vec(const T* p, float (&v)[VE]);
+
+template <>
+__device__ __forceinline__ void load_vec<float, 4>(const float* p, float (&v)[4]) {
+  const float4 t = *reinterpret_cast<const float4*>(p);
+  v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+}
+template <>
+__device__ __forceinline__ void load_vec<float, 1>(const float* p, float (&v)[1]) { v[0] = *p; }
+template <>
+__device__ __forceinline__ void load_vec<bf16_t, 8>(const bf16_t* p, float (&v)[8]) {
+  const uint4 t = *reinterpret_cast<const uint4*>(p);
+  const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    v[2 * i] = __uint_as_float(w[i] << 16);
+    v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+  }
+}
+template <>
+__device__ __forceinline__ void load_vec<bf16_t, 1>(const bf16_t* p, float (&v)[1]) {
+  v[0] = to_f32(*p);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Counter-based uniform numbers for stochastic rounding (the paper names the rounding mode in
+// Sec. 3 but no generator).  A 32-bit avalanche finaliser (xor-shift 16, multiply, xor-shift 13,
+// multiply, xor-shift 16) is applied to the low half of the element's NCHW index xor a key that
+// mixes the seed with the high half.  Stream 0 uses the hash, stream 1 the hash times an odd
+// constant.  u = (top 23 bits) * 2^-23.
+// ------------------------------------------------------------------------------------------------
+__host__ __device__ __forceinline__ uint32_t avalanche32(uint32_t h) {
+  h ^= h >> 16;
+  h *= 0x85EBCA6Bu;
+  h ^= h >> 13;
+  h *= 0xC2B2AE35u;
+  h ^= h >> 16;
+  return h;
+}
+__host__ __device__ __forceinline__ uint32_t sr_key(uint32_t seed, uint32_t index_hi) {
+  return avalanche32(seed ^ (0x9E3779B9u * (index_hi + 1u)));
+}
+__device__ __forceinline__ float sr_uniform(uint32_t h) {
+  return __uint_as_float(0x3F800000u | (h >> 9)) - 1.0f;  // exact: (h >> 9) * 2^-23
+}
+
+// Eq. 1 on one element, given inv = 127/s (0 when s <= 0).  The operation order (multiply, clamp,
+// then round) and the absence of fused multiply-add are part of the definition: codes must be
+// reproducible bit for bit.
+__device__ __forceinline__ int quant_nearest(float x, float inv) {
+  float v = __fmul_rn(x, inv);
+  v = fminf(fmaxf(v, -127.0f), 127.0f);
+  return __float2int_rn(v);
+}
+__device__ __forceinline__ int quant_stochastic(float x, float inv, float u) {
+  float v = __fmul_rn(x, inv);
+  v = fminf(fmaxf(v, -127.0f), 127.0f);
+  const int q = __float2int_rd(__fadd_rn(v, u));
+  return min(q, 127);
+}
+__device__ __forceinline__ float inv_scale(float s) { return s > 0.0f ? __fdiv_rn(127.0f, s) : 0.0f; }
+
+}  // namespace dai8

@@ -1,0 +1,731 @@
+// Gradient Vectorized Quantization with the Magnitude-aware Clipping Strategy (Algorithm 1,
+// lines 1-11) and the layer-wide quantizer of the forward pass (Eq. 1), as HBM-bound kernels.
+//
+// Three sweeps over dY, because each needs a per-channel scalar the previous one produces:
+//   1. stats   : |g|max,c, sum, sum of squares  -> mean, sigma          (Alg. 1 line 2)
+//   2. count   : #{|g| > sigma_c}                -> class, clip s_c      (Alg. 1 lines 4-9, Eq. 14/15)
+//   3. quantize: vq (per-channel s_c) and gq (layer |g|max) in one pass (Alg. 1 lines 10-11)
+// The last block of sweeps 1 and 2 (found with a ticket counter) finishes the per-channel
+// scalars, so no separate tiny launches are needed.  Floating-point sums are combined in a
+// fixed order (per-block partials, then a fixed tree), so results do not depend on scheduling;
+// max and the density count use integer atomics, which are order-independent.
+//
+// Layouts.  The native layout is NHWC: a thread owns one 16-byte vector of channels
+// (4 fp32 / 8 bf16) of one pixel and walks down the pixels, so per-channel scalars stay in
+// registers and every load/store instruction of a warp covers contiguous memory.  NCHW inputs are
+// read along H*W per (n, c) row and transposed through shared memory when codes are written.
+#include "dai8_common.cuh"
+
+namespace dai8 {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kMaxPixelBlocks = 592;  // 4 blocks on each of 148 SMs
+
+struct GvqWs {
+  uint32_t* tickets;    // [C] arrival counters of the stats sweep (per column block / channel)
+  uint32_t* ticket2;    // [1] arrival counter of the count sweep
+  uint32_t* cnt;        // [C] density counts
+  uint32_t* gmax_bits;  // [1] layer |g|max as the bit pattern of a non-negative float
+  float* absmax;        // [C]
+  float* mean;          // [C]
+  float* sigma;         // [C]
+  float* pmax;          // [PB][C] per-block partial max
+  double* psum;         // [PB][C]
+  double* pss;          // [PB][C]
+};
+
+size_t control_words(int C) { return (size_t)2 * C + 4; }
+
+size_t ws_bytes_for(int C) {
+  size_t b = control_words(C) * 4;
+  b = (b + 15) / 16 * 16;
+  b += (size_t)3 * C * 4;
+  b = (b + 15) / 16 * 16;
+  b += (size_t)kMaxPixelBlocks * C * (4 + 8 + 8);
+  return b + 64;
+}
+
+GvqWs carve(void* ws, int C) {
+  GvqWs w;
+  char* p = static_cast<char*>(ws);
+  w.tickets = reinterpret_cast<uint32_t*>(p);
+  w.ticket2 = w.tickets + C;
+  w.cnt = w.ticket2 + 1;
+  w.gmax_bits = w.cnt + C;
+  size_t off = (control_words(C) * 4 + 15) / 16 * 16;
+  w.absmax = reinterpret_cast<float*>(p + off);
+  w.mean = w.absmax + C;
+  w.sigma = w.mean + C;
+  off += (size_t)3 * C * 4;
+  off = (off + 15) / 16 * 16;
+  w.psum = reinterpret_cast<double*>(p + off);
+  w.pss = w.psum + (size_t)kMaxPixelBlocks * C;
+  w.pmax = reinterpret_cast<float*>(w.pss + (size_t)kMaxPixelBlocks * C);
+  return w;
+}
+
+struct McsDev {
+  float lambda, k, A;
+  int std_unbiased, center_mean;
+};
+
+// mean and sigma of one channel from the moments of d = g - pivot (binary64).  The pivot (the
+// channel's first element) keeps sum d^2 - (sum d)^2/M free of cancellation when |mean| >> sigma.
+__device__ __forceinline__ void finish_moments(double pivot, double s1, double s2, int64_t M,
+                                               const McsDev& mp, float* mean, float* sigma) {
+  const double md = s1 / (double)M;
+  double var = mp.center_mean ? (s2 - s1 * md)                                  // sum (g-mu)^2
+                              : (s2 + 2.0 * pivot * s1 + (double)M * pivot * pivot);  // sum g^2
+  if (var < 0.0) var = 0.0;
+  const double denom = mp.std_unbiased ? (double)(M - 1) : (double)M;
+  *mean = (float)(pivot + md);
+  *sigma = denom > 0.0 ? (float)sqrt(var / denom) : 0.0f;
+}
+
+// Returns true in every thread of the one block that arrives last at `ticket`.
+__device__ __forceinline__ bool last_block_arrives(uint32_t* ticket, uint32_t expected) {
+  __shared__ uint32_t s_last;
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = (atomicAdd(ticket, 1u) == expected - 1u) ? 1u : 0u;
+  __syncthreads();
+  const bool last = s_last != 0u;
+  if (last) __threadfence();
+  return last;
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sweep 1, NHWC.  grid = (pixel blocks, column blocks of up to 256 vectors).
+// ------------------------------------------------------------------------------------------------
+template <typename T, int VE>
+__global__ void __launch_bounds__(kThreads)
+stats_nhwc_kernel(const T* __restrict__ x, int64_t npix, int C, int G, GvqWs ws, McsDev mp,
+                  float* __restrict__ stats_out) {
+  __shared__ double sred[kThreads * VE];
+  const int tid = threadIdx.x;
+  const int colv0 = blockIdx.y * kThreads;
+  const int gcols = min(G - colv0, kThreads);
+  const int rpi = kThreads / gcols;
+  const int col = tid % gcols, rl = tid / gcols;
+  const int64_t chunk = (npix + gridDim.x - 1) / gridDim.x;
+  const int64_t p0 = (int64_t)blockIdx.x * chunk;
+  const int64_t p1 = min(npix, p0 + chunk);
+
+  float amax[VE], fs[VE], fss[VE];
+  double ds[VE], dss[VE];
+#pragma unroll
+  for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; ds[e] = 0.0; dss[e] = 0.0; }
+
+  if (rl < rpi) {
+    const T* base = x + (int64_t)(colv0 + col) * VE;
+    float piv[VE];
+    load_vec<T, VE>(base, piv);  // pixel 0 of these channels
+    int it = 0;
+    for (int64_t p = p0 + rl; p < p1; p += rpi) {
+      float v[VE];
+      load_vec<T, VE>(base + p * C, v);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) {
+        amax[e] = fmaxf(amax[e], fabsf(v[e]));
+        const float d = v[e] - piv[e];
+        fs[e] += d;
+        fss[e] = fmaf(d, d, fss[e]);
+      }
+      if (++it == 32) {  // short fp32 runs, combined in binary64
+        it = 0;
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; }
+  }
+
+  const int nch = gcols * VE;             // channels of this column block
+  const int c0 = colv0 * VE;
+  const size_t prow = (size_t)blockIdx.x * C + c0;
+  // three fixed-order reductions over the rpi row lanes
+  for (int pass = 0; pass < 3; ++pass) {
+    __syncthreads();
+#pragma unroll
+    for (int e = 0; e < VE; ++e)
+      sred[tid * VE + e] = pass == 0 ? (double)amax[e] : (pass == 1 ? ds[e] : dss[e]);
+    __syncthreads();
+    for (int j = tid; j < nch; j += kThreads) {
+      const int cc = j / VE, e = j % VE;
+      double acc = 0.0;
+      if (pass == 0) {
+        for (int r = 0; r < rpi; ++r) acc = fmax(acc, sred[(r * gcols + cc) * VE + e]);
+        ws.pmax[prow + j] = (float)acc;
+      } else {
+        for (int r = 0; r < rpi; ++r) acc += sred[(r * gcols + cc) * VE + e];
+        (pass == 1 ? ws.psum : ws.pss)[prow + j] = acc;
+      }
+    }
+  }
+
+  if (!last_block_arrives(ws.tickets + blockIdx.y, gridDim.x)) return;
+
+  // Last block of this column block: combine the per-block partials, channel by channel.
+  const int PB = gridDim.x;
+  const int nparts = nch >= kThreads ? 1 : kThreads / nch;
+  const int64_t M = npix;
+  float* smax = reinterpret_cast<float*>(sred);  // reuse: [kThreads] floats + 2*[kThreads] doubles
+  __shared__ double ssum[kThreads], sss[kThreads];
+  float block_max = 0.f;
+  for (int cbase = 0; cbase < nch; cbase += kThreads) {
+    const int j = (nparts == 1) ? cbase + tid : tid % nch;
+    const int part = (nparts == 1) ? 0 : tid / nch;
+    float m = 0.f;
+    double s = 0.0, q = 0.0;
+    if (j < nch && part < nparts) {
+      for (int pb = part; pb < PB; pb += nparts) {
+        const size_t idx = (size_t)pb * C + c0 + j;
+        m = fmaxf(m, __ldcg(ws.pmax + idx));
+        s += __ldcg(ws.psum + idx);
+        q += __ldcg(ws.pss + idx);
+      }
+    }
+    __syncthreads();
+    smax[tid] = m; ssum[tid] = s; sss[tid] = q;
+    __syncthreads();
+    if (j < nch && part == 0) {
+      for (int r = 1; r < nparts; ++r) {
+        m = fmaxf(m, smax[r * nch + j]);
+        s += ssum[r * nch + j];
+        q += sss[r * nch + j];
+      }
+      float mean, sigma;
+      const int c = c0 + j;
+      finish_moments((double)to_f32(x[c]), s, q, M, mp, &mean, &sigma);
+      ws.absmax[c] = m; ws.mean[c] = mean; ws.sigma[c] = sigma;
+      if (stats_out) {
+        stats_out[c * 4 + DAI8_STAT_ABSMAX] = m;
+        stats_out[c * 4 + DAI8_STAT_MEAN] = mean;
+        stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
+      }
+      block_max = fmaxf(block_max, m);
+    }
+  }
+  // layer |g|max: non-negative floats order like their bit patterns
+  for (int o = 16; o > 0; o >>= 1) block_max = fmaxf(block_max, __shfl_xor_sync(0xFFFFFFFFu, block_max, o));
+  if ((tid & 31) == 0 && block_max > 0.f) atomicMax(ws.gmax_bits, __float_as_uint(block_max));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sweep 1, NCHW.  grid = (C, slices over n).  Each block reduces rows (n, c, :) of one channel.
+// ------------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+stats_nchw_kernel(const T* __restrict__ x, int N, int C, int64_t HW, GvqWs ws, McsDev mp,
+                  float* __restrict__ stats_out) {
+  const int c = blockIdx.x, tid = threadIdx.x;
+  const int NS = gridDim.y;
+  const int nper = (N + NS - 1) / NS;
+  const int n0 = blockIdx.y * nper, n1 = min(N, n0 + nper);
+  float amax = 0.f;
+  double ds = 0.0, dss = 0.0;
+  const float piv = to_f32(x[(int64_t)c * HW]);  // element (0, c, 0, 0)
+  for (int n = n0; n < n1; ++n) {
+    const T* row = x + ((int64_t)n * C + c) * HW;
+    float fs = 0.f, fss = 0.f;
+    int it = 0;
+    for (int64_t i = tid; i < HW; i += kThreads) {
+      const float v = to_f32(row[i]);
+      amax = fmaxf(amax, fabsf(v));
+      const float d = v - piv;
+      fs += d;
+      fss = fmaf(d, d, fss);
+      if (++it == 32) { it = 0; ds += (double)fs; dss += (double)fss; fs = 0.f; fss = 0.f; }
+    }
+    ds += (double)fs; dss += (double)fss;
+  }
+  __shared__ float smax[kThreads];
+  __shared__ double ssum[kThreads], sss[kThreads];
+  smax[tid] = amax; ssum[tid] = ds; sss[tid] = dss;
+  __syncthreads();
+  for (int o = kThreads / 2; o > 0; o >>= 1) {  // fixed tree
+    if (tid < o) {
+      smax[tid] = fmaxf(smax[tid], smax[tid + o]);
+      ssum[tid] += ssum[tid + o];
+      sss[tid] += sss[tid + o];
+    }
+    __syncthreads();
+  }
+  if (tid == 0) {
+    const size_t idx = (size_t)blockIdx.y * C + c;
+    ws.pmax[idx] = smax[0]; ws.psum[idx] = ssum[0]; ws.pss[idx] = sss[0];
+  }
+  if (!last_block_arrives(ws.tickets + c, NS)) return;
+  if (tid == 0) {
+    float m = 0.f;
+    double s = 0.0, q = 0.0;
+    for (int pb = 0; pb < NS; ++pb) {
+      const size_t idx = (size_t)pb * C + c;
+      m = fmaxf(m, __ldcg(ws.pmax + idx));
+      s += __ldcg(ws.psum + idx);
+      q += __ldcg(ws.pss + idx);
+    }
+    float mean, sigma;
+    finish_moments((double)piv, s, q, (int64_t)N * HW, mp, &mean, &sigma);
+    ws.absmax[c] = m; ws.mean[c] = mean; ws.sigma[c] = sigma;
+    if (stats_out) {
+      stats_out[c * 4 + DAI8_STAT_ABSMAX] = m;
+      stats_out[c * 4 + DAI8_STAT_MEAN] = mean;
+      stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
+    }
+    if (m > 0.f) atomicMax(ws.gmax_bits, __float_as_uint(m));
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Algorithm 1 lines 5-9 for every channel, by the last block of the count sweep.
+//   P > lambda (cnt > lambda*M in binary64): s = |g|max,c                       (Eq. 11)
+//   otherwise: s = (1 - k*A)*s_prev + A*|g|max,c, each operation rounded to fp32  (Eq. 14)
+// ------------------------------------------------------------------------------------------------
+__device__ void solve_channels(const GvqWs& ws, int C, int64_t M, const McsDev& mp,
+                               float* __restrict__ s_state, int has_prev,
+                               float* __restrict__ gmax_layer, float* __restrict__ stats_out,
+                               uint8_t* __restrict__ cls) {
+  const float t = __fsub_rn(1.0f, __fmul_rn(mp.k, mp.A));
+  for (int c = threadIdx.x; c < C; c += blockDim.x) {
+    const uint32_t cnt = __ldcg(ws.cnt + c);
+    const float gmax = __ldcg(ws.absmax + c);
+    const bool bell = (double)cnt > (double)mp.lambda * (double)M;
+    float s;
+    if (bell) {
+      s = gmax;
+    } else {
+      const float s_prev = has_prev ? s_state[c] : gmax;
+      s = __fadd_rn(__fmul_rn(t, s_prev), __fmul_rn(mp.A, gmax));
+    }
+    s_state[c] = s;
+    if (cls) cls[c] = bell ? 1 : 0;
+    if (stats_out) stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt / (double)M);
+  }
+  if (threadIdx.x == 0) *gmax_layer = __uint_as_float(__ldcg(ws.gmax_bits));
+}
+
+// Sweep 2, NHWC.  grid = (pixel blocks, column blocks).
+template <typename T, int VE>
+__global__ void __launch_bounds__(kThreads)
+count_nhwc_kernel(const T* __restrict__ x, int64_t npix, int C, int G, GvqWs ws,
+                  const float* __restrict__ sigma, McsDev mp, float* __restrict__ s_state,
+                  int has_prev, float* __restrict__ gmax_layer, float* __restrict__ stats_out,
+                  uint8_t* __restrict__ cls) {
+  __shared__ uint32_t scnt[kThreads * VE];
+  const int tid = threadIdx.x;
+  const int colv0 = blockIdx.y * kThreads;
+  const int gcols = min(G - colv0, kThreads);
+  const int rpi = kThreads / gcols;
+  const int col = tid % gcols, rl = tid / gcols;
+  const int64_t chunk = (npix + gridDim.x - 1) / gridDim.x;
+  const int64_t p0 = (int64_t)blockIdx.x * chunk;
+  const int64_t p1 = min(npix, p0 + chunk);
+  uint32_t k[VE];
+#pragma unroll
+  for (int e = 0; e < VE; ++e) k[e] = 0;
+  if (rl < rpi) {
+    float sg[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) sg[e] = sigma[(colv0 + col) * VE + e];
+    const T* base = x + (int64_t)(colv0 + col) * VE;
+    for (int64_t p = p0 + rl; p < p1; p += rpi) {
+      float v[VE];
+      load_vec<T, VE>(base + p * C, v);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < VE; ++e) scnt[tid * VE + e] = k[e];
+  __syncthreads();
+  const int nch = gcols * VE;
+  for (int j = tid; j < nch; j += kThreads) {
+    const int cc = j / VE, e = j % VE;
+    uint32_t acc = 0;
+    for (int r = 0; r < rpi; ++r) acc += scnt[(r * gcols + cc) * VE + e];
+    if (acc) atomicAdd(ws.cnt + colv0 * VE + j, acc);
+  }
+  if (!last_block_arrives(ws.ticket2, gridDim.x * gridDim.y)) return;
+  solve_channels(ws, C, npix, mp, s_state, has_prev, gmax_layer, stats_out, cls);
+}
+
+// Sweep 2, NCHW.  grid = (C, slices over n).
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+count_nchw_kernel(const T* __restrict__ x, int N, int C, int64_t HW, GvqWs ws,
+                  const float* __restrict__ sigma, McsDev mp, float* __restrict__ s_state,
+                  int has_prev, float* __restrict__ gmax_layer, float* __restrict__ stats_out,
+                  uint8_t* __restrict__ cls) {
+  const int c = blockIdx.x, tid = threadIdx.x;
+  const int NS = gridDim.y;
+  const int nper = (N + NS - 1) / NS;
+  const int n0 = blockIdx.y * nper, n1 = min(N, n0 + nper);
+  const float sg = sigma[c];
+  uint32_t k = 0;
+  for (int n = n0; n < n1; ++n) {
+    const T* row = x + ((int64_t)n * C + c) * HW;
+    for (int64_t i = tid; i < HW; i += kThreads) k += (fabsf(to_f32(row[i])) > sg) ? 1u : 0u;
+  }
+  for (int o = 16; o > 0; o >>= 1) k += __shfl_xor_sync(0xFFFFFFFFu, k, o);
+  if ((tid & 31) == 0 && k) atomicAdd(ws.cnt + c, k);
+  if (!last_block_arrives(ws.ticket2, gridDim.x * gridDim.y)) return;
+  solve_channels(ws, C, (int64_t)N * HW, mp, s_state, has_prev, gmax_layer, stats_out, cls);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sweep 3: Eq. 1 on every element.  Output 1 uses `scale1` (per channel if PER_CHANNEL, else one
+// value) and generator stream 0; the optional output 2 uses the single value `scale2` and
+// stream 1 (Algorithm 1 lines 10-11 fused, as Sec. 3.4 suggests).  STOCH selects the rounding.
+// Codes are written as [pixel][Cp] with zero padding channels.
+// ------------------------------------------------------------------------------------------------
+template <int VE>
+__device__ __forceinline__ void store_codes(int8_t* dst, const int (&q)[VE]);
+template <>
+__device__ __forceinline__ void store_codes<1>(int8_t* dst, const int (&q)[1]) { *dst = (int8_t)q[0]; }
+template <>
+__device__ __forceinline__ void store_codes<4>(int8_t* dst, const int (&q)[4]) {
+  const uint32_t w = (q[0] & 0xFF) | ((q[1] & 0xFF) << 8) | ((q[2] & 0xFF) << 16) | ((uint32_t)q[3] << 24);
+  *reinterpret_cast<uint32_t*>(dst) = w;
+}
+template <>
+__device__ __forceinline__ void store_codes<8>(int8_t* dst, const int (&q)[8]) {
+  uint2 w;
+  w.x = (q[0] & 0xFF) | ((q[1] & 0xFF) << 8) | ((q[2] & 0xFF) << 16) | ((uint32_t)q[3] << 24);
+  w.y = (q[4] & 0xFF) | ((q[5] & 0xFF) << 8) | ((q[6] & 0xFF) << 16) | ((uint32_t)q[7] << 24);
+  *reinterpret_cast<uint2*>(dst) = w;
+}
+
+template <typename T, int VE, bool PER_CHANNEL, bool STOCH, bool DUAL>
+__global__ void __launch_bounds__(kThreads)
+quantize_nhwc_kernel(const T* __restrict__ x, int64_t npix, int64_t HW, int C, int Cp, int Gp,
+                     const float* __restrict__ scale1, const float* __restrict__ scale2,
+                     uint32_t seed, int8_t* __restrict__ q1, int8_t* __restrict__ q2) {
+  const int tid = threadIdx.x;
+  const int colv0 = blockIdx.y * kThreads;
+  const int gcols = min(Gp - colv0, kThreads);
+  const int rpi = kThreads / gcols;
+  const int col = tid % gcols, rl = tid / gcols;
+  if (rl >= rpi) return;
+  const int64_t chunk = (npix + gridDim.x - 1) / gridDim.x;
+  const int64_t p0 = (int64_t)blockIdx.x * chunk;
+  const int64_t p1 = min(npix, p0 + chunk);
+  const int c0 = (colv0 + col) * VE;  // first channel of this thread's vector
+  const bool real = c0 < C;           // else: padding channels, write zeros (C % VE == 0)
+  float inv1[VE];
+  float inv2 = 0.f;
+#pragma unroll
+  for (int e = 0; e < VE; ++e) inv1[e] = real ? inv_scale(PER_CHANNEL ? scale1[c0 + e] : scale1[0]) : 0.f;
+  if (DUAL) inv2 = inv_scale(scale2[0]);
+  const uint32_t key0 = sr_key(seed, 0u);
+
+  int64_t p = p0 + rl;
+  if (p >= p1) return;
+  int64_t n = p / HW;
+  int64_t hw = p - n * HW;
+  for (; p < p1; p += rpi) {
+    int qa[VE], qb[VE];
+    if (real) {
+      float v[VE];
+      load_vec<T, VE>(x + p * C + c0, v);
+      // NCHW index of element (n, c0+e, hw): (n*C + c0 + e)*HW + hw
+      const uint64_t idx0 = ((uint64_t)n * C + c0) * HW + hw;
+#pragma unroll
+      for (int e = 0; e < VE; ++e) {
+        if (STOCH) {
+          const uint64_t idx = idx0 + (uint64_t)e * HW;
+          const uint32_t hi = (uint32_t)(idx >> 32);
+          const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
+          const uint32_t h = avalanche32((uint32_t)idx ^ key);
+          qa[e] = quant_stochastic(v[e], inv1[e], sr_uniform(h));
+          qb[e] = DUAL ? quant_stochastic(v[e], inv2, sr_uniform(h * 0x9E3779B1u)) : 0;
+        } else {
+          qa[e] = quant_nearest(v[e], inv1[e]);
+          qb[e] = DUAL ? quant_nearest(v[e], inv2) : 0;
+        }
+      }
+    } else {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) { qa[e] = 0; qb[e] = 0; }
+    }
+    store_codes<VE>(q1 + p * Cp + c0, qa);
+    if (DUAL) store_codes<VE>(q2 + p * Cp + c0, qb);
+    hw += rpi;
+    while (hw >= HW) { hw -= HW; ++n; }
+  }
+}
+
+// NCHW input, NHWC codes: a block transposes a tile of 32 channels x 128 positions of one image
+// through shared memory.  grid = (hw tiles, channel tiles over Cp, N).
+constexpr int kTileC = 32, kTileHW = 128, kTileRow = 36;  // 36-byte rows: conflict-free byte writes
+
+template <typename T, bool PER_CHANNEL, bool STOCH, bool DUAL>
+__global__ void __launch_bounds__(kThreads)
+quantize_nchw_kernel(const T* __restrict__ x, int C, int Cp, int64_t HW,
+                     const float* __restrict__ scale1, const float* __restrict__ scale2,
+                     uint32_t seed, int8_t* __restrict__ q1, int8_t* __restrict__ q2) {
+  __shared__ __align__(16) int8_t t1[kTileHW * kTileRow];
+  __shared__ __align__(16) int8_t t2[kTileHW * kTileRow];
+  __shared__ float sinv[kTileC];
+  const int tid = threadIdx.x;
+  const int64_t hw0 = (int64_t)blockIdx.x * kTileHW;
+  const int c0 = blockIdx.y * kTileC;
+  const int n = blockIdx.z;
+  if (tid < kTileC) {
+    const int c = c0 + tid;
+    sinv[tid] = c < C ? inv_scale(PER_CHANNEL ? scale1[c] : scale1[0]) : 0.f;
+  }
+  const float inv2 = DUAL ? inv_scale(scale2[0]) : 0.f;
+  const uint32_t key0 = sr_key(seed, 0u);
+  __syncthreads();
+  for (int i = tid; i < kTileC * kTileHW; i += kThreads) {
+    const int cl = i / kTileHW, hl = i % kTileHW;
+    const int c = c0 + cl;
+    const int64_t hw = hw0 + hl;
+    int a = 0, b = 0;
+    if (c < C && hw < HW) {
+      const uint64_t idx = ((uint64_t)n * C + c) * HW + hw;
+      const float v = to_f32(x[idx]);
+      if (STOCH) {
+        const uint32_t hi = (uint32_t)(idx >> 32);
+        const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
+        const uint32_t h = avalanche32((uint32_t)idx ^ key);
+        a = quant_stochastic(v, sinv[cl], sr_uniform(h));
+        if (DUAL) b = quant_stochastic(v, inv2, sr_uniform(h * 0x9E3779B1u));
+      } else {
+        a = quant_nearest(v, sinv[cl]);
+        if (DUAL) b = quant_nearest(v, inv2);
+      }
+    }
+    t1[hl * kTileRow + cl] = (int8_t)a;
+    if (DUAL) t2[hl * kTileRow + cl] = (int8_t)b;
+  }
+  __syncthreads();
+  // 8 threads write the 32 bytes of one position; Cp is a multiple of 16, so a tile is 16 or 32 wide
+  const int cw = min(kTileC, Cp - c0);
+  for (int i = tid; i < kTileHW * (kTileC / 4); i += kThreads) {
+    const int hl = i / (kTileC / 4), w4 = i % (kTileC / 4);
+    const int64_t hw = hw0 + hl;
+    if (hw < HW && w4 * 4 < cw) {
+      const size_t o = ((size_t)n * HW + hw) * Cp + c0 + w4 * 4;
+      *reinterpret_cast<uint32_t*>(q1 + o) = *reinterpret_cast<const uint32_t*>(t1 + hl * kTileRow + w4 * 4);
+      if (DUAL) *reinterpret_cast<uint32_t*>(q2 + o) = *reinterpret_cast<const uint32_t*>(t2 + hl * kTileRow + w4 * 4);
+    }
+  }
+}
+
+// max|x| over a whole tensor (layout-free), into the bit pattern at out_bits (zeroed before).
+template <typename T, int VE>
+__global__ void __launch_bounds__(kThreads)
+absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_bits) {
+  float m = 0.f;
+  for (int64_t i = (int64_t)blockIdx.x * kThreads + threadIdx.x; i < nvec; i += (int64_t)gridDim.x * kThreads) {
+    float v[VE];
+    load_vec<T, VE>(x + i * VE, v);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) m = fmaxf(m, fabsf(v[e]));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(out_bits, __float_as_uint(m));
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host-side launch helpers
+// ------------------------------------------------------------------------------------------------
+struct NhwcGrid {
+  dim3 grid;
+  int G;   // vectors per pixel that are processed
+};
+
+// Pixel blocks x column blocks for the NHWC mapping: at most kMaxPixelBlocks blocks in total and
+// at least ~8 iterations of work per block.
+NhwcGrid nhwc_grid(int64_t npix, int vectors_per_pixel) {
+  NhwcGrid g;
+  g.G = vectors_per_pixel;
+  const int colblocks = (vectors_per_pixel + kThreads - 1) / kThreads;
+  const int gcols = vectors_per_pixel < kThreads ? vectors_per_pixel : kThreads;
+  const int rpi = kThreads / gcols;
+  int64_t pb = ceil_div64(npix, (int64_t)rpi * 8);
+  int64_t cap = kMaxPixelBlocks / colblocks;
+  if (cap < 1) cap = 1;
+  if (pb > cap) pb = cap;
+  if (pb < 1) pb = 1;
+  g.grid = dim3((unsigned)pb, (unsigned)colblocks, 1);
+  return g;
+}
+
+int nchw_slices(int N, int C) {
+  int ns = (kMaxPixelBlocks + C - 1) / C;
+  if (ns > N) ns = N;
+  if (ns > kMaxPixelBlocks) ns = kMaxPixelBlocks;
+  if (ns < 1) ns = 1;
+  return ns;
+}
+
+template <typename T>
+constexpr int vec_elems() { return 16 / (int)sizeof(T); }
+
+template <typename T>
+dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, int H, int W,
+                                const McsDev& mp, float* s_state, int has_prev, float* gmax_layer,
+                                float* stats, uint8_t* cls, int8_t* vq, int8_t* gq, uint32_t seed,
+                                const float* sigma_override, const GvqWs& ws, cudaStream_t st) {
+  const int64_t HW = (int64_t)H * W;
+  const int64_t npix = (int64_t)N * HW;
+  const int Cp = round_up(C, 16);
+  constexpr int VEfull = vec_elems<T>();
+  const float* sigma = sigma_override ? sigma_override : ws.sigma;
+  if (layout == DAI8_NHWC) {
+    if (C % VEfull == 0) {
+      const NhwcGrid g = nhwc_grid(npix, C / VEfull);
+      stats_nhwc_kernel<T, VEfull><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, mp, stats);
+      count_nhwc_kernel<T, VEfull><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, sigma, mp, s_state,
+                                                                has_prev, gmax_layer, stats, cls);
+      const NhwcGrid gq_ = nhwc_grid(npix, Cp / VEfull);
+      if (gq)
+        quantize_nhwc_kernel<T, VEfull, true, true, true><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, gq);
+      else
+        quantize_nhwc_kernel<T, VEfull, true, true, false><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, nullptr);
+    } else {
+      const NhwcGrid g = nhwc_grid(npix, C);
+      stats_nhwc_kernel<T, 1><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, mp, stats);
+      count_nhwc_kernel<T, 1><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, sigma, mp, s_state,
+                                                           has_prev, gmax_layer, stats, cls);
+      const NhwcGrid gq_ = nhwc_grid(npix, Cp);
+      if (gq)
+        quantize_nhwc_kernel<T, 1, true, true, true><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, gq);
+      else
+        quantize_nhwc_kernel<T, 1, true, true, false><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, nullptr);
+    }
+  } else {
+    const dim3 grid((unsigned)C, (unsigned)nchw_slices(N, C), 1);
+    stats_nchw_kernel<T><<<grid, kThreads, 0, st>>>(dY, N, C, HW, ws, mp, stats);
+    count_nchw_kernel<T><<<grid, kThreads, 0, st>>>(dY, N, C, HW, ws, sigma, mp, s_state, has_prev,
+                                                    gmax_layer, stats, cls);
+    const dim3 qgrid((unsigned)ceil_div64(HW, kTileHW), (unsigned)((Cp + kTileC - 1) / kTileC), (unsigned)N);
+    if (gq)
+      quantize_nchw_kernel<T, true, true, true><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, s_state,
+                                                                            gmax_layer, seed, vq, gq);
+    else
+      quantize_nchw_kernel<T, true, true, false><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, s_state,
+                                                                             gmax_layer, seed, vq, nullptr);
+  }
+  note_launch(3);
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+template <typename T>
+dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, int H, int W,
+                                  dai8_scale_mode mode, float* scale, dai8_round round,
+                                  uint32_t seed, int8_t* q, cudaStream_t st) {
+  const int64_t HW = (int64_t)H * W;
+  const int64_t npix = (int64_t)N * HW;
+  const int64_t total = npix * C;
+  const int Cp = round_up(C, 16);
+  constexpr int VEfull = vec_elems<T>();
+  if (mode == DAI8_SCALE_ABSMAX) {
+    DAI8_RETURN_IF_CUDA(cudaMemsetAsync(scale, 0, sizeof(float), st));
+    uint32_t* bits = reinterpret_cast<uint32_t*>(scale);
+    if (total % VEfull == 0) {
+      const int64_t nvec = total / VEfull;
+      const int blocks = (int)(ceil_div64(nvec, kThreads * 4) < kMaxPixelBlocks ? ceil_div64(nvec, kThreads * 4) : kMaxPixelBlocks);
+      absmax_kernel<T, VEfull><<<blocks, kThreads, 0, st>>>(x, nvec, bits);
+    } else {
+      const int blocks = (int)(ceil_div64(total, kThreads * 4) < kMaxPixelBlocks ? ceil_div64(total, kThreads * 4) : kMaxPixelBlocks);
+      absmax_kernel<T, 1><<<blocks, kThreads, 0, st>>>(x, total, bits);
+    }
+    note_launch(1);
+  }
+  const bool stoch = round == DAI8_ROUND_STOCHASTIC;
+  if (layout == DAI8_NHWC) {
+    if (C % VEfull == 0) {
+      const NhwcGrid g = nhwc_grid(npix, Cp / VEfull);
+      if (stoch)
+        quantize_nhwc_kernel<T, VEfull, false, true, false><<<g.grid, kThreads, 0, st>>>(x, npix, HW, C, Cp, g.G, scale, nullptr, seed, q, nullptr);
+      else
+        quantize_nhwc_kernel<T, VEfull, false, false, false><<<g.grid, kThreads, 0, st>>>(x, npix, HW, C, Cp, g.G, scale, nullptr, seed, q, nullptr);
+    } else {
+      const NhwcGrid g = nhwc_grid(npix, Cp);
+      if (stoch)
+        quantize_nhwc_kernel<T, 1, false, true, false><<<g.grid, kThreads, 0, st>>>(x, npix, HW, C, Cp, g.G, scale, nullptr, seed, q, nullptr);
+      else
+        quantize_nhwc_kernel<T, 1, false, false, false><<<g.grid, kThreads, 0, st>>>(x, npix, HW, C, Cp, g.G, scale, nullptr, seed, q, nullptr);
+    }
+  } else {
+    const dim3 qgrid((unsigned)ceil_div64(HW, kTileHW), (unsigned)((Cp + kTileC - 1) / kTileC), (unsigned)N);
+    if (stoch)
+      quantize_nchw_kernel<T, false, true, false><<<qgrid, kThreads, 0, st>>>(x, C, Cp, HW, scale, nullptr, seed, q, nullptr);
+    else
+      quantize_nchw_kernel<T, false, false, false><<<qgrid, kThreads, 0, st>>>(x, C, Cp, HW, scale, nullptr, seed, q, nullptr);
+  }
+  note_launch(1);
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+bool bad_dims(int N, int C, int H, int W) {
+  return N <= 0 || C <= 0 || H <= 0 || W <= 0 || N > 65535;
+}
+
+}  // namespace
+}  // namespace dai8
+
+using namespace dai8;
+
+extern "C" size_t dai8_quantize_grad_workspace_bytes(int C) { return C > 0 ? ws_bytes_for(C) : 0; }
+
+extern "C" dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8_layout layout, int N,
+                                          int C, int H, int W, const dai8_mcs_params* params,
+                                          float* s_state, int has_prev, float* gmax_layer,
+                                          float* stats, uint8_t* cls, int8_t* vq, int8_t* gq,
+                                          uint32_t seed, const float* sigma_override, void* ws,
+                                          size_t ws_bytes, void* stream) {
+  if (!dY || !s_state || !gmax_layer || !vq || !ws) return DAI8_ERR_INVALID_ARG;
+  if (bad_dims(N, C, H, W)) return DAI8_ERR_INVALID_ARG;
+  if (dtype != DAI8_F32 && dtype != DAI8_BF16) return DAI8_ERR_INVALID_ARG;
+  if (layout != DAI8_NCHW && layout != DAI8_NHWC) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(vq) || (gq && !aligned16(gq)) || !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if ((int64_t)N * H * W >= (int64_t)1 << 32) return DAI8_ERR_UNSUPPORTED;  // counts are 32-bit
+  if (ws_bytes < ws_bytes_for(C)) return DAI8_ERR_WORKSPACE;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  dai8_mcs_params p;
+  if (params) p = *params; else dai8_mcs_defaults(&p);
+  McsDev mp{p.lambda, p.k, p.A, p.std_unbiased, p.center_mean};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  GvqWs w = carve(ws, C);
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(w.tickets, 0, control_words(C) * 4, st));
+  if (dtype == DAI8_F32)
+    return quantize_grad_typed<float>(static_cast<const float*>(dY), layout, N, C, H, W, mp, s_state,
+                                      has_prev, gmax_layer, stats, cls, vq, gq, seed, sigma_override, w, st);
+  return quantize_grad_typed<bf16_t>(static_cast<const bf16_t*>(dY), layout, N, C, H, W, mp, s_state,
+                                     has_prev, gmax_layer, stats, cls, vq, gq, seed, sigma_override, w, st);
+}
+
+extern "C" dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout layout, int N,
+                                            int C, int H, int W, dai8_scale_mode scale_mode,
+                                            float* scale, dai8_round round, uint32_t seed, int8_t* q,
+                                            void* stream) {
+  if (!x || !scale || !q) return DAI8_ERR_INVALID_ARG;
+  if (bad_dims(N, C, H, W)) return DAI8_ERR_INVALID_ARG;
+  if (dtype != DAI8_F32 && dtype != DAI8_BF16) return DAI8_ERR_INVALID_ARG;
+  if (layout != DAI8_NCHW && layout != DAI8_NHWC) return DAI8_ERR_INVALID_ARG;
+  if (scale_mode != DAI8_SCALE_ABSMAX && scale_mode != DAI8_SCALE_GIVEN) return DAI8_ERR_INVALID_ARG;
+  if (round != DAI8_ROUND_NEAREST_EVEN && round != DAI8_ROUND_STOCHASTIC) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(q)) return DAI8_ERR_INVALID_ARG;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (dtype == DAI8_F32)
+    return quantize_tensor_typed<float>(static_cast<const float*>(x), layout, N, C, H, W, scale_mode,
+                                        scale, round, seed, q, st);
+  return quantize_tensor_typed<bf16_t>(static_cast<const bf16_t*>(x), layout, N, C, H, W, scale_mode,
+                                       scale, round, seed, q, st);
+}

@@ -1,0 +1,191 @@
+"""GPU parity of the int8 convolutions against the CPU oracle: int32 accumulators bit-exact given
+identical codes, de-quantized outputs within rel 1e-5 of max|value|.  Small shapes are compared
+element by element; the benchmark's full-size layers on sampled outputs (each output of a direct
+convolution is an independent dot product) plus an exact adjoint identity over the whole tensor."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cpu as O
+from paper_2102_04782_b200 import api, synth
+
+from helpers import codes_from_nchw, geom, out_to_nchw, scalar, ws_bytes
+
+pytestmark = pytest.mark.gpu
+
+REL = 1e-5
+
+GEOMS = [
+    # N, Cin, Cout, H, W, R, S, stride, pad
+    (8, 64, 64, 14, 14, 3, 3, 1, 1),        # config 1
+    (2, 3, 16, 17, 19, 7, 7, 2, 3),         # stem-like: 3 channels, 7x7 stride 2
+    (3, 24, 40, 9, 11, 1, 1, 1, 0),         # ragged channels, pointwise
+    (2, 32, 48, 12, 12, 3, 3, 2, 1),        # stride-2 3x3
+    (2, 48, 32, 10, 10, 1, 1, 2, 0),        # stride-2 projection
+    (1, 16, 16, 5, 7, 3, 5, (1, 2), (1, 2)),
+    (2, 130, 70, 6, 6, 3, 3, 1, 1),         # channel counts that are not multiples of 16
+    (1, 64, 128, 30, 30, 3, 3, 1, 1),       # several 128-pixel tiles with a ragged tail
+]
+
+
+def rand_codes(rng, shape):
+    return rng.integers(-127, 128, size=shape, dtype=np.int64).astype(np.int8)
+
+
+def weights_dev(qW):
+    """(Cout,Cin,R,S) codes -> device [Cout][R][S][Cinp]."""
+    Cout, Cin, R, S = qW.shape
+    Cp = (Cin + 15) // 16 * 16
+    out = np.zeros((Cout, R, S, Cp), np.int8)
+    out[..., :Cin] = qW.transpose(0, 2, 3, 1)
+    return torch.from_numpy(out).cuda()
+
+
+def run_all(g, qX, qW, qG, sX, sW, gmax, s_c, dtype, layout, backend=0):
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    gg = geom(*g)
+    P, Q = gg.P, gg.Q
+    api.set_conv_backend(backend)
+    try:
+        dX_shape = (N, Cin, H, W) if layout == api.NCHW else (N, H, W, Cin)
+        Y_shape = (N, Cout, P, Q) if layout == api.NCHW else (N, P, Q, Cout)
+        Y = torch.empty(Y_shape, dtype=dtype, device="cuda")
+        dX = torch.empty(dX_shape, dtype=dtype, device="cuda")
+        dW = torch.empty((Cout, Cin, R, S), dtype=dtype if dtype != torch.bfloat16 else torch.float32,
+                         device="cuda")
+        dqX, dqW, dqG = codes_from_nchw(qX), weights_dev(qW), codes_from_nchw(qG)
+        api.conv_fwd(dqX, dqW, scalar(sX), scalar(sW), gg, Y, layout,
+                     ws_bytes(api.conv_workspace_bytes(api.OP_FWD, gg)))
+        api.conv_bwd_data(dqG, dqW, scalar(gmax), scalar(sW), gg, dX, layout,
+                          ws_bytes(api.conv_workspace_bytes(api.OP_BWD_DATA, gg)))
+        api.conv_bwd_filter(dqX, dqG, scalar(sX), torch.from_numpy(s_c).cuda(), gg, dW,
+                            ws_bytes(api.conv_workspace_bytes(api.OP_BWD_FILTER, gg)))
+        torch.cuda.synchronize()
+        assert api.get_device_status() == api.OK
+    finally:
+        api.set_conv_backend(0)
+    return out_to_nchw(Y, layout), out_to_nchw(dX, layout), dW.cpu().numpy()
+
+
+@pytest.mark.parametrize("g", GEOMS)
+@pytest.mark.parametrize("backend", [0, 1])
+def test_accumulators_bit_exact(g, backend):
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    rng = np.random.default_rng(31)
+    P, Q = O.out_hw(H, W, R, S, st, pad)
+    qX, qW, qG = rand_codes(rng, (N, Cin, H, W)), rand_codes(rng, (Cout, Cin, R, S)), rand_codes(rng, (N, Cout, P, Q))
+    s_c = np.ones(Cout, np.float32)
+    for layout in (api.NHWC, api.NCHW):
+        Y, dX, dW = run_all(g, qX, qW, qG, 1.0, 1.0, 1.0, s_c, torch.int32, layout, backend)
+        y_o, ov1 = O.conv_fwd_acc(qX, qW, st, pad)
+        dx_o, ov2 = O.conv_bwd_data_acc(qG, qW, (H, W), st, pad)
+        dw_o, ov3 = O.conv_bwd_filter_acc(qX, qG, (R, S), st, pad)
+        assert ov1 == ov2 == ov3 == 0
+        np.testing.assert_array_equal(Y, y_o)
+        np.testing.assert_array_equal(dX, dx_o)
+        np.testing.assert_array_equal(dW, dw_o)
+
+
+@pytest.mark.parametrize("g", [GEOMS[0], GEOMS[3], GEOMS[6]])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_dequantized_outputs(g, dtype):
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    rng = np.random.default_rng(32)
+    P, Q = O.out_hw(H, W, R, S, st, pad)
+    qX, qW, qG = rand_codes(rng, (N, Cin, H, W)), rand_codes(rng, (Cout, Cin, R, S)), rand_codes(rng, (N, Cout, P, Q))
+    sX, sW, gmax = 3.7, 0.21, 8.3e-4
+    s_c = (10.0 ** rng.uniform(-6, -3, Cout)).astype(np.float32)
+    Y, dX, dW = run_all(g, qX, qW, qG, sX, sW, gmax, s_c, dtype, api.NHWC)
+    y_o = O.dequant_acc(O.conv_fwd_acc(qX, qW, st, pad)[0], sX, sW)
+    dx_o = O.dequant_acc(O.conv_bwd_data_acc(qG, qW, (H, W), st, pad)[0], gmax, sW)
+    dw_o = O.dequant_acc(O.conv_bwd_filter_acc(qX, qG, (R, S), st, pad)[0], sX, s_c)
+    rel = REL if dtype == torch.float32 else 2.0 ** -8   # bf16 output: half an ulp of bf16
+    for got, want in ((Y, y_o), (dX, dx_o)):
+        assert np.abs(got - want).max() <= rel * np.abs(want).max()
+    for co in range(Cout):  # per output channel, since the scales differ by decades
+        assert np.abs(dW[co] - dw_o[co]).max() <= REL * np.abs(dw_o[co]).max() + 1e-45
+
+
+def test_config1_end_to_end_layer_step():
+    """One layer step on config 1 through the whole path: forward quantization, forward conv,
+    gradient quantization, both backward convolutions -- each stage against the oracle fed with the
+    GPU's scales."""
+    from helpers import GradQuant, codes_to_nchw, dev_input
+    layer = synth.config1_layer()
+    N = 8
+    x, w, g, _, _ = synth.layer_inputs(layer, N, seed=41, bf16=False)
+    gg = geom(N, layer.Cin, layer.Cout, layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad)
+    Cp = api.padded_channels(layer.Cin)
+    qX = torch.empty((N, layer.H, layer.W, Cp), dtype=torch.int8, device="cuda")
+    qW = torch.empty((layer.Cout, layer.R, layer.S, Cp), dtype=torch.int8, device="cuda")
+    sX, sW = scalar(0), scalar(0)
+    api.quantize_tensor(dev_input(x, False, api.NHWC), api.NHWC, N, layer.Cin, layer.H, layer.W,
+                        api.SCALE_ABSMAX, sX, api.ROUND_NEAREST_EVEN, 0, qX)
+    api.quantize_tensor(torch.from_numpy(w).cuda(), api.NCHW, layer.Cout, layer.Cin, layer.R, layer.S,
+                        api.SCALE_ABSMAX, sW, api.ROUND_NEAREST_EVEN, 0, qW)
+    Y = torch.empty((N, layer.P, layer.Q, layer.Cout), dtype=torch.float32, device="cuda")
+    api.conv_fwd(qX, qW, sX, sW, gg, Y, api.NHWC, None)
+    gqb = GradQuant(N, layer.Cout, layer.P, layer.Q)
+    gqb.run(dev_input(g, False, api.NHWC), api.NHWC, 17, has_prev=False)
+    dX = torch.empty((N, layer.H, layer.W, layer.Cin), dtype=torch.float32, device="cuda")
+    dW = torch.empty((layer.Cout, layer.Cin, layer.R, layer.S), dtype=torch.float32, device="cuda")
+    api.conv_bwd_data(gqb.gq, qW, gqb.gmax, sW, gg, dX, api.NHWC,
+                      ws_bytes(api.conv_workspace_bytes(api.OP_BWD_DATA, gg)))
+    api.conv_bwd_filter(qX, gqb.vq, sX, gqb.s_state, gg, dW,
+                        ws_bytes(api.conv_workspace_bytes(api.OP_BWD_FILTER, gg)))
+    torch.cuda.synchronize()
+    sx, sw = float(sX.item()), float(sW.item())
+    assert sx == float(np.abs(x).max()) and sw == float(np.abs(w).max())
+    qx_o, qw_o = O.quantize(x, sx), O.quantize(w, sw)
+    np.testing.assert_array_equal(codes_to_nchw(qX, layer.Cin), qx_o)
+    s_c = gqb.s_state.cpu().numpy()
+    gl = float(gqb.gmax.item())
+    vq_o = O.quantize(g, s_c, True, 17, 0)
+    gq_o = O.quantize(g, gl, True, 17, 1)
+    y_o = O.dequant_acc(O.conv_fwd_acc(qx_o, qw_o, 1, 1)[0], sx, sw)
+    dx_o = O.dequant_acc(O.conv_bwd_data_acc(gq_o, qw_o, (layer.H, layer.W), 1, 1)[0], gl, sw)
+    dw_o = O.dequant_acc(O.conv_bwd_filter_acc(qx_o, vq_o, (3, 3), 1, 1)[0], sx, s_c)
+    assert np.abs(out_to_nchw(Y, api.NHWC) - y_o).max() <= REL * np.abs(y_o).max()
+    assert np.abs(out_to_nchw(dX, api.NHWC) - dx_o).max() <= REL * np.abs(dx_o).max()
+    got = dW.cpu().numpy()
+    for co in range(layer.Cout):
+        assert np.abs(got[co] - dw_o[co]).max() <= REL * np.abs(dw_o[co]).max() + 1e-45
+
+
+def _sample_check(g, rng, backend=0, nsamp=2048):
+    """Full-size layer: accumulators at sampled outputs, plus the exact adjoint identity
+    <Y, G> = <X, dX> = <W, dW> over whole tensors (integers, so equality is exact)."""
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    P, Q = O.out_hw(H, W, R, S, st, pad)
+    qX, qW, qG = rand_codes(rng, (N, Cin, H, W)), rand_codes(rng, (Cout, Cin, R, S)), rand_codes(rng, (N, Cout, P, Q))
+    # keep accumulators far from int32 overflow for the dW contraction over N*P*Q pixels
+    qG = (qG.astype(np.int16) * (rng.random(qG.shape) < 0.02)).astype(np.int8)
+    s_c = np.ones(Cout, np.float32)
+    Y, dX, dW = run_all(g, qX, qW, qG, 1.0, 1.0, 1.0, s_c, torch.int32, api.NHWC, backend)
+    for full, fn, args in ((Y, O.conv_fwd_acc, (qX, qW, st, pad)),
+                           (dX, O.conv_bwd_data_acc, (qG, qW, (H, W), st, pad)),
+                           (dW, O.conv_bwd_filter_acc, (qX, qG, (R, S), st, pad))):
+        idx = rng.choice(full.size, min(nsamp, full.size), replace=False)
+        want, ov = fn(*args, idx=idx)
+        assert ov == 0
+        np.testing.assert_array_equal(full.reshape(-1)[idx], want)
+    lhs = int((Y.astype(np.int64) * qG).sum())
+    assert lhs == int((dX.astype(np.int64) * qX).sum()) == int((dW.astype(np.int64) * qW).sum())
+
+
+@pytest.mark.parametrize("li", [0, 1, 2])
+def test_config2_layers_sampled(li):
+    """ResNet-50 conv2_x bottleneck at N=64, 56x56 (the benchmark's configuration)."""
+    layer = synth.resnet50_conv2x_block()[li]
+    g = (64, layer.Cin, layer.Cout, layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad)
+    _sample_check(g, np.random.default_rng(50 + li))
+
+
+def test_unsupported_and_errors():
+    gg = geom(1, 16, 16, 4, 4, 3, 3, 1, 1)
+    q = torch.zeros((1, 4, 4, 16), dtype=torch.int8, device="cuda")
+    w = torch.zeros((16, 3, 3, 16), dtype=torch.int8, device="cuda")
+    out = torch.zeros((1, 4, 4, 16), dtype=torch.float32, device="cuda")
+    with pytest.raises(api.Dai8Error) as e:
+        api.conv_bwd_data(q, w, scalar(1), scalar(1), gg, out, api.NHWC, ws_bytes(16))
+    assert e.value.code == api.ERR_WORKSPACE

@@ -1,0 +1,178 @@
+"""GPU parity of dai8_quantize_grad / dai8_quantize_tensor against the CPU oracle, stage by stage
+so that a discrete decision (class, code) is always compared given identical upstream values:
+  (1) |g|max bit-exact, mean / sigma within rel 1e-5;
+  (2) density count exact given the GPU's sigma;
+  (3) class exact and clip within rel 1e-5 given identical (count, |g|max, s_prev);
+  (4) int8 codes bit-exact given identical scales;
+then end to end (the oracle running on its own sigma), where only channels whose count lies within
+2 of the threshold lambda*M may differ."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import cpu as O
+from paper_2102_04782_b200 import api, synth
+
+from helpers import GradQuant, codes_to_nchw, dev_input, padding_is_zero, scalar
+
+pytestmark = pytest.mark.gpu
+
+REL = 1e-5
+
+
+def check_grad_quant(g, bf16, layout, seed=5, iters=2, params=None):
+    N, C, H, W = g.shape
+    M = N * H * W
+    gq = GradQuant(N, C, H, W)
+    d = dev_input(g, bf16, layout)
+    kw = {}
+    if params is not None:
+        kw = dict(lam=params.lam, k=params.k, A=params.A)
+    s_prev_gpu = None
+    s_prev_e2e = None
+    band_ever = np.zeros(C, bool)
+    for t in range(iters):
+        gq.run(d, layout, seed + t, has_prev=t > 0, params=params)
+        stats = gq.stats.cpu().numpy()
+        s_gpu = gq.s_state.cpu().numpy()
+        cls_gpu = gq.cls.cpu().numpy()
+        gmax_gpu = float(gq.gmax.item())
+        # (1)
+        absmax, mean, sigma, gl = O.channel_stats(g, bool(params.std_unbiased) if params else False,
+                                                  bool(params.center_mean) if params else True)
+        np.testing.assert_array_equal(stats[:, 0], absmax)
+        assert gmax_gpu == gl
+        np.testing.assert_allclose(stats[:, 2], sigma, rtol=REL, atol=0)
+        assert np.all(np.abs(stats[:, 1] - mean) <= REL * np.maximum(sigma, 1e-30) + 1e-7 * np.abs(mean))
+        # (2) count given the GPU's sigma
+        cnt = O.density_count(g, stats[:, 2])
+        np.testing.assert_array_equal(stats[:, 3], (cnt.astype(np.float64) / M).astype(np.float32))
+        # (3) class and clip given identical inputs
+        s_or, cls_or = O.classify_clip(cnt, absmax, M, s_prev=s_prev_gpu, **kw)
+        np.testing.assert_array_equal(cls_gpu, cls_or)
+        np.testing.assert_allclose(s_gpu, s_or, rtol=REL, atol=0)
+        # (4) codes given identical scales
+        vq = codes_to_nchw(gq.vq, C)
+        gqc = codes_to_nchw(gq.gq, C)
+        np.testing.assert_array_equal(vq, O.quantize(g, s_gpu, stochastic=True, seed=seed + t, stream=0))
+        np.testing.assert_array_equal(gqc, O.quantize(g, gmax_gpu, stochastic=True, seed=seed + t, stream=1))
+        assert padding_is_zero(gq.vq, C) and padding_is_zero(gq.gq, C)
+        # end to end: the oracle on its own sigma
+        cnt_e = O.density_count(g, sigma)
+        s_e, cls_e = O.classify_clip(cnt_e, absmax, M, s_prev=s_prev_e2e, **kw)
+        lam = np.float32(params.lam if params else 0.3)
+        band_ever |= np.abs(cnt_e.astype(np.float64) - float(lam) * M) <= 2
+        assert np.array_equal(cls_gpu[~band_ever], cls_e[~band_ever])
+        np.testing.assert_allclose(s_gpu[~band_ever], s_e[~band_ever], rtol=REL)
+        s_prev_gpu = s_gpu
+        s_prev_e2e = s_e
+    return gq
+
+
+@pytest.mark.parametrize("layout", [api.NHWC, api.NCHW])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_config1_grad_quant(layout, bf16):
+    """Config 1: N=8, C=64, 14x14, per-channel bell-shaped / long-tailed mix."""
+    g, is_bell, _ = synth.channel_mixed_grad(8, 64, 14, 14, seed=1)
+    if bf16:
+        g = synth.round_to_bf16(g)
+    gq = check_grad_quant(g, bf16, layout, iters=3)
+    cls = gq.cls.cpu().numpy()
+    # long-tailed channels are never classed bell-shaped; most bell-shaped ones are
+    assert not np.any(cls[~is_bell])
+    assert cls[is_bell].mean() > 0.8
+
+
+@pytest.mark.parametrize("shape", [
+    (2, 24, 7, 9),      # C multiple of 8 but not 16: padded code channels
+    (3, 20, 5, 5),      # bf16: C not a multiple of 8 -> element-wise path; fp32: vector path
+    (1, 3, 11, 13),     # tiny C, odd extents, misaligned NCHW rows
+    (2, 2048, 2, 2),    # several column blocks
+    (5, 96, 9, 9),
+    (1, 1, 1, 1),
+    (2, 16, 1, 300),
+])
+@pytest.mark.parametrize("layout", [api.NHWC, api.NCHW])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_ragged_shapes(shape, layout, bf16):
+    g, _, _ = synth.channel_mixed_grad(*shape, seed=2)
+    if bf16:
+        g = synth.round_to_bf16(g)
+    check_grad_quant(g, bf16, layout, iters=2)
+
+
+def test_hyper_parameters_and_flags():
+    g, _, _ = synth.channel_mixed_grad(4, 32, 12, 12, seed=3)
+    g = g + np.float32(2e-5)  # a mean offset so that center_mean matters
+    for k, A, unb, cen in [(1.5, 0.5, 0, 1), (1.2, 0.8, 1, 1), (1.0, 0.8, 0, 0)]:
+        p = api.mcs_defaults()
+        p.k, p.A, p.std_unbiased, p.center_mean = k, A, unb, cen
+        check_grad_quant(g, False, api.NHWC, iters=3, params=p)
+
+
+def test_zero_channel_and_sigma_override():
+    g, _, _ = synth.channel_mixed_grad(2, 16, 6, 6, seed=4)
+    g[:, 3] = 0.0
+    gq = check_grad_quant(g, False, api.NHWC, iters=2)
+    assert float(gq.s_state[3].item()) == 0.0
+    assert np.all(codes_to_nchw(gq.vq, 16)[:, 3] == 0)
+    # a caller-provided sigma replaces the computed one in the density count
+    sig = torch.full((16,), 1e-9, dtype=torch.float32, device="cuda")
+    d = dev_input(g, False, api.NHWC)
+    gq.run(d, api.NHWC, 1, has_prev=False, sigma_override=sig)
+    P = gq.stats.cpu().numpy()[:, 3]
+    want = O.density_count(g, np.full(16, 1e-9, np.float32)) / (2 * 36)
+    np.testing.assert_allclose(P, want, rtol=1e-6)
+
+
+def test_without_layer_codes():
+    g, _, _ = synth.channel_mixed_grad(2, 32, 5, 5, seed=6)
+    gq = GradQuant(2, 32, 5, 5)
+    gq.run(dev_input(g, False, api.NHWC), api.NHWC, 3, has_prev=False, with_gq=False)
+    assert bool((gq.gq == 77).all().item())  # untouched
+    s = gq.s_state.cpu().numpy()
+    np.testing.assert_array_equal(codes_to_nchw(gq.vq, 32), O.quantize(g, s, True, 3, 0))
+
+
+@pytest.mark.parametrize("layout", [api.NHWC, api.NCHW])
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("shape", [(2, 64, 14, 14), (1, 3, 17, 19), (64, 3, 7, 7), (2, 40, 3, 5)])
+def test_quantize_tensor(shape, layout, bf16):
+    N, C, H, W = shape
+    x = synth.activations(N, C, H, W, seed=7) - np.float32(0.3)
+    if bf16:
+        x = synth.round_to_bf16(x)
+    Cp = api.padded_channels(C)
+    d = dev_input(x, bf16, layout)
+    q = torch.full((N, H, W, Cp), 55, dtype=torch.int8, device="cuda")
+    s = scalar(0.0)
+    api.quantize_tensor(d, layout, N, C, H, W, api.SCALE_ABSMAX, s, api.ROUND_NEAREST_EVEN, 0, q)
+    torch.cuda.synchronize()
+    assert float(s.item()) == float(np.abs(x).max())
+    np.testing.assert_array_equal(codes_to_nchw(q, C), O.quantize(x, float(s.item())))
+    assert padding_is_zero(q, C)
+    # given scale (clipping) and stochastic rounding
+    s2 = scalar(0.5)
+    api.quantize_tensor(d, layout, N, C, H, W, api.SCALE_GIVEN, s2, api.ROUND_STOCHASTIC, 11, q)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(codes_to_nchw(q, C), O.quantize(x, 0.5, stochastic=True, seed=11))
+
+
+def test_weight_layout_from_quantize_tensor():
+    """Weights passed as an NCHW tensor (N=Cout, C=Cin, H=R, W=S) come out as [Cout][R][S][Cinp]."""
+    w = synth.weights(8, 5, 3, 3, seed=8)
+    q = torch.empty((8, 3, 3, 16), dtype=torch.int8, device="cuda")
+    s = scalar(0.0)
+    api.quantize_tensor(torch.from_numpy(w).cuda(), api.NCHW, 8, 5, 3, 3, api.SCALE_ABSMAX, s,
+                        api.ROUND_NEAREST_EVEN, 0, q)
+    torch.cuda.synchronize()
+    want = O.quantize(w, float(np.abs(w).max()))           # (Cout,Cin,R,S)
+    np.testing.assert_array_equal(q.cpu().numpy()[..., :5], want.transpose(0, 2, 3, 1))
+
+
+def test_config2_full_size_grad_quant():
+    """ResNet-50 conv2_x 3x3 layer: dY (64,64,56,56) bf16 NHWC, the launch configuration the
+    benchmark times; full-tensor comparison (the oracle's O(elements) parts run in seconds)."""
+    g, _, _ = synth.channel_mixed_grad(64, 64, 56, 56, seed=9)
+    g = synth.round_to_bf16(g)
+    check_grad_quant(g, True, api.NHWC, iters=2)
