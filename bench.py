@@ -1,0 +1,401 @@
+#!/usr/bin/env python
+"""Benchmark of the dai8 hot path on one B200 (or N independent replicas, one per GPU).
+
+Workload: the ResNet-50 conv2_x bottleneck block (1x1 256->64, 3x3 64->64 pad 1, 1x1 64->256) at
+N=64, 56x56, bf16 NHWC inputs, synthetic tensors (X = ReLU(N(0,1)), He weights, per-channel
+bell-shaped / long-tailed dY).  One step = the whole path for the three layers: forward
+quantization of X and W, int8 forward conv, gradient vectorized quantization of dY (statistics,
+density count, clip update, vq + gq codes), int8 dW and dX convs with de-quantizing epilogues.
+
+Prints ONE JSON line.  `value` = int8 backward-convolution throughput, 2*MACs(dX+dW) of the step
+divided by the time of the WHOLE step (quantization and the forward conv included), in TOPS, summed
+over ranks.  `detail` holds the per-call breakdown measured with CUDA events inside the same timed
+region, `roofline` the dominant call, `e2e` the same metric with pinned-host inputs and outputs
+copied inside the timed region, `cpu_baseline` the CPU oracle on a bounded sample of the workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "int8 conv-backward TOPS (dX+dW)"
+UNIT = "TOPS"
+WORKLOAD = "resnet50_conv2x_bottleneck_N64_56x56_bf16_nhwc"
+BATCH = 64
+SEED = 2024
+INT8_OVER_BF16 = 2.0   # nominal dense ratio 4.5 / 2.25 PFLOP/s
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_burst": p["bf16_tflops"],
+                "bf16_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_burst": 1590.0, "bf16_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle arm (cpu_baseline leg and --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_step(inputs):
+    """The whole path for a list of (layer, x, w, g) with the CPU oracle, as it stands."""
+    from oracle import cpu as O
+    for L, x, w, g in inputs:
+        sx, sw = float(np.abs(x).max()), float(np.abs(w).max())
+        qx, qw = O.quantize(x, sx), O.quantize(w, sw)
+        O.dequant_acc(O.conv_fwd_acc(qx, qw, L.stride, L.pad)[0], sx, sw)
+        absmax, _, sigma, gl = O.channel_stats(g)
+        cnt = O.density_count(g, sigma)
+        s, _ = O.classify_clip(cnt, absmax, g.size // g.shape[1])
+        vq = O.quantize(g, s, True, SEED, 0)
+        gq = O.quantize(g, gl, True, SEED, 1)
+        O.dequant_acc(O.conv_bwd_filter_acc(qx, vq, (L.R, L.S), L.stride, L.pad)[0], sx, s)
+        O.dequant_acc(O.conv_bwd_data_acc(gq, qw, (L.H, L.W), L.stride, L.pad)[0], gl, sw)
+
+
+def oracle_inputs(batch):
+    from paper_2102_04782_b200 import synth
+    out = []
+    for i, L in enumerate(synth.resnet50_conv2x_block()):
+        x, w, g, _, _ = synth.layer_inputs(L, batch, SEED + i, bf16=True)
+        out.append((L, x, w, g))
+    return out
+
+
+def bwd_ops(layers, batch):
+    return sum(2 * 2 * L.macs(batch) for L in layers)   # dX + dW, 2 ops per MAC
+
+
+def time_oracle(batch, steps, warmup):
+    from oracle import cpu as O
+    from paper_2102_04782_b200 import synth
+    inputs = oracle_inputs(batch)
+    for _ in range(warmup):
+        oracle_step(inputs)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle_step(inputs)
+    dt = (time.perf_counter() - t0) / steps
+    ops = bwd_ops(synth.resnet50_conv2x_block(), batch)
+    return ops / dt / 1e12, dt, O.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    batch = 4
+    value, dt, cores = time_oracle(batch, args.steps, args.warmup)
+    sample = f"same three layers at batch {batch} of {BATCH} per step (bounded sample), CPU oracle as it stands"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA arm
+# ------------------------------------------------------------------------------------------------
+class LayerBuffers:
+    def __init__(self, L, N, seed, torch, api, synth, dev):
+        self.L, self.N = L, N
+        x, w, g, _, _ = synth.layer_inputs(L, N, seed, bf16=True)
+        bf = torch.bfloat16
+        self.h_x = torch.from_numpy(x).permute(0, 2, 3, 1).contiguous().to(bf).pin_memory()
+        self.h_w = torch.from_numpy(w).to(bf).pin_memory()
+        self.h_g = torch.from_numpy(g).permute(0, 2, 3, 1).contiguous().to(bf).pin_memory()
+        self.x, self.w, self.g = self.h_x.to(dev), self.h_w.to(dev), self.h_g.to(dev)
+        self.geom = api.ConvGeom(N, L.Cin, L.Cout, L.H, L.W, L.R, L.S, L.stride, L.stride, L.pad, L.pad)
+        Cip, Cop = api.padded_channels(L.Cin), api.padded_channels(L.Cout)
+        i8 = dict(dtype=torch.int8, device=dev)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.qX = torch.empty((N, L.H, L.W, Cip), **i8)
+        self.qW = torch.empty((L.Cout, L.R, L.S, Cip), **i8)
+        self.vq = torch.empty((N, L.P, L.Q, Cop), **i8)
+        self.gq = torch.empty((N, L.P, L.Q, Cop), **i8)
+        self.sX, self.sW, self.gmax = torch.zeros(1, **f32), torch.zeros(1, **f32), torch.zeros(1, **f32)
+        self.s_state = torch.zeros(L.Cout, **f32)
+        self.Y = torch.empty((N, L.P, L.Q, L.Cout), dtype=bf, device=dev)
+        self.dX = torch.empty((N, L.H, L.W, L.Cin), dtype=bf, device=dev)
+        self.dW = torch.empty((L.Cout, L.Cin, L.R, L.S), **f32)
+        u8 = dict(dtype=torch.uint8, device=dev)
+        self.ws_g = torch.empty(api.quantize_grad_workspace_bytes(L.Cout), **u8)
+        self.ws_f = torch.empty(api.conv_workspace_bytes(api.OP_FWD, self.geom), **u8)
+        self.ws_d = torch.empty(api.conv_workspace_bytes(api.OP_BWD_DATA, self.geom), **u8)
+        self.ws_w = torch.empty(api.conv_workspace_bytes(api.OP_BWD_FILTER, self.geom), **u8)
+        self.h_Y = torch.empty(self.Y.shape, dtype=bf).pin_memory()
+        self.h_dX = torch.empty(self.dX.shape, dtype=bf).pin_memory()
+        self.h_dW = torch.empty(self.dW.shape, dtype=torch.float32).pin_memory()
+        self.has_prev = False
+        self.h2d = sum(t.numel() * t.element_size() for t in (self.h_x, self.h_w, self.h_g))
+        self.d2h = sum(t.numel() * t.element_size() for t in (self.h_Y, self.h_dX, self.h_dW))
+        npix_in, npix_out = N * L.H * L.W, N * L.P * L.Q
+        wbytes = L.Cout * L.R * L.S * Cip
+        # algorithmic bytes / ops per call (operands once, outputs once)
+        self.alg = {
+            "quantize_x": {"bytes": npix_in * L.Cin * 2 + npix_in * Cip},
+            "quantize_w": {"bytes": L.Cout * L.Cin * L.R * L.S * 2 + wbytes},
+            "conv_fwd": {"bytes": npix_in * Cip + wbytes + npix_out * L.Cout * 2, "ops": 2 * L.macs(N)},
+            "quantize_grad": {"bytes": npix_out * L.Cout * 2 + 2 * npix_out * Cop},
+            "conv_bwd_filter": {"bytes": npix_in * Cip + npix_out * Cop + L.Cout * L.Cin * L.R * L.S * 4,
+                                "ops": 2 * L.macs(N)},
+            "conv_bwd_data": {"bytes": npix_out * Cop + wbytes + npix_in * L.Cin * 2, "ops": 2 * L.macs(N)},
+        }
+
+    def calls(self, api, seed):
+        L, N = self.L, self.N
+        return [
+            ("quantize_x", lambda: api.quantize_tensor(self.x, api.NHWC, N, L.Cin, L.H, L.W, api.SCALE_ABSMAX,
+                                                       self.sX, api.ROUND_NEAREST_EVEN, 0, self.qX)),
+            ("quantize_w", lambda: api.quantize_tensor(self.w, api.NCHW, L.Cout, L.Cin, L.R, L.S, api.SCALE_ABSMAX,
+                                                       self.sW, api.ROUND_NEAREST_EVEN, 0, self.qW)),
+            ("conv_fwd", lambda: api.conv_fwd(self.qX, self.qW, self.sX, self.sW, self.geom, self.Y, api.NHWC,
+                                              self.ws_f)),
+            ("quantize_grad", lambda: api.quantize_grad(self.g, api.NHWC, N, L.Cout, L.P, L.Q, None, self.s_state,
+                                                        self.has_prev, self.gmax, None, None, self.vq, self.gq,
+                                                        seed, self.ws_g)),
+            ("conv_bwd_filter", lambda: api.conv_bwd_filter(self.qX, self.vq, self.sX, self.s_state, self.geom,
+                                                            self.dW, self.ws_w)),
+            ("conv_bwd_data", lambda: api.conv_bwd_data(self.gq, self.qW, self.gmax, self.sW, self.geom, self.dX,
+                                                        api.NHWC, self.ws_d)),
+        ]
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            p = [t.strip() for t in line.split(",")]
+            if len(p) < 7:
+                continue
+            try:
+                sm.append(float(p[0])); mx.append(float(p[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, p[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def run_dai8(args):
+    import torch
+    from paper_2102_04782_b200 import api, synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device; there is no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    api.lib()
+
+    layers = synth.resnet50_conv2x_block()
+    bufs = [LayerBuffers(L, BATCH, SEED + i, torch, api, synth, dev) for i, L in enumerate(layers)]
+    step_no = [0]
+
+    def step(record=None):
+        seed = SEED + step_no[0]
+        for b in bufs:
+            for name, fn in b.calls(api, seed):
+                if record is not None:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
+                fn()
+                if record is not None:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
+                    record.append((b.L.name, name, e0, e1))
+            b.has_prev = True
+        step_no[0] += 1
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if dist is None:
+            return ms
+        t = torch.tensor([ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+
+    # ---- timed region: K steps, device-timed, per-call events inside -----------------------------
+    sampler = ClockSampler(local) if rank == 0 else None
+    launches0 = api.launch_count()
+    records = []
+    barrier()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        step(records)
+    t1.record()
+    barrier()
+    total_ms = max_over_ranks(t0.elapsed_time(t1))
+    launches = api.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    assert api.get_device_status() == api.OK
+    ms_per_step = total_ms / args.steps
+    ops_step = bwd_ops(layers, BATCH)
+    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end: pinned host inputs -> device, results -> pinned host, every step ------------
+    def e2e_step():
+        for b in bufs:
+            b.x.copy_(b.h_x, non_blocking=True); b.w.copy_(b.h_w, non_blocking=True)
+            b.g.copy_(b.h_g, non_blocking=True)
+        step()
+        for b in bufs:
+            b.h_Y.copy_(b.Y, non_blocking=True); b.h_dX.copy_(b.dX, non_blocking=True)
+            b.h_dW.copy_(b.dW, non_blocking=True)
+    e2e_step()
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    e2e_value = world * ops_step / (e2e_ms * 1e-3) / 1e12
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    # ---- per-call breakdown and roofline of the dominant call -------------------------------------
+    peaks = measured_peaks()
+    agg = {}
+    for lname, cname, a, b_ in records:
+        agg.setdefault((lname, cname), []).append(a.elapsed_time(b_))
+    alg = {(b.L.name, k): v for b in bufs for k, v in b.alg.items()}
+    detail, dominant = [], None
+    sustained = total_ms > 1000.0
+    int8_peak = INT8_OVER_BF16 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
+    ridge = int8_peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    for key, times in agg.items():
+        ms = sum(times) / len(times)
+        a = alg[key]
+        ent = {"layer": key[0], "call": key[1], "ms": round(ms, 5), "gbs": round(a["bytes"] / ms / 1e6, 1)}
+        if "ops" in a:
+            ent["tops"] = round(a["ops"] / ms / 1e9, 2)
+            ent["bound"] = "tensor" if a["ops"] / a["bytes"] > ridge else "hbm"
+        else:
+            ent["bound"] = "hbm"
+        detail.append(ent)
+        if dominant is None or ms > dominant[0]:
+            dominant = (ms, key, ent)
+    dms, dkey, dent = dominant
+    if dent["bound"] == "tensor":
+        achieved, peak, unit = alg[dkey]["ops"] / dms / 1e9, int8_peak, "TOPS"
+    else:
+        achieved, peak, unit = alg[dkey]["bytes"] / dms / 1e6, peaks["hbm_gbs"], "GB/s"
+    roofline = {"bound": dent["bound"], "achieved": round(achieved, 2), "peak": peak, "unit": unit,
+                "frac": round(achieved / peak, 4), "traffic": None,
+                "kernel": f"{dkey[1]} @ {dkey[0]}", "peak_source": peaks["source"],
+                "peak_kind": ("int8 = 2 x bf16 " + ("sustained" if sustained else "burst")) if unit == "TOPS" else "copy"}
+    def phase_ms(names):
+        return sum(e["ms"] for e in detail if e["call"] in names)
+    conv_bwd_ms = phase_ms(("conv_bwd_filter", "conv_bwd_data"))
+    gvq_ms = phase_ms(("quantize_grad",))
+    gvq_bytes = sum(b.alg["quantize_grad"]["bytes"] for b in bufs)
+    summary = {
+        "conv_bwd_tops_calls_only": round(ops_step / conv_bwd_ms / 1e9, 2),
+        "conv_bwd_frac_int8_peak": round(ops_step / conv_bwd_ms / 1e9 / int8_peak, 4),
+        "gvq_effective_gbs": round(gvq_bytes / gvq_ms / 1e6, 1),
+        "gvq_frac_hbm": round(gvq_bytes / gvq_ms / 1e6 / peaks["hbm_gbs"], 4),
+        "int8_peak_tops": int8_peak, "hbm_peak_gbs": peaks["hbm_gbs"], "calls": detail,
+    }
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        cb = 8
+        v, dt, cores = time_oracle(cb, 1, 0)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"same three layers at batch {cb} of {BATCH}, one pass, {dt:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "layers": [l.name for l in layers], "batch": BATCH,
+                   "outputs": "Y,dX bf16 NHWC; dW fp32", "l2": "inputs larger than L2 (about 0.9 GB touched per step)",
+                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3),
+                "h2d_bytes_per_step": int(sum(b.h2d for b in bufs)),
+                "d2h_bytes_per_step": int(sum(b.d2h for b in bufs))},
+        "roofline": roofline, "cpu_baseline": cpu, "detail": summary,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="dai8", choices=["dai8", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_dai8(args)
+
+
+if __name__ == "__main__":
+    main()
