@@ -1,4 +1,22 @@
-// Tensor-core (tcgen05) convolution kernels.  Placeholder: nothing is routed here yet.
+// Tensor-core convolutions for sm_100a: implicit GEMM on tcgen05.mma.kind::i8 with int32
+// accumulators in tensor memory, operands staged in shared memory by TMA.
+//
+// Forward and input-gradient convolutions (Fig. 2; Eq. 3) share one kernel: the output is a
+// matrix [pixels][channels], D[m][j] = sum over filter taps t and contraction channels k of
+// A[pixel(m) + offset(t)][k] * B[j][t][k].  A is an NHWC code tensor read with TMA in im2col mode
+// (128 consecutive output pixels per tile, padding filled with zeros by the copy engine), B the
+// weight codes [rows][taps][channels] read with a tiled TMA box; both land in shared memory in the
+// K-major swizzled layout the MMA descriptors name.  For the input gradient A is q(G) and B the
+// transposed, tap-mirrored weights, with padding R-1-pad.
+//
+// Roles inside a CTA of 192 threads: warp 0 issues TMA loads, warp 1 owns the tensor memory and
+// issues the MMAs (one elected lane), warps 2-5 read the accumulators back (tcgen05.ld), apply the
+// de-quantization scale and store.  Stages are handed over with mbarriers; every wait is bounded
+// and a wait that expires records DAI8_ERR_TIMEOUT in the device status word instead of hanging.
+#include <cuda.h>
+
+#include <mutex>
+
 #include "conv_internal.cuh"
 
 namespace dai8 {
@@ -14,13 +32,462 @@ dai8_status read_clear_device_status(int* host_status, cudaStream_t stream) {
   return DAI8_OK;
 }
 
-bool umma_fwd_supported(const ConvShape&) { return false; }
-bool umma_bwd_data_supported(const ConvShape&) { return false; }
+namespace {
+
+constexpr int kBM = 128;                      // output pixels per tile (MMA M)
+constexpr int kThreadsIgemm = 192;
+constexpr long long kTimeoutCycles = 2000000000LL;  // about one second
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is aborting (this wait or another one expired).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kTimeoutCycles) {
+      *abort_flag = 1u;
+      atomicExch(&g_device_status, (unsigned int)DAI8_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void tma_load_im2col_4d(const CUtensorMap* map, uint64_t* bar, void* dst, int c,
+                                                   int w, int h, int n, uint16_t off_w, uint16_t off_h) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h),
+        "r"(n), "h"(off_w), "h"(off_h)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_tile_3d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0,
+                                                 int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
+  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
+               "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+               : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], int8 x int8 -> int32, one instruction covers K = 32.
+__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+      : "memory");
+}
+// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i).
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor for a K-major operand tile [rows][kc_bytes] written by TMA with
+// the matching swizzle (rows of 32/64/128 bytes; groups of 8 rows are `8*kc_bytes` apart).
+__device__ __forceinline__ uint64_t kmajor_desc(uint32_t saddr, int kc_bytes) {
+  const uint64_t layout = kc_bytes == 128 ? 2ull : (kc_bytes == 64 ? 4ull : 6ull);
+  const uint64_t sbo = (uint64_t)(8 * kc_bytes) >> 4;
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (sbo << 32) | (1ull << 46) | (layout << 61);
+}
+// Instruction descriptor: int32 accumulator, signed 8-bit A and B, both K-major, M = 128, N = bn.
+__device__ __forceinline__ uint32_t idesc_i8_kmajor(int bn) {
+  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
+}
+
+struct IgemmParams {
+  int Mtot, P, Q;        // output pixels and output extent (pixel m = (n*P + p)*Q + q)
+  int Nout;              // real output channels
+  int R, S;              // filter taps
+  int kc_bytes;          // contraction bytes per chunk: 32, 64 or 128
+  int chunks_per_tap;    // ceil(contraction channels / kc_bytes)
+  int G;                 // chunks per pipeline stage
+  int k_iters;           // ceil(R*S*chunks_per_tap / G)
+  int BN;                // output channels per tile (multiple of 16, <= 256)
+  int tmem_cols;         // power of two >= max(32, BN)
+  int stages;
+  int sh, sw, lower_h, lower_w;  // pixel (p,q) reads input (lower_h + p*sh + r, lower_w + q*sw + s)
+  ConvOut out;
+  const float* sa;
+  const float* sb;
+};
+
+__global__ void __launch_bounds__(kThreadsIgemm, 1)
+igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
+                    const IgemmParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[8], empty_bar[8], acc_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile uint32_t abort_flag;
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int a_chunk_bytes = kBM * prm.kc_bytes;
+  const int b_chunk_bytes = prm.BN * prm.kc_bytes;
+  const int stage_bytes = prm.G * (a_chunk_bytes + b_chunk_bytes);
+  const int total_chunks = prm.R * prm.S * prm.chunks_per_tap;
+
+  // the last tile is shifted back so that every tile covers 128 existing pixels
+  int m0 = blockIdx.x * kBM;
+  if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
+  const int n0 = blockIdx.y * prm.BN;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    for (int s = 0; s < prm.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&acc_bar, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_slot, (uint32_t)prm.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&mapA);
+      tma_prefetch_desc(&mapB);
+      const int q0 = m0 % prm.Q;
+      const int t = m0 / prm.Q;
+      const int p0 = t % prm.P, img = t / prm.P;
+      const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
+      for (int it = 0; it < prm.k_iters; ++it) {
+        const int s = it % prm.stages;
+        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag)) break;
+        const int c_begin = it * prm.G;
+        const int c_end = min(total_chunks, c_begin + prm.G);
+        mbar_expect_tx(&full_bar[s], (uint32_t)((c_end - c_begin) * (a_chunk_bytes + b_chunk_bytes)));
+        uint8_t* sa = smem + (size_t)s * stage_bytes;
+        uint8_t* sb = sa + prm.G * a_chunk_bytes;
+        for (int c = c_begin; c < c_end; ++c) {
+          const int tap = c / prm.chunks_per_tap;
+          const int k0 = (c - tap * prm.chunks_per_tap) * prm.kc_bytes;
+          const int r = tap / prm.S, ss = tap - r * prm.S;
+          tma_load_im2col_4d(&mapA, &full_bar[s], sa + (c - c_begin) * a_chunk_bytes, k0, cw, ch, img,
+                             (uint16_t)ss, (uint16_t)r);
+          tma_load_tile_3d(&mapB, &full_bar[s], sb + (c - c_begin) * b_chunk_bytes, k0, tap, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = idesc_i8_kmajor(prm.BN);
+      uint32_t accumulate = 0;
+      bool ok = true;
+      for (int it = 0; it < prm.k_iters && ok; ++it) {
+        const int s = it % prm.stages;
+        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const int c_begin = it * prm.G;
+        const int c_end = min(total_chunks, c_begin + prm.G);
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t sb = sa + prm.G * a_chunk_bytes;
+        for (int c = 0; c < c_end - c_begin; ++c) {
+          const uint64_t ad = kmajor_desc(sa + c * a_chunk_bytes, prm.kc_bytes);
+          const uint64_t bd = kmajor_desc(sb + c * b_chunk_bytes, prm.kc_bytes);
+          for (int kk = 0; kk < prm.kc_bytes / 32; ++kk) {
+            mma_i8(tmem_base, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, accumulate);
+            accumulate = 1;
+          }
+        }
+        tc_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+      }
+      if (ok) tc_commit(&acc_bar);  // accumulator complete
+    }
+  } else {
+    // epilogue: warp w may touch tensor-memory lanes 32*(w%4) .. 32*(w%4)+31
+    const int quarter = warp & 3;
+    const bool ok = mbar_wait(&acc_bar, 0, &abort_flag);
+    tc_fence_after();
+    if (ok) {
+      const int m = m0 + quarter * 32 + lane;
+      const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
+      const int q = m % prm.Q;
+      const int t = m / prm.Q;
+      const int p = t % prm.P, img = t / prm.P;
+      const bool nhwc = prm.out.layout == DAI8_NHWC;
+      const size_t pix_base = nhwc ? (size_t)m * prm.Nout : 0;
+      const size_t plane = (size_t)prm.P * prm.Q;
+      for (int cg = 0; cg < prm.BN / 16; ++cg) {
+        int v[16];
+        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cg * 16), v);
+        tmem_ld_wait();
+        const int j0 = n0 + cg * 16;
+        if (j0 >= prm.Nout) break;
+        if (nhwc && j0 + 16 <= prm.Nout && (prm.Nout & 15) == 0) {
+          if (prm.out.dtype == DAI8_F32) {
+            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.out.ptr) + pix_base + j0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+              dst[i] = make_float4(__fmul_rn(__int2float_rn(v[4 * i]), scale), __fmul_rn(__int2float_rn(v[4 * i + 1]), scale),
+                                   __fmul_rn(__int2float_rn(v[4 * i + 2]), scale), __fmul_rn(__int2float_rn(v[4 * i + 3]), scale));
+          } else if (prm.out.dtype == DAI8_BF16) {
+            uint32_t w[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+              w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i]), scale)) |
+                     ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i + 1]), scale)) << 16);
+            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(prm.out.ptr) + pix_base + j0);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+          } else {
+            int4* dst = reinterpret_cast<int4*>(static_cast<int*>(prm.out.ptr) + pix_base + j0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) dst[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+          }
+        } else {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int j = j0 + i;
+            if (j < prm.Nout) {
+              const size_t idx = nhwc ? pix_base + j : ((size_t)img * prm.Nout + j) * plane + (size_t)p * prm.Q + q;
+              store_result(prm.out.ptr, prm.out.dtype, idx, v[i], scale);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  // teardown: everything this CTA issued must have drained before tensor memory is released
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    // a wait expired: give in-flight copies and MMAs time to land before the CTA's resources go
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)prm.tmem_cols);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side: tensor maps and launch
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
+                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+std::once_flag g_driver_once;
+
+bool load_driver_entry_points() {
+  std::call_once(g_driver_once, [] {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
+  });
+  return g_encode_tiled && g_encode_im2col;
+}
+
+CUtensorMapSwizzle swizzle_for(int kc_bytes) {
+  return kc_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
+                         : (kc_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+}
+
+// Contraction bytes per chunk for a code tensor with `cp` channels (multiple of 16, >= 32).
+int chunk_bytes_for(int cp) {
+  if (cp % 128 == 0) return 128;
+  if (cp % 64 == 0) return 64;
+  if (cp >= 128) return 128;  // ragged tail chunk, zero-filled by the copy engine
+  if (cp >= 64) return 64;
+  return 32;
+}
+
+struct IgemmProblem {
+  const int8_t* A;  // [N][Hi][Wi][Kc]
+  const int8_t* B;  // [Brows][R*S][Kc]
+  int N, Hi, Wi, Kc, Brows;
+  int P, Q, Nout, R, S, sh, sw, lower_h, lower_w;
+};
+
+bool igemm_supported(const IgemmProblem& pb) {
+  if (pb.Kc < 32) return false;
+  if ((int64_t)pb.N * pb.P * pb.Q < kBM) return false;
+  // small activation tensors stay on the direct kernels (im2col descriptors of tiny tensors are
+  // not relied upon)
+  if ((int64_t)pb.N * pb.Hi * pb.Wi * pb.Kc < 131072) return false;
+  if (pb.sh > 8 || pb.sw > 8 || pb.R > 16 || pb.S > 16) return false;
+  if (pb.lower_h < -16 || pb.lower_w < -16 || pb.lower_h > 0 || pb.lower_w > 0) return false;
+  if (pb.Nout < 1) return false;
+  return true;
+}
+
+dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* sb, const ConvOut& out,
+                         cudaStream_t st) {
+  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
+  IgemmParams prm;
+  prm.Mtot = pb.N * pb.P * pb.Q;
+  prm.P = pb.P; prm.Q = pb.Q; prm.Nout = pb.Nout; prm.R = pb.R; prm.S = pb.S;
+  prm.kc_bytes = chunk_bytes_for(pb.Kc);
+  prm.chunks_per_tap = (pb.Kc + prm.kc_bytes - 1) / prm.kc_bytes;
+  prm.G = 128 / prm.kc_bytes;
+  const int total_chunks = pb.R * pb.S * prm.chunks_per_tap;
+  if (prm.G > total_chunks) prm.G = total_chunks;
+  prm.k_iters = (total_chunks + prm.G - 1) / prm.G;
+  const int noutp = round_up(pb.Nout, 16);
+  prm.BN = noutp < 256 ? noutp : 256;
+  if (noutp > 256 && noutp % 256 != 0 && noutp % 128 == 0) prm.BN = 128;
+  prm.tmem_cols = 32;
+  while (prm.tmem_cols < prm.BN) prm.tmem_cols *= 2;
+  const int stage_bytes = prm.G * (kBM + prm.BN) * prm.kc_bytes;
+  int stages = (200 * 1024) / stage_bytes;
+  if (stages > 8) stages = 8;
+  if (stages > prm.k_iters) stages = prm.k_iters;
+  if (stages < 1) return DAI8_ERR_UNSUPPORTED;
+  prm.stages = stages;
+  prm.sh = pb.sh; prm.sw = pb.sw; prm.lower_h = pb.lower_h; prm.lower_w = pb.lower_w;
+  prm.out = out; prm.sa = sa; prm.sb = sb;
+
+  CUtensorMap mapA, mapB;
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.Wi, (cuuint64_t)pb.Hi, (cuuint64_t)pb.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.Wi * pb.Kc, (cuuint64_t)pb.Hi * pb.Wi * pb.Kc};
+    // base pixel w ranges over [lower_w, Wi - 1 + upper_w]; there are Q of them at step sw
+    const int lower[2] = {pb.lower_w, pb.lower_h};
+    const int upper[2] = {pb.lower_w + (pb.Q - 1) * pb.sw - (pb.Wi - 1), pb.lower_h + (pb.P - 1) * pb.sh - (pb.Hi - 1)};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)pb.sw, (cuuint32_t)pb.sh, 1};
+    CUresult r = g_encode_im2col(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides,
+                                 lower, upper, (cuuint32_t)prm.kc_bytes, (cuuint32_t)kBM, estr,
+                                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)(pb.R * pb.S), (cuuint64_t)pb.Brows};
+    const cuuint64_t strides[2] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.R * pb.S * pb.Kc};
+    const cuuint32_t box[3] = {(cuuint32_t)prm.kc_bytes, 1, (cuuint32_t)prm.BN};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  }
+  const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+  static std::once_flag attr_once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(attr_once, [] {
+    attr_err = cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
+  });
+  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  const dim3 grid((unsigned)((prm.Mtot + kBM - 1) / kBM), (unsigned)((noutp + prm.BN - 1) / prm.BN), 1);
+  igemm_kmajor_kernel<<<grid, kThreadsIgemm, smem_bytes, st>>>(mapA, mapB, prm);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+IgemmProblem fwd_problem(const int8_t* qX, const int8_t* qW, const ConvShape& cs) {
+  IgemmProblem pb;
+  pb.A = qX; pb.B = qW;
+  pb.N = cs.N; pb.Hi = cs.H; pb.Wi = cs.W; pb.Kc = cs.Cinp; pb.Brows = cs.Cout;
+  pb.P = cs.P; pb.Q = cs.Q; pb.Nout = cs.Cout; pb.R = cs.R; pb.S = cs.S;
+  pb.sh = cs.sh; pb.sw = cs.sw; pb.lower_h = -cs.ph; pb.lower_w = -cs.pw;
+  return pb;
+}
+
+// Input gradient at stride 1: a forward convolution of q(G) with the mirrored, transposed filter
+// and padding R-1-pad.
+IgemmProblem bwd_data_problem(const int8_t* gq, const int8_t* wTflip, const ConvShape& cs) {
+  IgemmProblem pb;
+  pb.A = gq; pb.B = wTflip;
+  pb.N = cs.N; pb.Hi = cs.P; pb.Wi = cs.Q; pb.Kc = cs.Coutp; pb.Brows = cs.Cinp;
+  pb.P = cs.H; pb.Q = cs.W; pb.Nout = cs.Cin; pb.R = cs.R; pb.S = cs.S;
+  pb.sh = 1; pb.sw = 1; pb.lower_h = -(cs.R - 1 - cs.ph); pb.lower_w = -(cs.S - 1 - cs.pw);
+  return pb;
+}
+
+}  // namespace
+
+bool umma_fwd_supported(const ConvShape& cs) { return igemm_supported(fwd_problem(nullptr, nullptr, cs)); }
+
+bool umma_bwd_data_supported(const ConvShape& cs) {
+  if (cs.sh != 1 || cs.sw != 1) return false;
+  if (cs.ph > cs.R - 1 || cs.pw > cs.S - 1) return false;
+  return igemm_supported(bwd_data_problem(nullptr, nullptr, cs));
+}
+
 bool umma_bwd_filter_supported(const ConvShape&) { return false; }
-dai8_status umma_fwd(const int8_t*, const int8_t*, const float*, const float*, const ConvShape&,
-                     const ConvOut&, cudaStream_t) { return DAI8_ERR_UNSUPPORTED; }
-dai8_status umma_bwd_data(const int8_t*, const int8_t*, const float*, const float*, const ConvShape&,
-                          const ConvOut&, cudaStream_t) { return DAI8_ERR_UNSUPPORTED; }
+
+dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW, const ConvShape& cs,
+                     const ConvOut& out, cudaStream_t st) {
+  return launch_igemm(fwd_problem(qX, qW, cs), sX, sW, out, st);
+}
+
+dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* gmax, const float* sW,
+                          const ConvShape& cs, const ConvOut& out, cudaStream_t st) {
+  return launch_igemm(bwd_data_problem(gq, wTflip, cs), gmax, sW, out, st);
+}
+
 dai8_status umma_bwd_filter_acc(const int8_t*, const int8_t*, const ConvShape&, int*, cudaStream_t) {
   return DAI8_ERR_UNSUPPORTED;
 }
