@@ -466,6 +466,265 @@ IgemmProblem bwd_data_problem(const int8_t* gq, const int8_t* wTflip, const Conv
   return pb;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Weight gradient (Eq. 4): D[co][tap][ci] = sum over output pixels of vq[pix][co] * qX[pix+tap][ci].
+// The contraction runs over pixels, so with NHWC codes both operands are "MN-major" (the channel
+// index is contiguous, the contraction index strided): the paper's X -> X', G -> G' dimension
+// transformation is just the major-ness bit of the MMA descriptors, no transposed copy is made.
+// A CTA owns 128 output channels x (a group of taps) x (up to 256 input channels) in tensor memory
+// and a slice of the pixels; slices are combined with integer atomics (exact in any order).
+// ---------------------------------------------------------------------------------------------
+constexpr int kKP = 128;  // pixels per pipeline stage (4 MMAs of K = 32)
+
+struct WgradParams {
+  int npix, P, Q;
+  int Cout, Cinp, R, S;
+  int sh, sw, lower_h, lower_w;
+  int bw;                // channels per B box: 32, 64 or 128 (selects the swizzle)
+  int nb;                // B boxes per tap (1 or 2); MMA N = nb * bw
+  int tg;                // taps per CTA
+  int ci_tiles;
+  int chunks_total, chunks_per_split;
+  int stages, tmem_cols;
+  int* acc;              // [Cout][R*S][Cinp]
+};
+
+__device__ __forceinline__ uint64_t mnmajor_desc(uint32_t saddr, int width_bytes, uint32_t lbo_bytes) {
+  const uint64_t layout = width_bytes == 128 ? 2ull : (width_bytes == 64 ? 4ull : 6ull);
+  const uint64_t sbo = (uint64_t)(8 * width_bytes) >> 4;  // eight contraction rows
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | (sbo << 32) | (1ull << 46) |
+         (layout << 61);
+}
+
+__device__ __forceinline__ void tma_load_tile_2d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
+      : "memory");
+}
+
+__global__ void __launch_bounds__(kThreadsIgemm, 1)
+wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_constant__ CUtensorMap mapX,
+                     const WgradParams prm) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ uint64_t full_bar[8], empty_bar[8], acc_bar;
+  __shared__ uint32_t tmem_base_slot;
+  __shared__ volatile uint32_t abort_flag;
+  __shared__ int tr[4][32][33];
+
+  const int chunk_begin = blockIdx.x * prm.chunks_per_split;
+  const int k_iters = min(prm.chunks_total, chunk_begin + prm.chunks_per_split) - chunk_begin;
+  if (k_iters <= 0) return;  // uniform over the CTA
+
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int T = prm.R * prm.S;
+  const int grp = blockIdx.y / prm.ci_tiles, cit = blockIdx.y - grp * prm.ci_tiles;
+  const int Nw = prm.nb * prm.bw;
+  const int ci0 = cit * Nw;
+  const int co0 = blockIdx.z * kBM;
+  const int tap_begin = grp * prm.tg;
+  const int ntap = min(T, tap_begin + prm.tg) - tap_begin;
+  const int a_bytes = kKP * 128;
+  const int b_box_bytes = kKP * prm.bw;
+  const int stage_bytes = a_bytes + prm.tg * prm.nb * b_box_bytes;
+
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    for (int s = 0; s < prm.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    mbar_init(&acc_bar, 1);
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(&tmem_base_slot, (uint32_t)prm.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      tma_prefetch_desc(&mapG);
+      tma_prefetch_desc(&mapX);
+      for (int it = 0; it < k_iters; ++it) {
+        const int s = it % prm.stages;
+        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag)) break;
+        const int pix0 = (chunk_begin + it) * kKP;
+        const int q0 = pix0 % prm.Q;
+        const int t = pix0 / prm.Q;
+        const int p0 = t % prm.P, img = t / prm.P;
+        const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
+        mbar_expect_tx(&full_bar[s], (uint32_t)(a_bytes + ntap * prm.nb * b_box_bytes));
+        uint8_t* sa = smem + (size_t)s * stage_bytes;
+        uint8_t* sb = sa + a_bytes;
+        tma_load_tile_2d(&mapG, &full_bar[s], sa, co0, pix0);
+        for (int tl = 0; tl < ntap; ++tl) {
+          const int tap = tap_begin + tl;
+          const int r = tap / prm.S, ss = tap - r * prm.S;
+          for (int b = 0; b < prm.nb; ++b)
+            tma_load_im2col_4d(&mapX, &full_bar[s], sb + (tl * prm.nb + b) * b_box_bytes, ci0 + b * prm.bw, cw, ch,
+                               img, (uint16_t)ss, (uint16_t)r);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128, N = Nw
+      const uint32_t idesc = idesc_i8_kmajor(Nw) | (1u << 15) | (1u << 16);
+      bool ok = true;
+      for (int it = 0; it < k_iters && ok; ++it) {
+        const int s = it % prm.stages;
+        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t sb = sa + a_bytes;
+        const uint64_t ad = mnmajor_desc(sa, 128, (uint32_t)a_bytes);
+        for (int tl = 0; tl < ntap; ++tl) {
+          const uint64_t bd = mnmajor_desc(sb + tl * prm.nb * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
+          for (int kk = 0; kk < kKP / 32; ++kk)
+            mma_i8(tmem_base + (uint32_t)(tl * Nw), ad + (uint64_t)((kk * 32 * 128) >> 4),
+                   bd + (uint64_t)((kk * 32 * prm.bw) >> 4), idesc, (it > 0 || kk > 0) ? 1u : 0u);
+        }
+        tc_commit(&empty_bar[s]);
+      }
+      if (ok) tc_commit(&acc_bar);
+    }
+  } else {
+    const int quarter = warp & 3;
+    const bool ok = mbar_wait(&acc_bar, 0, &abort_flag);
+    tc_fence_after();
+    if (ok) {
+      int (*trw)[33] = tr[warp - 2];
+      for (int tl = 0; tl < ntap; ++tl) {
+        const int tap = tap_begin + tl;
+        for (int cg = 0; cg < Nw / 32; ++cg) {
+          int v0[16], v1[16];
+          const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(tl * Nw + cg * 32);
+          tmem_ld16(taddr, v0);
+          tmem_ld16(taddr + 16, v1);
+          tmem_ld_wait();
+          __syncwarp();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) { trw[lane][i] = v0[i]; trw[lane][16 + i] = v1[i]; }
+          __syncwarp();
+          const int ci = ci0 + cg * 32 + lane;
+          if (ci < prm.Cinp) {
+            for (int rr = 0; rr < 32; ++rr) {
+              const int co = co0 + quarter * 32 + rr;
+              if (co >= prm.Cout) break;
+              const int val = trw[rr][lane];
+              if (val != 0) atomicAdd(prm.acc + ((size_t)co * T + tap) * prm.Cinp + ci, val);
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (abort_flag) {
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)prm.tmem_cols);
+  }
+}
+
+bool wgrad_supported(const ConvShape& cs) {
+  if (cs.Cinp < 32) return false;
+  if ((int64_t)cs.N * cs.P * cs.Q < kKP) return false;
+  if ((int64_t)cs.N * cs.H * cs.W * cs.Cinp < 131072) return false;
+  if (cs.sh > 8 || cs.sw > 8 || cs.R > 16 || cs.S > 16 || cs.ph > 16 || cs.pw > 16) return false;
+  return true;
+}
+
+dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, cudaStream_t st) {
+  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
+  WgradParams prm;
+  prm.npix = cs.N * cs.P * cs.Q;
+  prm.P = cs.P; prm.Q = cs.Q; prm.Cout = cs.Cout; prm.Cinp = cs.Cinp; prm.R = cs.R; prm.S = cs.S;
+  prm.sh = cs.sh; prm.sw = cs.sw; prm.lower_h = -cs.ph; prm.lower_w = -cs.pw;
+  if (cs.Cinp >= 128) {
+    prm.bw = 128;
+    const int blocks128 = (cs.Cinp + 127) / 128;
+    prm.nb = (blocks128 % 2 == 0) ? 2 : 1;
+  } else {
+    prm.bw = cs.Cinp > 32 ? 64 : 32;
+    prm.nb = 1;
+  }
+  const int Nw = prm.nb * prm.bw;
+  prm.ci_tiles = (cs.Cinp + Nw - 1) / Nw;
+  const int T = cs.R * cs.S;
+  const int b_tap_bytes = prm.nb * kKP * prm.bw;
+  int tg_max = 512 / Nw;
+  const int tg_smem = (100 * 1024 - kKP * 128) / b_tap_bytes;
+  if (tg_max > tg_smem) tg_max = tg_smem;
+  if (tg_max < 1) return DAI8_ERR_UNSUPPORTED;
+  const int ngroups = (T + tg_max - 1) / tg_max;
+  prm.tg = (T + ngroups - 1) / ngroups;
+  prm.tmem_cols = 32;
+  while (prm.tmem_cols < prm.tg * Nw) prm.tmem_cols *= 2;
+  const int stage_bytes = kKP * 128 + prm.tg * b_tap_bytes;
+  int stages = (200 * 1024) / stage_bytes;
+  if (stages > 8) stages = 8;
+  prm.chunks_total = (prm.npix + kKP - 1) / kKP;
+  const int co_tiles = (cs.Cout + kBM - 1) / kBM;
+  const int tiles = ngroups * prm.ci_tiles * co_tiles;
+  int ksplit = 148 / tiles;
+  if (ksplit < 1) ksplit = 1;
+  if (ksplit > prm.chunks_total) ksplit = prm.chunks_total;
+  prm.chunks_per_split = (prm.chunks_total + ksplit - 1) / ksplit;
+  ksplit = (prm.chunks_total + prm.chunks_per_split - 1) / prm.chunks_per_split;
+  if (stages > prm.chunks_per_split) stages = prm.chunks_per_split;
+  if (stages < 1) return DAI8_ERR_UNSUPPORTED;
+  prm.stages = stages;
+  prm.acc = acc;
+
+  CUtensorMap mapG, mapX;
+  {
+    const cuuint64_t dims[2] = {(cuuint64_t)cs.Coutp, (cuuint64_t)prm.npix};
+    const cuuint64_t strides[1] = {(cuuint64_t)cs.Coutp};
+    const cuuint32_t box[2] = {128, (cuuint32_t)kKP};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  }
+  {
+    const cuuint64_t dims[4] = {(cuuint64_t)cs.Cinp, (cuuint64_t)cs.W, (cuuint64_t)cs.H, (cuuint64_t)cs.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)cs.Cinp, (cuuint64_t)cs.W * cs.Cinp, (cuuint64_t)cs.H * cs.W * cs.Cinp};
+    const int lower[2] = {-cs.pw, -cs.ph};
+    const int upper[2] = {-cs.pw + (cs.Q - 1) * cs.sw - (cs.W - 1), -cs.ph + (cs.P - 1) * cs.sh - (cs.H - 1)};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)cs.sw, (cuuint32_t)cs.sh, 1};
+    CUresult r = g_encode_im2col(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(qX), dims, strides, lower,
+                                 upper, (cuuint32_t)prm.bw, (cuuint32_t)kKP, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 swizzle_for(prm.bw), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  }
+  const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+  static std::once_flag attr_once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(attr_once, [] {
+    attr_err = cudaFuncSetAttribute(wgrad_mnmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    227 * 1024 - 20 * 1024);
+  });
+  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
+  wgrad_mnmajor_kernel<<<grid, kThreadsIgemm, smem_bytes, st>>>(mapG, mapX, prm);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
 }  // namespace
 
 bool umma_fwd_supported(const ConvShape& cs) { return igemm_supported(fwd_problem(nullptr, nullptr, cs)); }
@@ -476,7 +735,7 @@ bool umma_bwd_data_supported(const ConvShape& cs) {
   return igemm_supported(bwd_data_problem(nullptr, nullptr, cs));
 }
 
-bool umma_bwd_filter_supported(const ConvShape&) { return false; }
+bool umma_bwd_filter_supported(const ConvShape& cs) { return wgrad_supported(cs); }
 
 dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW, const ConvShape& cs,
                      const ConvOut& out, cudaStream_t st) {
@@ -488,8 +747,8 @@ dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* g
   return launch_igemm(bwd_data_problem(gq, wTflip, cs), gmax, sW, out, st);
 }
 
-dai8_status umma_bwd_filter_acc(const int8_t*, const int8_t*, const ConvShape&, int*, cudaStream_t) {
-  return DAI8_ERR_UNSUPPORTED;
+dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, cudaStream_t st) {
+  return launch_wgrad(qX, vq, cs, acc, st);
 }
 
 }  // namespace dai8

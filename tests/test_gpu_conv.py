@@ -86,7 +86,69 @@ def test_accumulators_bit_exact(g, backend):
         np.testing.assert_array_equal(dW, dw_o)
 
 
-@pytest.mark.parametrize("g", [GEOMS[0], GEOMS[3], GEOMS[6]])
+# Geometries large enough for the tensor-core kernels (activation tensors of at least 128 KiB),
+# chosen to hit every shared-memory swizzle width, ragged channel tails filled by the copy engine,
+# 256-wide accumulator tiles, tap groups, strides and a pixel count that is not a tile multiple.
+TC_GEOMS = [
+    (2, 128, 64, 32, 32, 1, 1, 1, 0),
+    (2, 64, 256, 48, 48, 1, 1, 1, 0),
+    (2, 64, 64, 34, 34, 3, 3, 1, 1),
+    (2, 64, 64, 34, 34, 3, 3, 2, 1),
+    (3, 48, 40, 33, 35, 3, 3, 1, 1),
+    (2, 256, 512, 24, 24, 1, 1, 1, 0),
+    (2, 144, 200, 24, 24, 3, 3, 1, 1),
+    (1, 32, 32, 70, 70, 5, 5, 1, 2),
+    (2, 384, 130, 16, 16, 1, 1, 1, 0),
+    (4, 128, 128, 20, 20, 1, 1, 2, 0),
+]
+
+
+@pytest.mark.parametrize("g", TC_GEOMS)
+def test_tensor_core_kernels_bit_exact(g):
+    """Backend 2 = tensor-core kernels only: a geometry they do not take raises instead of being
+    silently served by the direct kernels."""
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    rng = np.random.default_rng(33)
+    P, Q = O.out_hw(H, W, R, S, st, pad)
+    qX, qW, qG = rand_codes(rng, (N, Cin, H, W)), rand_codes(rng, (Cout, Cin, R, S)), rand_codes(rng, (N, Cout, P, Q))
+    s_c = np.ones(Cout, np.float32)
+    stride1 = st == 1
+    gg = geom(*g)
+    api.set_conv_backend(2)
+    try:
+        for layout in (api.NHWC, api.NCHW):
+            Y = torch.empty((N, P, Q, Cout) if layout == api.NHWC else (N, Cout, P, Q), dtype=torch.int32, device="cuda")
+            api.conv_fwd(codes_from_nchw(qX), weights_dev(qW), scalar(1), scalar(1), gg, Y, layout, None)
+            np.testing.assert_array_equal(out_to_nchw(Y, layout), O.conv_fwd_acc(qX, qW, st, pad)[0])
+            if stride1 and N * P * Q * ((Cout + 15) // 16 * 16) >= 131072:
+                dX = torch.empty((N, H, W, Cin) if layout == api.NHWC else (N, Cin, H, W), dtype=torch.int32, device="cuda")
+                api.conv_bwd_data(codes_from_nchw(qG), weights_dev(qW), scalar(1), scalar(1), gg, dX, layout,
+                                  ws_bytes(api.conv_workspace_bytes(api.OP_BWD_DATA, gg)))
+                np.testing.assert_array_equal(out_to_nchw(dX, layout), O.conv_bwd_data_acc(qG, qW, (H, W), st, pad)[0])
+        dW = torch.empty((Cout, Cin, R, S), dtype=torch.int32, device="cuda")
+        api.conv_bwd_filter(codes_from_nchw(qX), codes_from_nchw(qG), scalar(1), torch.from_numpy(s_c).cuda(), gg, dW,
+                            ws_bytes(api.conv_workspace_bytes(api.OP_BWD_FILTER, gg)))
+        np.testing.assert_array_equal(dW.cpu().numpy(), O.conv_bwd_filter_acc(qX, qG, (R, S), st, pad)[0])
+        assert api.get_device_status() == api.OK
+    finally:
+        api.set_conv_backend(0)
+
+
+def test_tensor_core_backend_refuses_small_shapes():
+    g = GEOMS[0]
+    gg = geom(*g)
+    api.set_conv_backend(2)
+    try:
+        with pytest.raises(api.Dai8Error) as e:
+            api.conv_fwd(torch.zeros((8, 14, 14, 64), dtype=torch.int8, device="cuda"),
+                         torch.zeros((64, 3, 3, 64), dtype=torch.int8, device="cuda"), scalar(1), scalar(1), gg,
+                         torch.zeros((8, 14, 14, 64), dtype=torch.int32, device="cuda"), api.NHWC, None)
+        assert e.value.code == api.ERR_UNSUPPORTED
+    finally:
+        api.set_conv_backend(0)
+
+
+@pytest.mark.parametrize("g", [GEOMS[0], GEOMS[3], GEOMS[6], TC_GEOMS[2], TC_GEOMS[6]])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_dequantized_outputs(g, dtype):
     N, Cin, Cout, H, W, R, S, st, pad = g
@@ -179,6 +241,21 @@ def test_config2_layers_sampled(li):
     layer = synth.resnet50_conv2x_block()[li]
     g = (64, layer.Cin, layer.Cout, layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad)
     _sample_check(g, np.random.default_rng(50 + li))
+
+
+def test_config2_kernel_families_agree_on_whole_tensors():
+    """Full-size 3x3 layer of the benchmark: the tensor-core kernels and the direct kernels are
+    independent implementations; every accumulator of Y, dX and dW must be identical."""
+    layer = synth.resnet50_conv2x_block()[1]
+    g = (64, layer.Cin, layer.Cout, layer.H, layer.W, layer.R, layer.S, layer.stride, layer.pad)
+    rng = np.random.default_rng(60)
+    qX, qW, qG = rand_codes(rng, (64, 64, 56, 56)), rand_codes(rng, (64, 64, 3, 3)), rand_codes(rng, (64, 64, 56, 56))
+    qG = (qG.astype(np.int16) * (rng.random(qG.shape) < 0.02)).astype(np.int8)
+    s_c = np.ones(64, np.float32)
+    a = run_all(g, qX, qW, qG, 1.0, 1.0, 1.0, s_c, torch.int32, api.NHWC, backend=1)
+    b = run_all(g, qX, qW, qG, 1.0, 1.0, 1.0, s_c, torch.int32, api.NHWC, backend=2)
+    for x, y in zip(a, b):
+        np.testing.assert_array_equal(x, y)
 
 
 def test_unsupported_and_errors():
