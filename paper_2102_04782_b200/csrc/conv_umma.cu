@@ -32,6 +32,12 @@ dai8_status read_clear_device_status(int* host_status, cudaStream_t stream) {
   return DAI8_OK;
 }
 
+unsigned int* device_status_address() {
+  void* p = nullptr;
+  if (cudaGetSymbolAddress(&p, g_device_status) != cudaSuccess) return nullptr;
+  return static_cast<unsigned int*>(p);
+}
+
 namespace {
 
 constexpr int kBM = 128;                      // output pixels per tile (MMA M)

@@ -20,6 +20,8 @@ inline void note_launch(int n = 1) { g_launch_count.fetch_add((uint64_t)n, std::
 
 // Reads and clears the device status word kept beside the tensor-core kernels (conv_umma.cu).
 dai8_status read_clear_device_status(int* host_status, cudaStream_t stream);
+// Device address of that status word on the current device (nullptr on failure).
+unsigned int* device_status_address();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }

@@ -14,6 +14,8 @@
 // (4 fp32 / 8 bf16) of one pixel and walks down the pixels, so per-channel scalars stay in
 // registers and every load/store instruction of a warp covers contiguous memory.  NCHW inputs are
 // read along H*W per (n, c) row and transposed through shared memory when codes are written.
+#include <mutex>
+
 #include "dai8_common.cuh"
 
 namespace dai8 {
@@ -27,6 +29,7 @@ struct GvqWs {
   uint32_t* ticket2;    // [1] arrival counter of the count sweep
   uint32_t* cnt;        // [C] density counts
   uint32_t* gmax_bits;  // [1] layer |g|max as the bit pattern of a non-negative float
+  uint32_t* gridbar;    // [1] arrival counter of the fused kernel's grid barriers
   float* absmax;        // [C]
   float* mean;          // [C]
   float* sigma;         // [C]
@@ -53,6 +56,7 @@ GvqWs carve(void* ws, int C) {
   w.ticket2 = w.tickets + C;
   w.cnt = w.ticket2 + 1;
   w.gmax_bits = w.cnt + C;
+  w.gridbar = w.gmax_bits + 1;
   size_t off = (control_words(C) * 4 + 15) / 16 * 16;
   w.absmax = reinterpret_cast<float*>(p + off);
   w.mean = w.absmax + C;
@@ -532,8 +536,429 @@ absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_
 }
 
 // ------------------------------------------------------------------------------------------------
+// Fused NHWC path: the three sweeps in ONE persistent cooperative kernel (one CTA of 512 threads
+// per SM).  Every thread owns the same elements in all three phases (one 16-byte vector of channels
+// of every rpi-th pixel of the CTA's pixel range), so the part of the tensor that fits is parked in
+// shared memory during the first sweep and the later sweeps never touch HBM for it; the rest is
+// re-read (L2 hits for tensors of up to ~100 MB).  Between the phases the CTAs meet at a bounded
+// grid barrier and every CTA finishes the per-channel scalars for itself, in one fixed order, so
+// all of them hold identical sigma, class and clip values.
+// ------------------------------------------------------------------------------------------------
+constexpr int kFT = 512;             // threads per CTA of the fused kernel (one CTA per SM)
+constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
+constexpr long long kBarrierTimeoutCycles = 2000000000LL;
+
+template <typename T, int VE> struct RawVec { using type = uint4; };
+template <typename T> struct RawVec<T, 1> { using type = T; };
+
+template <typename T, int VE>
+__device__ __forceinline__ typename RawVec<T, VE>::type load_raw(const T* p) {
+  if constexpr (VE == 1) return *p;
+  else return *reinterpret_cast<const uint4*>(p);
+}
+__device__ __forceinline__ void unpack_raw(const uint4& r, float (&v)[4], const float*) {
+  v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+}
+__device__ __forceinline__ void unpack_raw(const uint4& r, float (&v)[8], const bf16_t*) {
+  const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
+}
+__device__ __forceinline__ void unpack_raw(const float& r, float (&v)[1], const float*) { v[0] = r; }
+__device__ __forceinline__ void unpack_raw(const bf16_t& r, float (&v)[1], const bf16_t*) { v[0] = to_f32(r); }
+
+struct FusedArgs {
+  int64_t npix, HW;
+  int C, Cp, G, Gp;        // G input vector columns, Gp output vector columns (>= G, zero padding)
+  int slots;               // vectors per thread kept in shared memory
+  GvqWs ws;
+  uint32_t* gridbar;
+  const float* sigma_override;
+  McsDev mp;
+  float* s_state;
+  int has_prev;
+  float* gmax_layer;
+  float* stats_out;
+  uint8_t* cls;
+  uint32_t seed;
+  int8_t* q1;
+  int8_t* q2;
+  unsigned int* status;
+};
+
+// All CTAs of a cooperative launch meet here.  Bounded: returns false (in every thread of the CTA)
+// if the others do not arrive in time, after recording DAI8_ERR_TIMEOUT.
+__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target, unsigned int* status) {
+  __shared__ uint32_t s_ok;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    atomicAdd(counter, 1u);
+    uint32_t ok = 1u;
+    const long long t0 = clock64();
+    while (*reinterpret_cast<volatile uint32_t*>(counter) < target) {
+      if (clock64() - t0 > kBarrierTimeoutCycles) {
+        atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
+        ok = 0u;
+        break;
+      }
+      __nanosleep(64);
+    }
+    __threadfence();
+    s_ok = ok;
+  }
+  __syncthreads();
+  return s_ok != 0u;
+}
+
+// Sum (or max) over the row lanes of a CTA for every vector column: thread (rl, col) contributes
+// v, the result for column j lands in thread j (tid < Gp).  Fixed order -> deterministic.
+// Gp <= 32: lanes of a warp hold rows_per_warp rows; first a shuffle chain inside the warp.
+template <typename V, bool IS_MAX>
+__device__ __forceinline__ V column_reduce(V v, V* sred, int Gp, int rows_per_warp, int nrows_flat) {
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int nrows;
+  if (Gp <= 32) {
+    V acc = v;
+    for (int k = 1; k < rows_per_warp; ++k) {
+      const V o = __shfl_sync(0xFFFFFFFFu, v, (lane + k * Gp) & 31);
+      acc = IS_MAX ? (o > acc ? o : acc) : acc + o;
+    }
+    if (lane < Gp) sred[warp * Gp + lane] = acc;
+    nrows = kFT / 32;
+  } else {
+    if (tid < nrows_flat * Gp) sred[tid] = v;
+    nrows = nrows_flat;
+  }
+  __syncthreads();
+  V res = V(0);
+  if (tid < Gp) {
+    for (int r = 0; r < nrows; ++r) {
+      const V o = sred[r * Gp + tid];
+      res = IS_MAX ? (o > res ? o : res) : res + o;
+    }
+  }
+  __syncthreads();
+  return res;
+}
+
+template <typename T, int VE, bool DUAL>
+__global__ void __launch_bounds__(kFT, 1)
+gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
+  using Raw = typename RawVec<T, VE>::type;
+  extern __shared__ __align__(16) uint8_t fsmem[];
+  double* sred_d = reinterpret_cast<double*>(fsmem);                 // [kFT]
+  float* sred_f = reinterpret_cast<float*>(fsmem + kFT * 8);         // [kFT]
+  uint32_t* sred_u = reinterpret_cast<uint32_t*>(sred_f);
+  float* ch_absmax = reinterpret_cast<float*>(fsmem + kFT * 12);     // [C]
+  float* ch_sigma = ch_absmax + a.C;                                 // [C]
+  float* ch_sprev = ch_sigma + a.C;                                  // [C]
+  float* ch_inv = ch_sprev + a.C;                                    // [C]
+  Raw* slab = reinterpret_cast<Raw*>(fsmem + ((kFT * 12 + (size_t)a.C * 16 + 15) / 16) * 16);
+  __shared__ float s_gmax;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int C = a.C, Gp = a.Gp, G = a.G;
+  int rows_per_warp = 0, rpi, col, rl;
+  bool active;
+  if (Gp <= 32) {
+    rows_per_warp = 32 / Gp;
+    rpi = (kFT / 32) * rows_per_warp;
+    col = lane % Gp;
+    rl = warp * rows_per_warp + lane / Gp;
+    active = lane < rows_per_warp * Gp;
+  } else {
+    rpi = kFT / Gp;
+    col = tid % Gp;
+    rl = tid / Gp;
+    active = rl < rpi;
+  }
+  const bool real = active && col < G;     // has input; columns >= G are code padding
+  const int c0 = col * VE;
+  const int64_t chunk = (a.npix + gridDim.x - 1) / gridDim.x;
+  const int64_t p0 = (int64_t)blockIdx.x * chunk;
+  const int64_t p1 = min(a.npix, p0 + chunk);
+  const int64_t first = p0 + rl;
+  const int n_it = (active && first < p1) ? (int)((p1 - first + rpi - 1) / rpi) : 0;
+  const T* base = x + c0;
+
+  // ---------------- phase 1: statistics, parking the slab in shared memory ----------------------
+  float amax[VE], fs[VE], fss[VE];
+  double ds[VE], dss[VE];
+#pragma unroll
+  for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; ds[e] = 0.0; dss[e] = 0.0; }
+  if (real) {
+    float piv[VE];
+    load_vec<T, VE>(base, piv);
+    for (int i0 = 0; i0 < n_it; i0 += 8) {
+      Raw raw[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (i0 + u < n_it) raw[u] = load_raw<T, VE>(base + (first + (int64_t)(i0 + u) * rpi) * C);
+#pragma unroll
+      for (int u = 0; u < 8; ++u) {
+        if (i0 + u < n_it) {
+          if (i0 + u < a.slots) slab[(size_t)(i0 + u) * kFT + tid] = raw[u];
+          float v[VE];
+          unpack_raw(raw[u], v, (const T*)nullptr);
+#pragma unroll
+          for (int e = 0; e < VE; ++e) {
+            amax[e] = fmaxf(amax[e], fabsf(v[e]));
+            const float d = v[e] - piv[e];
+            fs[e] += d;
+            fss[e] = fmaf(d, d, fss[e]);
+          }
+        }
+      }
+      if (((i0 >> 3) & 3) == 3) {  // every 32 elements: short fp32 runs, combined in binary64
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; }
+  }
+  {
+    const size_t prow = (size_t)blockIdx.x * C;
+#pragma unroll
+    for (int e = 0; e < VE; ++e) {
+      const float m = column_reduce<float, true>(amax[e], sred_f, Gp, rows_per_warp, rpi);
+      const double s1 = column_reduce<double, false>(ds[e], sred_d, Gp, rows_per_warp, rpi);
+      const double s2 = column_reduce<double, false>(dss[e], sred_d, Gp, rows_per_warp, rpi);
+      if (tid < G) {
+        a.ws.pmax[prow + tid * VE + e] = m;
+        a.ws.psum[prow + tid * VE + e] = s1;
+        a.ws.pss[prow + tid * VE + e] = s2;
+      }
+    }
+  }
+  // previous clip values are read before the barrier after which CTA 0 overwrites them
+  for (int c = tid; c < C; c += kFT) ch_sprev[c] = a.has_prev ? a.s_state[c] : 0.f;
+  bool ok = grid_barrier(a.gridbar, gridDim.x, a.status);
+
+  // every CTA combines the per-CTA partials of every channel, in the same fixed order
+  if (ok) {
+    const int nblk = gridDim.x;
+    const int parts = C >= kFT ? 1 : kFT / C;
+    float gm = 0.f;
+    for (int cb = 0; cb < C; cb += kFT) {
+      const int c = parts == 1 ? cb + tid : tid % C;
+      const int part = parts == 1 ? 0 : tid / C;
+      float m = 0.f;
+      double s1 = 0.0, s2 = 0.0;
+      if (c < C && part < parts) {
+        for (int b = part; b < nblk; b += parts) {
+          const size_t idx = (size_t)b * C + c;
+          m = fmaxf(m, __ldcg(a.ws.pmax + idx));
+          s1 += __ldcg(a.ws.psum + idx);
+          s2 += __ldcg(a.ws.pss + idx);
+        }
+      }
+      // combine the parts: three rounds through the scratch buffers
+      float mm = m; double t1 = s1, t2 = s2;
+      if (parts > 1) {
+        __syncthreads();
+        sred_f[tid] = m; sred_d[tid] = s1;
+        __syncthreads();
+        if (part == 0 && c < C) for (int r = 1; r < parts; ++r) { mm = fmaxf(mm, sred_f[r * C + c]); t1 += sred_d[r * C + c]; }
+        __syncthreads();
+        sred_d[tid] = s2;
+        __syncthreads();
+        if (part == 0 && c < C) for (int r = 1; r < parts; ++r) t2 += sred_d[r * C + c];
+        __syncthreads();
+      }
+      if (part == 0 && c < C) {
+        float mean, sigma;
+        finish_moments((double)to_f32(x[c]), t1, t2, a.npix, a.mp, &mean, &sigma);
+        ch_absmax[c] = mm;
+        ch_sigma[c] = a.sigma_override ? a.sigma_override[c] : sigma;
+        gm = fmaxf(gm, mm);
+        if (blockIdx.x == 0) {
+          a.ws.absmax[c] = mm; a.ws.mean[c] = mean; a.ws.sigma[c] = sigma;
+          if (a.stats_out) {
+            a.stats_out[c * 4 + DAI8_STAT_ABSMAX] = mm;
+            a.stats_out[c * 4 + DAI8_STAT_MEAN] = mean;
+            a.stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
+          }
+        }
+      }
+    }
+    __syncthreads();
+    sred_f[tid] = gm;
+    __syncthreads();
+    for (int o = kFT / 2; o > 0; o >>= 1) {
+      if (tid < o) sred_f[tid] = fmaxf(sred_f[tid], sred_f[tid + o]);
+      __syncthreads();
+    }
+    if (tid == 0) s_gmax = sred_f[0];
+    __syncthreads();
+  }
+
+  // ---------------- phase 2: density count -----------------------------------------------------
+  if (ok) {
+    uint32_t k[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) k[e] = 0u;
+    if (real) {
+      float sg[VE];
+#pragma unroll
+      for (int e = 0; e < VE; ++e) sg[e] = ch_sigma[c0 + e];
+      for (int i0 = 0; i0 < n_it; i0 += 4) {
+        Raw raw[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int i = i0 + u;
+          if (i < n_it)
+            raw[u] = i < a.slots ? slab[(size_t)i * kFT + tid] : load_raw<T, VE>(base + (first + (int64_t)i * rpi) * C);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (i0 + u < n_it) {
+            float v[VE];
+            unpack_raw(raw[u], v, (const T*)nullptr);
+#pragma unroll
+            for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < VE; ++e) {
+      const uint32_t tot = column_reduce<uint32_t, false>(k[e], sred_u, Gp, rows_per_warp, rpi);
+      if (tid < G && tot) atomicAdd(a.ws.cnt + tid * VE + e, tot);
+    }
+    ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status);
+  }
+
+  // ---------------- classify + clip (Alg. 1 lines 5-9), identically in every CTA -----------------
+  if (ok) {
+    const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
+    for (int c = tid; c < C; c += kFT) {
+      const uint32_t cnt = __ldcg(a.ws.cnt + c);
+      const float gmax = ch_absmax[c];
+      const bool bell = (double)cnt > (double)a.mp.lambda * (double)a.npix;
+      float s;
+      if (bell) {
+        s = gmax;
+      } else {
+        const float s_prev = a.has_prev ? ch_sprev[c] : gmax;
+        s = __fadd_rn(__fmul_rn(tcoef, s_prev), __fmul_rn(a.mp.A, gmax));
+      }
+      ch_inv[c] = inv_scale(s);
+      if (blockIdx.x == 0) {
+        a.s_state[c] = s;
+        if (a.cls) a.cls[c] = bell ? 1 : 0;
+        if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt / (double)a.npix);
+      }
+    }
+    if (blockIdx.x == 0 && tid == 0) *a.gmax_layer = s_gmax;
+    __syncthreads();
+
+    // ---------------- phase 3: both sets of codes -------------------------------------------------
+    if (active && n_it > 0) {
+      float inv1[VE];
+#pragma unroll
+      for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
+      const float inv2 = inv_scale(s_gmax);
+      const uint32_t key0 = sr_key(a.seed, 0u);
+      int64_t n = first / a.HW;
+      int64_t hw = first - n * a.HW;
+      for (int i0 = 0; i0 < n_it; i0 += 4) {
+        Raw pre[4];
+        if (real) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const int j = i0 + u;
+            if (j < n_it)
+              pre[u] = j < a.slots ? slab[(size_t)j * kFT + tid] : load_raw<T, VE>(base + (first + (int64_t)j * rpi) * C);
+          }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          if (i0 + u >= n_it) break;
+          const int64_t p = first + (int64_t)(i0 + u) * rpi;
+          int qa[VE], qb[VE];
+          if (real) {
+            float v[VE];
+            unpack_raw(pre[u], v, (const T*)nullptr);
+            const uint64_t idx0 = ((uint64_t)n * C + c0) * a.HW + hw;
+#pragma unroll
+            for (int e = 0; e < VE; ++e) {
+              const uint64_t idx = idx0 + (uint64_t)e * a.HW;
+              const uint32_t hi = (uint32_t)(idx >> 32);
+              const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
+              const uint32_t h = avalanche32((uint32_t)idx ^ key);
+              qa[e] = quant_stochastic(v[e], inv1[e], sr_uniform(h));
+              qb[e] = DUAL ? quant_stochastic(v[e], inv2, sr_uniform(h * 0x9E3779B1u)) : 0;
+            }
+          } else {
+#pragma unroll
+            for (int e = 0; e < VE; ++e) { qa[e] = 0; qb[e] = 0; }
+          }
+          store_codes<VE>(a.q1 + p * a.Cp + c0, qa);
+          if (DUAL) store_codes<VE>(a.q2 + p * a.Cp + c0, qb);
+          hw += rpi;
+          while (hw >= a.HW) { hw -= a.HW; ++n; }
+        }
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Host-side launch helpers
 // ------------------------------------------------------------------------------------------------
+struct FusedConfig {
+  int sms = 0;
+  size_t smem_max = 0;
+  bool coop = false;
+};
+
+const FusedConfig& fused_config() {
+  static FusedConfig cfg;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    int dev = 0, coop = 0, sms = 0, smem = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return;
+    cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    cfg.sms = sms;
+    cfg.smem_max = (size_t)smem;
+    cfg.coop = coop != 0 && sms > 0;
+  });
+  return cfg;
+}
+
+template <typename T, int VE, bool DUAL>
+dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
+  const FusedConfig& cfg = fused_config();
+  const size_t fixed = ((size_t)kFT * 12 + (size_t)a.C * 16 + 15) / 16 * 16;
+  const size_t budget = cfg.smem_max - 1024;   // static shared memory of the kernel
+  const size_t slot_bytes = sizeof(typename RawVec<T, VE>::type) * kFT;
+  // pixel rows handled per CTA iteration
+  const int rpi = a.Gp <= 32 ? (kFT / 32) * (32 / a.Gp) : kFT / a.Gp;
+  int64_t ctas = ceil_div64(a.npix, rpi);
+  if (ctas > cfg.sms) ctas = cfg.sms;
+  const int64_t chunk = ceil_div64(a.npix, ctas);
+  const int64_t its = ceil_div64(chunk, rpi);
+  int64_t slots = (int64_t)((budget - fixed) / slot_bytes);
+  if (slots > its) slots = its;
+  a.slots = (int)slots;
+  const size_t smem = fixed + (size_t)slots * slot_bytes;
+  auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] {
+    attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(cfg.smem_max - 1024));
+  });
+  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  void* args[] = {(void*)&dY, (void*)&a};
+  DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFT), args, smem, st));
+  note_launch(1);
+  return DAI8_OK;
+}
+
 struct NhwcGrid {
   dim3 grid;
   int G;   // vectors per pixel that are processed
@@ -577,6 +1002,20 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
   const float* sigma = sigma_override ? sigma_override : ws.sigma;
+  if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC) {
+    const bool vec = C % VEfull == 0;
+    const int ve = vec ? VEfull : 1;
+    if (Cp / ve <= kFT) {
+      FusedArgs a;
+      a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / ve; a.Gp = Cp / ve; a.slots = 0;
+      a.ws = ws; a.gridbar = ws.gridbar; a.sigma_override = sigma_override; a.mp = mp;
+      a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
+      a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
+      if (!a.status) return DAI8_ERR_CUDA;
+      if (vec) return gq ? launch_fused<T, VEfull, true>(dY, a, st) : launch_fused<T, VEfull, false>(dY, a, st);
+      return gq ? launch_fused<T, 1, true>(dY, a, st) : launch_fused<T, 1, false>(dY, a, st);
+    }
+  }
   if (layout == DAI8_NHWC) {
     if (C % VEfull == 0) {
       const NhwcGrid g = nhwc_grid(npix, C / VEfull);
