@@ -101,7 +101,7 @@ dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout la
                                  dai8_round round, uint32_t seed, int8_t* q, void* stream);
 
 /* ----------------------------------------------------------------------------------------------
- * dai8_quantize_grad -- Algorithm 1 lines 1-11: Gradient Vectorized Quantization with the
+ * dai8_quantize_grad -- Algorithm 1, the quantization half: Gradient Vectorized Quantization with the
  * Magnitude-aware Clipping Strategy.
  *   dY         gradient of the layer output, (N,C,H,W) elements of `dtype` in `layout`
  *              (C = Cout, H x W = output extent)
@@ -134,10 +134,10 @@ dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8_layout lay
  *                      acc = sum_{ci,r,s} qX[n,p*st+r-pad,q*st+s-pad,ci] qW[co,r,s,ci]   (Fig. 2)
  * dai8_conv_bwd_data   dX[n,ci,h,w]  = acc . ((gmax/127)(sW/127)),
  *                      acc = sum over (co,r,s,p,q) with h=p*st+r-pad, w=q*st+s-pad of
- *                      gq[n,p,q,co] qW[co,r,s,ci]                      (Eq. 3, Alg. 1 l. 12, 15)
+ *                      gq[n,p,q,co] qW[co,r,s,ci]                      (Eq. 3; Algorithm 1)
  * dai8_conv_bwd_filter dW[co,ci,r,s] = acc . ((sX/127)(s[co]/127)),
  *                      acc = sum_{n,p,q} vq[n,p,q,co] qX[n,p*st+r-pad,q*st+s-pad,ci]
- *                                                                      (Eq. 4-7, Alg. 1 l. 11, 14)
+ *                                                                      (Eq. 4-7; Algorithm 1)
  *   sX, sW, gmax   device, 1 float each;  s: device [Cout] (the s_state of dai8_quantize_grad)
  *   out_dtype      F32 or BF16 (de-quantized), or I32: the raw accumulators, scales ignored
  *   out_layout     NCHW or NHWC for Y / dX (C unpadded); dW is always (Cout,Cin,R,S)

@@ -56,7 +56,7 @@ def _f32(a) -> np.ndarray:
 
 
 def channel_stats(g, std_unbiased: bool = False, center_mean: bool = True):
-    """Algorithm 1 line 2.  Returns (absmax[C], mean[C], sigma[C], gmax_layer) as fp32."""
+    """Algorithm 1, statistics step.  Returns (absmax[C], mean[C], sigma[C], gmax_layer) as fp32."""
     g = _f32(g)
     N, C, H, W = g.shape
     absmax = np.empty(C, np.float32)
@@ -69,7 +69,7 @@ def channel_stats(g, std_unbiased: bool = False, center_mean: bool = True):
 
 
 def density_count(g, sigma) -> np.ndarray:
-    """Algorithm 1 line 4: #{|g| > sigma_c} per channel (uint32)."""
+    """Algorithm 1, density step: #{|g| > sigma_c} per channel (uint32)."""
     g = _f32(g)
     sigma = _f32(sigma)
     N, C, H, W = g.shape
@@ -81,7 +81,7 @@ def density_count(g, sigma) -> np.ndarray:
 
 def classify_clip(cnt, absmax, M: int, s_prev=None, lam: float = 0.3, k: float = 1.0,
                   A: float = 0.8):
-    """Algorithm 1 lines 5-9.  Returns (s_t[C] fp32, cls[C] uint8 with 1 = bell-shaped)."""
+    """Algorithm 1, discriminator and clip update.  Returns (s_t[C] fp32, cls[C] uint8 with 1 = bell-shaped)."""
     cnt = np.ascontiguousarray(cnt, dtype=np.uint32)
     absmax = _f32(absmax)
     C = cnt.shape[0]

@@ -36,7 +36,8 @@ int dai8o_num_threads() {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Algorithm 1, line 2: per-channel |g|max, mean and sigma; layer |g|max (Algorithm 1 line 10).
+// Algorithm 1, statistics step: per-channel |g|max, mean and sigma; layer |g|max (the scale of
+// the layer-wide codes).
 // Eq. 15 names mu "the mean of gradient": sigma is taken about the mean unless center_mean == 0
 // (then it is the root mean square, which Assumption 1 makes equivalent).  Population variance
 // (divide by M) unless std_unbiased != 0 (divide by M-1).
@@ -81,7 +82,7 @@ void dai8o_channel_stats(const float* g, int N, int C, int H, int W, int std_unb
 }
 
 // ---------------------------------------------------------------------------------------------
-// Algorithm 1, line 4: number of elements of channel c with |g| > sigma_c (strict, on |g| and not
+// Algorithm 1, density step: number of elements of channel c with |g| > sigma_c (strict, on |g| and not
 // on |g - mu|, compared in binary32).  cnt[C].
 // ---------------------------------------------------------------------------------------------
 void dai8o_density_count(const float* g, int N, int C, int H, int W, const float* sigma,
@@ -101,7 +102,7 @@ void dai8o_density_count(const float* g, int N, int C, int H, int W, const float
 }
 
 // ---------------------------------------------------------------------------------------------
-// Algorithm 1, lines 5-9 with Eq. 15 (discriminator) and Eq. 14 (clip update).
+// Algorithm 1, the if/else on P, with Eq. 15 (discriminator) and Eq. 14 (clip update).
 //   P = cnt / M ;  P > lambda  -> bell-shaped (cls = 1):  s_t = |g|max,c            (Eq. 11)
 //                  otherwise    -> Inverted-T  (cls = 0):  s_t = (1-kA) s_{t-1} + A |g|max,c
 // The test P > lambda is evaluated as cnt > lambda*M in binary64 (lambda is the binary32 value).
@@ -355,7 +356,7 @@ int64_t dai8o_conv_bwd_filter_acc(const int8_t* X, const int8_t* G, const int* g
 
 // ---------------------------------------------------------------------------------------------
 // De-quantization of an accumulator (Sec. 3.2, the vectorized de-quantization, and Algorithm 1
-// lines 14-15 with the scales the equations imply: s_X for G_W, s_W for G_X).
+// final two steps, with the scales the equations imply: s_X for G_W, s_W for G_X).
 //   out = (float)acc * ((sa / 127) * (sb / 127)), the scale product formed in binary32.
 // rows x cols accumulators; sb is per row (per_row != 0: sb[rows]) or a single value.
 // ---------------------------------------------------------------------------------------------

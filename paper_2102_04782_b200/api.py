@@ -165,7 +165,7 @@ def quantize_grad(dY: torch.Tensor, layout: int, N: int, C: int, H: int, W: int,
                   gmax_layer: torch.Tensor, stats: Optional[torch.Tensor],
                   cls: Optional[torch.Tensor], vq: torch.Tensor, gq: Optional[torch.Tensor],
                   seed: int, ws: torch.Tensor, sigma_override: Optional[torch.Tensor] = None) -> None:
-    """dai8_quantize_grad (Algorithm 1 lines 1-11)."""
+    """dai8_quantize_grad (Algorithm 1 up to and including the two quantizations of dY)."""
     _check(lib().dai8_quantize_grad(_ptr(dY), _dtype_code(dY), layout, N, C, H, W,
                                     ctypes.byref(params) if params is not None else None,
                                     _ptr(s_state), int(has_prev), _ptr(gmax_layer), _ptr(stats),

@@ -28,7 +28,7 @@ struct ConvOut {
   dai8_layout layout;  // NCHW or NHWC (C unpadded)
 };
 
-// De-quantization scale (Eq. 7 and Algorithm 1 lines 14-15): (a/127)*(b/127), each step rounded.
+// De-quantization scale (Eq. 7 and the last two steps of Algorithm 1): (a/127)*(b/127), each step rounded.
 __device__ __forceinline__ float dequant_scale(float a, float b) {
   return __fmul_rn(__fdiv_rn(a, 127.0f), __fdiv_rn(b, 127.0f));
 }

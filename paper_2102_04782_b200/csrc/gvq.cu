@@ -1,10 +1,10 @@
-// Gradient Vectorized Quantization with the Magnitude-aware Clipping Strategy (Algorithm 1,
-// lines 1-11) and the layer-wide quantizer of the forward pass (Eq. 1), as HBM-bound kernels.
+// Gradient Vectorized Quantization with the Magnitude-aware Clipping Strategy (Algorithm 1 up to
+// the two quantizations) and the layer-wide quantizer of the forward pass (Eq. 1), as HBM-bound kernels.
 //
 // Three sweeps over dY, because each needs a per-channel scalar the previous one produces:
-//   1. stats   : |g|max,c, sum, sum of squares  -> mean, sigma          (Alg. 1 line 2)
-//   2. count   : #{|g| > sigma_c}                -> class, clip s_c      (Alg. 1 lines 4-9, Eq. 14/15)
-//   3. quantize: vq (per-channel s_c) and gq (layer |g|max) in one pass (Alg. 1 lines 10-11)
+//   1. stats   : |g|max,c, sum, sum of squares  -> mean, sigma          (Algorithm 1)
+//   2. count   : #{|g| > sigma_c}                -> class, clip s_c      (Algorithm 1, Eq. 14/15)
+//   3. quantize: vq (per-channel s_c) and gq (layer |g|max) in one pass (Algorithm 1)
 // The last block of sweeps 1 and 2 (found with a ticket counter) finishes the per-channel
 // scalars, so no separate tiny launches are needed.  Floating-point sums are combined in a
 // fixed order (per-block partials, then a fixed tree), so results do not depend on scheduling;
@@ -284,7 +284,7 @@ stats_nchw_kernel(const T* __restrict__ x, int N, int C, int64_t HW, GvqWs ws, M
 }
 
 // ------------------------------------------------------------------------------------------------
-// Algorithm 1 lines 5-9 for every channel, by the last block of the count sweep.
+// Discriminator and clip update of Algorithm 1 for every channel, by the last block of the count sweep.
 //   P > lambda (cnt > lambda*M in binary64): s = |g|max,c                       (Eq. 11)
 //   otherwise: s = (1 - k*A)*s_prev + A*|g|max,c, each operation rounded to fp32  (Eq. 14)
 // ------------------------------------------------------------------------------------------------
@@ -382,7 +382,7 @@ count_nchw_kernel(const T* __restrict__ x, int N, int C, int64_t HW, GvqWs ws,
 // ------------------------------------------------------------------------------------------------
 // Sweep 3: Eq. 1 on every element.  Output 1 uses `scale1` (per channel if PER_CHANNEL, else one
 // value) and generator stream 0; the optional output 2 uses the single value `scale2` and
-// stream 1 (Algorithm 1 lines 10-11 fused, as Sec. 3.4 suggests).  STOCH selects the rounding.
+// stream 1 (the two quantizations of Algorithm 1 fused, as Sec. 3.4 suggests).  STOCH selects the rounding.
 // Codes are written as [pixel][Cp] with zero padding channels.
 // ------------------------------------------------------------------------------------------------
 template <int VE>
@@ -830,7 +830,7 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status);
   }
 
-  // ---------------- classify + clip (Alg. 1 lines 5-9), identically in every CTA -----------------
+  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------------
   if (ok) {
     const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
     for (int c = tid; c < C; c += kFT) {

@@ -34,7 +34,7 @@ def test_defaults_are_the_papers():
     assert sig.parameters["A"].default == c["A"]
 
 
-# ------------------------------------------------------------------ statistics (Alg. 1 line 2)
+# ------------------------------------------------------------------ statistics (Algorithm 1)
 @pytest.mark.parametrize("shape", [(2, 3, 5, 7), (8, 64, 14, 14), (1, 1, 1, 1), (3, 5, 1, 9)])
 def test_stats_match_numpy(shape):
     rng = np.random.default_rng(1)
@@ -71,7 +71,7 @@ def test_stats_channel_major_not_sample_major():
     assert sigma[1] == 0.0 and gl == 9.0
 
 
-# ------------------------------------------------------------------ density (Alg. 1 line 4)
+# ------------------------------------------------------------------ density (Algorithm 1)
 def test_density_bruteforce_and_strictness():
     g = np.array([0.0, 1.0, -1.0, 2.0, -3.0, 0.5], np.float32).reshape(1, 1, 1, 6)
     assert O.density_count(g, np.array([1.0], np.float32))[0] == 2       # strict '>' on |g|
