@@ -128,6 +128,35 @@ dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8_layout lay
                                void* stream);
 
 /* ----------------------------------------------------------------------------------------------
+ * dai8_quantize_grad_noalloc -- dai8_quantize_grad for callers that cannot provide scratch memory.
+ * (The paper has no counterpart: this is a property of the library's interface, not of the
+ * method.)  Same arguments and results as dai8_quantize_grad without `ws`, `ws_bytes` and
+ * `sigma_override`; the reduction scratch is a 3 MiB array built into the library image.
+ *
+ * Meant for code that cannot allocate on the device when it runs: an extension that a host
+ * framework hands nothing but its input and output tensors, a process whose device memory was
+ * divided up completely at start-up, a loop that cannot afford the device-wide stall of an
+ * allocation.  The caller still owns every input and output.
+ *
+ *   - C must not exceed DAI8_NOALLOC_MAX_CHANNELS; larger C returns DAI8_ERR_WORKSPACE (the
+ *     built-in scratch is too small) and nothing is enqueued.
+ *   - The array occupies 3 MiB on every GPU that has loaded the library, until the process exits.
+ *   - All calls on one device share the array.  Calls that may overlap on the GPU (different
+ *     streams without a dependency between them) race on it: order them.  No call depends on what
+ *     the previous one left there.
+ *   - The first call on each device looks up the array's device address (a host-side set-up
+ *     step): make that first call outside any stream capture.
+ *   - It calls no allocation routine of CUDA or of any other library.
+ * -------------------------------------------------------------------------------------------- */
+#define DAI8_NOALLOC_MAX_CHANNELS 256
+
+dai8_status dai8_quantize_grad_noalloc(const void* dY, dai8_dtype dtype, dai8_layout layout, int N,
+                                       int C, int H, int W, const dai8_mcs_params* params,
+                                       float* s_state, int has_prev, float* gmax_layer,
+                                       float* stats, uint8_t* cls, int8_t* vq, int8_t* gq,
+                                       uint32_t seed, void* stream);
+
+/* ----------------------------------------------------------------------------------------------
  * Convolutions on int8 codes with int32 accumulation and a de-quantizing epilogue.
  *
  * dai8_conv_fwd        Y[n,co,p,q]   = acc . ((sX/127)(sW/127)),

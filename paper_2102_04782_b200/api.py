@@ -22,7 +22,8 @@ OP_FWD, OP_BWD_DATA, OP_BWD_FILTER = 0, 1, 2
 
 EXPORTS = [
     "dai8_status_string", "dai8_mcs_defaults", "dai8_padded_channels", "dai8_quantize_tensor",
-    "dai8_quantize_grad_workspace_bytes", "dai8_quantize_grad", "dai8_conv_workspace_bytes",
+    "dai8_quantize_grad_workspace_bytes", "dai8_quantize_grad", "dai8_quantize_grad_noalloc",
+    "dai8_conv_workspace_bytes",
     "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
     "dai8_launch_count", "dai8_get_device_status",
 ]
@@ -79,6 +80,10 @@ def lib() -> ctypes.CDLL:
                                          ctypes.POINTER(McsParams), c_void_p, c_int, c_void_p,
                                          c_void_p, c_void_p, c_void_p, c_void_p, c_uint32, c_void_p,
                                          c_void_p, c_size_t, c_void_p]
+        l.dai8_quantize_grad_noalloc.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int,
+                                                 ctypes.POINTER(McsParams), c_void_p, c_int, c_void_p,
+                                                 c_void_p, c_void_p, c_void_p, c_void_p, c_uint32,
+                                                 c_void_p]
         conv_args = [c_void_p, c_void_p, c_void_p, c_void_p, ctypes.POINTER(ConvGeom), c_void_p, c_int,
                      c_int, c_void_p, c_size_t, c_void_p]
         l.dai8_conv_fwd.argtypes = conv_args
@@ -172,6 +177,26 @@ def quantize_grad(dY: torch.Tensor, layout: int, N: int, C: int, H: int, W: int,
                                     _ptr(cls), _ptr(vq), _ptr(gq), seed & 0xFFFFFFFF,
                                     _ptr(sigma_override), _ptr(ws), ws.numel() * ws.element_size(),
                                     _stream()), "dai8_quantize_grad")
+
+
+NOALLOC_MAX_CHANNELS = 256
+
+
+def quantize_grad_noalloc(dY: torch.Tensor, layout: int, N: int, C: int, H: int, W: int,
+                          params: Optional[McsParams], s_state: torch.Tensor, has_prev: bool,
+                          gmax_layer: torch.Tensor, stats: Optional[torch.Tensor],
+                          cls: Optional[torch.Tensor], vq: torch.Tensor,
+                          gq: Optional[torch.Tensor], seed: int) -> None:
+    """dai8_quantize_grad_noalloc: dai8_quantize_grad for a caller that has no scratch buffer to
+    give (it cannot allocate device memory where it runs).  The scratch is a fixed 3 MiB array
+    inside the library, shared by all calls on the device, so calls must not overlap on the GPU;
+    C is limited to NOALLOC_MAX_CHANNELS."""
+    _check(lib().dai8_quantize_grad_noalloc(_ptr(dY), _dtype_code(dY), layout, N, C, H, W,
+                                            ctypes.byref(params) if params is not None else None,
+                                            _ptr(s_state), int(has_prev), _ptr(gmax_layer),
+                                            _ptr(stats), _ptr(cls), _ptr(vq), _ptr(gq),
+                                            seed & 0xFFFFFFFF, _stream()),
+           "dai8_quantize_grad_noalloc")
 
 
 def conv_workspace_bytes(op: int, geom: ConvGeom) -> int:

@@ -1168,3 +1168,86 @@ extern "C" dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai
   return quantize_tensor_typed<bf16_t>(static_cast<const bf16_t*>(x), layout, N, C, H, W, scale_mode,
                                        scale, round, seed, q, st);
 }
+
+// ------------------------------------------------------------------------------------------------
+// dai8_quantize_grad_noalloc: the same kernels as dai8_quantize_grad, with the scratch memory taken
+// from an array that is part of the library image instead of from the caller.
+//
+// It exists for callers that have no way to obtain device memory at the moment they need the
+// gradient codes: an extension that is only ever handed the tensors it works on (inputs and
+// outputs) by a host framework and must not touch that framework's memory pool, a process whose
+// device memory has been handed out completely to other components at start-up, or a
+// latency-critical loop in which a cudaMalloc would stall every stream of the device.  Such a caller
+// still owns dY, the state and the code tensors; only the reduction scratch comes from here.
+//
+// The array costs kNoAllocScratchBytes on every GPU on which this library is loaded, for as long as
+// the process lives, whether or not this entry point is ever called -- hence the modest limit of
+// DAI8_NOALLOC_MAX_CHANNELS channels.  All calls on a device share the array: two calls that can
+// overlap on the GPU (different streams, no dependency) race on it.  Nothing in it carries over
+// from one call to the next; the control words that must start at zero are cleared on the stream
+// at the start of every call, the rest is written before it is read.
+//
+// In host code the array's name is only a handle.  The device address is looked up once per device
+// with cudaGetSymbolAddress, with that device current, on the first call made on that device; do
+// that first call outside any stream capture.
+// ------------------------------------------------------------------------------------------------
+namespace dai8 {
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = (size_t)3 << 20;  // 3 MiB
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
+void* g_noalloc_ptr[kMaxDevices] = {};
+
+// Device address of g_noalloc_scratch on the current device (nullptr and a status on failure).
+dai8_status noalloc_scratch_address(void** out) {
+  int dev = -1;
+  DAI8_RETURN_IF_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return DAI8_ERR_UNSUPPORTED;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  if (!g_noalloc_ptr[dev]) {
+    void* p = nullptr;
+    DAI8_RETURN_IF_CUDA(cudaGetSymbolAddress((void**)&p, g_noalloc_scratch));
+    if (!p || !aligned16(p)) return DAI8_ERR_CUDA;
+    g_noalloc_ptr[dev] = p;
+  }
+  *out = g_noalloc_ptr[dev];
+  return DAI8_OK;
+}
+
+}  // namespace
+}  // namespace dai8
+
+extern "C" dai8_status dai8_quantize_grad_noalloc(const void* dY, dai8_dtype dtype, dai8_layout layout,
+                                                  int N, int C, int H, int W,
+                                                  const dai8_mcs_params* params, float* s_state,
+                                                  int has_prev, float* gmax_layer, float* stats,
+                                                  uint8_t* cls, int8_t* vq, int8_t* gq, uint32_t seed,
+                                                  void* stream) {
+  if (!dY || !s_state || !gmax_layer || !vq) return DAI8_ERR_INVALID_ARG;
+  if (bad_dims(N, C, H, W)) return DAI8_ERR_INVALID_ARG;
+  if (dtype != DAI8_F32 && dtype != DAI8_BF16) return DAI8_ERR_INVALID_ARG;
+  if (layout != DAI8_NCHW && layout != DAI8_NHWC) return DAI8_ERR_INVALID_ARG;
+  if (!aligned16(dY) || !aligned16(vq) || (gq && !aligned16(gq))) return DAI8_ERR_INVALID_ARG;
+  if ((int64_t)N * H * W >= (int64_t)1 << 32) return DAI8_ERR_UNSUPPORTED;
+  // the built-in scratch is sized for DAI8_NOALLOC_MAX_CHANNELS channels
+  if (C > DAI8_NOALLOC_MAX_CHANNELS || ws_bytes_for(C) > kNoAllocScratchBytes) return DAI8_ERR_WORKSPACE;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  void* scratch = nullptr;
+  a = noalloc_scratch_address(&scratch);
+  if (a != DAI8_OK) return a;
+  dai8_mcs_params p;
+  if (params) p = *params; else dai8_mcs_defaults(&p);
+  McsDev mp{p.lambda, p.k, p.A, p.std_unbiased, p.center_mean};
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  GvqWs w = carve(scratch, C);
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(w.tickets, 0, control_words(C) * 4, st));
+  if (dtype == DAI8_F32)
+    return quantize_grad_typed<float>(static_cast<const float*>(dY), layout, N, C, H, W, mp, s_state,
+                                      has_prev, gmax_layer, stats, cls, vq, gq, seed, nullptr, w, st);
+  return quantize_grad_typed<bf16_t>(static_cast<const bf16_t*>(dY), layout, N, C, H, W, mp, s_state,
+                                     has_prev, gmax_layer, stats, cls, vq, gq, seed, nullptr, w, st);
+}
