@@ -101,6 +101,42 @@ __device__ __forceinline__ int quant_stochastic(float x, float inv, float u) {
   const int q = __float2int_rd(__fadd_rn(v, u));
   return min(q, 127);
 }
+
+// The same two quantizers without a float-to-int conversion: adding 1.5*2^23 to a value in
+// [-127, 127] leaves its rounded integer in the low mantissa bits (two's complement), so the LOW
+// BYTE of the returned bit pattern is the int8 code.  Round-to-nearest-even of the sum is Eq. 1's
+// nearest rounding; round-down of the sum is the floor of stochastic rounding.  For the stochastic
+// form the upper clamp moves behind the addition of u: floor(min(v + u, 127)) equals
+// min(floor(min(v, 127) + u), 127) for every v and every u in [0, 1).
+constexpr float kRoundMagic = 12582912.0f;  // 1.5 * 2^23
+__device__ __forceinline__ uint32_t quant_nearest_bits(float x, float inv) {
+  float v = __fmul_rn(x, inv);
+  v = fminf(fmaxf(v, -127.0f), 127.0f);
+  return __float_as_uint(__fadd_rn(v, kRoundMagic));
+}
+__device__ __forceinline__ uint32_t quant_stochastic_bits(float x, float inv, float u) {
+  const float v = fmaxf(__fmul_rn(x, inv), -127.0f);
+  const float t = fminf(__fadd_rn(v, u), 127.0f);
+  return __float_as_uint(__fadd_rd(t, kRoundMagic));
+}
+// Low bytes of four such bit patterns -> one word of four consecutive int8 codes.
+__device__ __forceinline__ uint32_t pack_codes4(uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  return __byte_perm(__byte_perm(a, b, 0x0040), __byte_perm(c, d, 0x0040), 0x5410);
+}
+// u in [0,1) from a hash: one funnel shift builds the bits of 1.0 + (h >> 9) * 2^-23.
+__device__ __forceinline__ float sr_uniform_fast(uint32_t h) {
+  return __uint_as_float(__funnelshift_r(h, 0x7Fu, 9)) - 1.0f;
+}
+// avalanche32(idx ^ key) with the first xor-shift folded: (a ^ a>>16) for a = idx ^ key equals
+// idx ^ (idx >> 16) ^ keyx with keyx = key ^ (key >> 16).
+__device__ __forceinline__ uint32_t sr_hash_folded(uint32_t idx, uint32_t keyx) {
+  uint32_t h = idx ^ (idx >> 16) ^ keyx;
+  h *= 0x85EBCA6Bu;
+  h ^= h >> 13;
+  h *= 0xC2B2AE35u;
+  h ^= h >> 16;
+  return h;
+}
 __device__ __forceinline__ float inv_scale(float s) { return s > 0.0f ? __fdiv_rn(127.0f, s) : 0.0f; }
 
 }  // namespace dai8

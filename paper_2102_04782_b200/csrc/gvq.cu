@@ -15,6 +15,7 @@
 // registers and every load/store instruction of a warp covers contiguous memory.  NCHW inputs are
 // read along H*W per (n, c) row and transposed through shared memory when codes are written.
 #include <mutex>
+#include <type_traits>
 
 #include "dai8_common.cuh"
 
@@ -543,10 +544,18 @@ absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_
 // re-read (L2 hits for tensors of up to ~100 MB).  Between the phases the CTAs meet at a bounded
 // grid barrier and every CTA finishes the per-channel scalars for itself, in one fixed order, so
 // all of them hold identical sigma, class and clip values.
+//
+// The kernel is bound by instruction issue rather than by HBM (two stochastic roundings per
+// element, each with its own hash-derived uniform), so the per-element instruction count is what
+// is optimised: bf16 inputs take |g|max and the density count two elements at a time in packed
+// bf16 arithmetic (both are exact there), codes come out of a magic-number addition instead of a
+// float-to-int conversion, and tensors of fewer than 2^32 elements use 32-bit index arithmetic.
 // ------------------------------------------------------------------------------------------------
 constexpr int kFT = 512;             // threads per CTA of the fused kernel (one CTA per SM)
 constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
 constexpr long long kBarrierTimeoutCycles = 2000000000LL;
+// reduction scratch at the start of the dynamic shared memory: VE arrays of kFT doubles (at least 3)
+__host__ __device__ constexpr size_t fused_red_bytes(int ve) { return (size_t)(ve < 3 ? 3 : ve) * kFT * 8; }
 
 template <typename T, int VE> struct RawVec { using type = uint4; };
 template <typename T> struct RawVec<T, 1> { using type = T; };
@@ -566,6 +575,24 @@ __device__ __forceinline__ void unpack_raw(const uint4& r, float (&v)[8], const 
 }
 __device__ __forceinline__ void unpack_raw(const float& r, float (&v)[1], const float*) { v[0] = r; }
 __device__ __forceinline__ void unpack_raw(const bf16_t& r, float (&v)[1], const bf16_t*) { v[0] = to_f32(r); }
+
+// Packed bf16 helpers (two values per 32-bit word).  max and compare are exact in bf16.
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// 1.0 (0x3F80) in every half where a > b, else 0.
+__device__ __forceinline__ uint32_t bf16x2_gt_one(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("set.gt.bf16x2.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+__device__ __forceinline__ uint32_t bf16x2_add(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
 
 struct FusedArgs {
   int64_t npix, HW;
@@ -602,7 +629,6 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target,
         ok = 0u;
         break;
       }
-      __nanosleep(64);
     }
     __threadfence();
     s_ok = ok;
@@ -611,126 +637,167 @@ __device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target,
   return s_ok != 0u;
 }
 
-// Sum (or max) over the row lanes of a CTA for every vector column: thread (rl, col) contributes
-// v, the result for column j lands in thread j (tid < Gp).  Fixed order -> deterministic.
-// Gp <= 32: lanes of a warp hold rows_per_warp rows; first a shuffle chain inside the warp.
-template <typename V, bool IS_MAX>
-__device__ __forceinline__ V column_reduce(V v, V* sred, int Gp, int rows_per_warp, int nrows_flat) {
+// How the 512 threads of a CTA tile (pixel row, vector column) pairs.
+struct FusedMap {
+  int rows_per_warp;  // > 0 when a warp holds whole rows (Gp <= 32)
+  int rpi;            // pixel rows per CTA iteration
+  int col, rl;        // this thread's vector column and row lane
+  int nrows_smem;     // rows that reach shared memory in a column reduction
+  int row_smem;       // this thread's row there
+  bool active;
+};
+
+__device__ __forceinline__ FusedMap fused_map(int Gp) {
+  FusedMap m;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  int nrows;
   if (Gp <= 32) {
-    V acc = v;
-    for (int k = 1; k < rows_per_warp; ++k) {
-      const V o = __shfl_sync(0xFFFFFFFFu, v, (lane + k * Gp) & 31);
-      acc = IS_MAX ? (o > acc ? o : acc) : acc + o;
-    }
-    if (lane < Gp) sred[warp * Gp + lane] = acc;
-    nrows = kFT / 32;
+    m.rows_per_warp = 32 / Gp;
+    m.rpi = (kFT / 32) * m.rows_per_warp;
+    m.col = lane % Gp;
+    m.rl = warp * m.rows_per_warp + lane / Gp;
+    m.active = lane < m.rows_per_warp * Gp;
+    m.nrows_smem = kFT / 32;
+    m.row_smem = warp;
   } else {
-    if (tid < nrows_flat * Gp) sred[tid] = v;
-    nrows = nrows_flat;
+    m.rows_per_warp = 0;
+    m.rpi = kFT / Gp;
+    m.col = tid % Gp;
+    m.rl = tid / Gp;
+    m.active = m.rl < m.rpi;
+    m.nrows_smem = m.rpi;
+    m.row_smem = m.rl;
   }
-  __syncthreads();
-  V res = V(0);
-  if (tid < Gp) {
-    for (int r = 0; r < nrows; ++r) {
-      const V o = sred[r * Gp + tid];
-      res = IS_MAX ? (o > res ? o : res) : res + o;
-    }
-  }
-  __syncthreads();
-  return res;
+  return m;
 }
 
-template <typename T, int VE, bool DUAL>
+struct OpAdd { template <typename V> __device__ __forceinline__ V operator()(V a, V b) const { return a + b; } };
+struct OpMax { template <typename V> __device__ __forceinline__ V operator()(V a, V b) const { return a > b ? a : b; } };
+
+// Combines val[e] over the row lanes of the CTA for every (column, e), in a fixed order.  The result
+// for channel col*VE + e is handed to out(channel, value) by thread e*Gp + col.  `red` holds
+// VE * kFT values.  Two __syncthreads; `red` may be reused after the call returns.
+template <int VE, typename V, typename Op, typename Out>
+__device__ __forceinline__ void column_reduce(const FusedMap& m, int Gp, V (&val)[VE], V* red, Op op, Out out) {
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (m.rows_per_warp > 1) {
+#pragma unroll
+    for (int e = 0; e < VE; ++e) {
+      V acc = val[e];
+      for (int k = 1; k < m.rows_per_warp; ++k) acc = op(acc, __shfl_sync(0xFFFFFFFFu, val[e], (lane + k * Gp) & 31));
+      val[e] = acc;
+    }
+  }
+  const bool writer = m.rows_per_warp > 0 ? lane < Gp : m.active;
+  if (writer) {
+#pragma unroll
+    for (int e = 0; e < VE; ++e) red[e * kFT + m.row_smem * Gp + m.col] = val[e];
+  }
+  __syncthreads();
+  for (int t = tid; t < VE * Gp; t += kFT) {
+    const int e = t / Gp, col = t - e * Gp;
+    V acc = red[e * kFT + col];
+    for (int r = 1; r < m.nrows_smem; ++r) acc = op(acc, red[e * kFT + r * Gp + col]);
+    out(col * VE + e, acc);
+  }
+  __syncthreads();
+}
+
+// Runs f(i, raw) for i in [begin, end), loading U vectors ahead of the work on them.
+template <int U, typename Raw, typename Load, typename F>
+__device__ __forceinline__ void for_each_batched(int begin, int end, Load load, F f) {
+  int i = begin;
+  for (; i + U <= end; i += U) {
+    Raw r[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) r[u] = load(i + u);
+#pragma unroll
+    for (int u = 0; u < U; ++u) f(i + u, r[u]);
+  }
+  for (; i < end; ++i) f(i, load(i));
+}
+
+template <typename T, int VE, bool DUAL, bool IDX32>
 __global__ void __launch_bounds__(kFT, 1)
 gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   using Raw = typename RawVec<T, VE>::type;
+  constexpr bool kPacked = VE == 8;  // bf16 vectors: packed max / compare
   extern __shared__ __align__(16) uint8_t fsmem[];
-  double* sred_d = reinterpret_cast<double*>(fsmem);                 // [kFT]
-  float* sred_f = reinterpret_cast<float*>(fsmem + kFT * 8);         // [kFT]
-  uint32_t* sred_u = reinterpret_cast<uint32_t*>(sred_f);
-  float* ch_absmax = reinterpret_cast<float*>(fsmem + kFT * 12);     // [C]
-  float* ch_sigma = ch_absmax + a.C;                                 // [C]
-  float* ch_sprev = ch_sigma + a.C;                                  // [C]
-  float* ch_inv = ch_sprev + a.C;                                    // [C]
-  Raw* slab = reinterpret_cast<Raw*>(fsmem + ((kFT * 12 + (size_t)a.C * 16 + 15) / 16) * 16);
+  double* red_d = reinterpret_cast<double*>(fsmem);                      // [VE][kFT]
+  float* red_f = reinterpret_cast<float*>(fsmem);
+  uint32_t* red_u = reinterpret_cast<uint32_t*>(fsmem);
+  float* ch_absmax = reinterpret_cast<float*>(fsmem + fused_red_bytes(VE));      // [C]
+  float* ch_sigma = ch_absmax + a.C;                                     // [C]
+  float* ch_sprev = ch_sigma + a.C;                                      // [C]
+  float* ch_inv = ch_sprev + a.C;                                        // [C]
+  Raw* slab = reinterpret_cast<Raw*>(fsmem + ((fused_red_bytes(VE) + (size_t)a.C * 16 + 15) / 16) * 16);
   __shared__ float s_gmax;
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int tid = threadIdx.x;
   const int C = a.C, Gp = a.Gp, G = a.G;
-  int rows_per_warp = 0, rpi, col, rl;
-  bool active;
-  if (Gp <= 32) {
-    rows_per_warp = 32 / Gp;
-    rpi = (kFT / 32) * rows_per_warp;
-    col = lane % Gp;
-    rl = warp * rows_per_warp + lane / Gp;
-    active = lane < rows_per_warp * Gp;
-  } else {
-    rpi = kFT / Gp;
-    col = tid % Gp;
-    rl = tid / Gp;
-    active = rl < rpi;
-  }
-  const bool real = active && col < G;     // has input; columns >= G are code padding
+  const FusedMap m = fused_map(Gp);
+  const int rpi = m.rpi, col = m.col;
+  const bool real = m.active && col < G;     // has input; columns >= G are code padding
   const int c0 = col * VE;
   const int64_t chunk = (a.npix + gridDim.x - 1) / gridDim.x;
   const int64_t p0 = (int64_t)blockIdx.x * chunk;
   const int64_t p1 = min(a.npix, p0 + chunk);
-  const int64_t first = p0 + rl;
-  const int n_it = (active && first < p1) ? (int)((p1 - first + rpi - 1) / rpi) : 0;
-  const T* base = x + c0;
+  const int64_t first = p0 + m.rl;
+  const int n_it = (m.active && first < p1) ? (int)((p1 - first + rpi - 1) / rpi) : 0;
+  const int n_slab = min(n_it, a.slots);
+  const T* base = x + c0 + first * C;
+  const size_t it_stride = (size_t)rpi * C;
+  auto load_global = [&](int i) { return load_raw<T, VE>(base + (size_t)i * it_stride); };
+  auto load_slab = [&](int i) { return slab[(size_t)i * kFT + tid]; };
 
   // ---------------- phase 1: statistics, parking the slab in shared memory ----------------------
-  float amax[VE], fs[VE], fss[VE];
-  double ds[VE], dss[VE];
+  {
+    float amax[VE], fs[VE], fss[VE], piv[VE];
+    uint32_t amax2[VE / 2 + 1];
+    double ds[VE], dss[VE];
 #pragma unroll
-  for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; ds[e] = 0.0; dss[e] = 0.0; }
-  if (real) {
-    float piv[VE];
-    load_vec<T, VE>(base, piv);
-    for (int i0 = 0; i0 < n_it; i0 += 8) {
-      Raw raw[8];
+    for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; ds[e] = 0.0; dss[e] = 0.0; piv[e] = 0.f; }
 #pragma unroll
-      for (int u = 0; u < 8; ++u)
-        if (i0 + u < n_it) raw[u] = load_raw<T, VE>(base + (first + (int64_t)(i0 + u) * rpi) * C);
+    for (int j = 0; j < VE / 2 + 1; ++j) amax2[j] = 0u;
+    if (real) {
+      load_vec<T, VE>(x + c0, piv);  // pixel 0 of these channels
+      int run = 0;
+      auto body = [&](int i, const Raw& raw) {
+        if (i < n_slab) slab[(size_t)i * kFT + tid] = raw;
+        float v[VE];
+        unpack_raw(raw, v, (const T*)nullptr);
+        if constexpr (kPacked) {
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-      for (int u = 0; u < 8; ++u) {
-        if (i0 + u < n_it) {
-          if (i0 + u < a.slots) slab[(size_t)(i0 + u) * kFT + tid] = raw[u];
-          float v[VE];
-          unpack_raw(raw[u], v, (const T*)nullptr);
+          for (int j = 0; j < 4; ++j) amax2[j] = bf16x2_max(amax2[j], w[j] & 0x7FFF7FFFu);
+        }
 #pragma unroll
-          for (int e = 0; e < VE; ++e) {
-            amax[e] = fmaxf(amax[e], fabsf(v[e]));
-            const float d = v[e] - piv[e];
-            fs[e] += d;
-            fss[e] = fmaf(d, d, fss[e]);
-          }
+        for (int e = 0; e < VE; ++e) {
+          if constexpr (!kPacked) amax[e] = fmaxf(amax[e], fabsf(v[e]));
+          const float d = v[e] - piv[e];
+          fs[e] += d;
+          fss[e] = fmaf(d, d, fss[e]);
+        }
+        if (++run == 32) {  // short fp32 runs, combined in binary64
+          run = 0;
+#pragma unroll
+          for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
+        }
+      };
+      for_each_batched<4, Raw>(0, n_it, load_global, body);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; }
+      if constexpr (kPacked) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          amax[2 * j] = __uint_as_float(amax2[j] << 16);
+          amax[2 * j + 1] = __uint_as_float(amax2[j] & 0xFFFF0000u);
         }
       }
-      if (((i0 >> 3) & 3) == 3) {  // every 32 elements: short fp32 runs, combined in binary64
-#pragma unroll
-        for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
-      }
     }
-#pragma unroll
-    for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; }
-  }
-  {
     const size_t prow = (size_t)blockIdx.x * C;
-#pragma unroll
-    for (int e = 0; e < VE; ++e) {
-      const float m = column_reduce<float, true>(amax[e], sred_f, Gp, rows_per_warp, rpi);
-      const double s1 = column_reduce<double, false>(ds[e], sred_d, Gp, rows_per_warp, rpi);
-      const double s2 = column_reduce<double, false>(dss[e], sred_d, Gp, rows_per_warp, rpi);
-      if (tid < G) {
-        a.ws.pmax[prow + tid * VE + e] = m;
-        a.ws.psum[prow + tid * VE + e] = s1;
-        a.ws.pss[prow + tid * VE + e] = s2;
-      }
-    }
+    column_reduce<VE>(m, Gp, amax, red_f, OpMax(), [&](int c, float v) { if (c < C) a.ws.pmax[prow + c] = v; });
+    column_reduce<VE>(m, Gp, ds, red_d, OpAdd(), [&](int c, double v) { if (c < C) a.ws.psum[prow + c] = v; });
+    column_reduce<VE>(m, Gp, dss, red_d, OpAdd(), [&](int c, double v) { if (c < C) a.ws.pss[prow + c] = v; });
   }
   // previous clip values are read before the barrier after which CTA 0 overwrites them
   for (int c = tid; c < C; c += kFT) ch_sprev[c] = a.has_prev ? a.s_state[c] : 0.f;
@@ -744,27 +811,25 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     for (int cb = 0; cb < C; cb += kFT) {
       const int c = parts == 1 ? cb + tid : tid % C;
       const int part = parts == 1 ? 0 : tid / C;
-      float m = 0.f;
+      float mx = 0.f;
       double s1 = 0.0, s2 = 0.0;
       if (c < C && part < parts) {
         for (int b = part; b < nblk; b += parts) {
           const size_t idx = (size_t)b * C + c;
-          m = fmaxf(m, __ldcg(a.ws.pmax + idx));
+          mx = fmaxf(mx, __ldcg(a.ws.pmax + idx));
           s1 += __ldcg(a.ws.psum + idx);
           s2 += __ldcg(a.ws.pss + idx);
         }
       }
-      // combine the parts: three rounds through the scratch buffers
-      float mm = m; double t1 = s1, t2 = s2;
-      if (parts > 1) {
+      float mm = mx; double t1 = s1, t2 = s2;
+      if (parts > 1) {   // combine the parts through shared memory: [0,kFT) s1, [kFT,2kFT) s2, then max
         __syncthreads();
-        sred_f[tid] = m; sred_d[tid] = s1;
+        red_d[tid] = s1; red_d[kFT + tid] = s2; red_f[4 * kFT + tid] = mx;  // floats behind the two double arrays
         __syncthreads();
-        if (part == 0 && c < C) for (int r = 1; r < parts; ++r) { mm = fmaxf(mm, sred_f[r * C + c]); t1 += sred_d[r * C + c]; }
-        __syncthreads();
-        sred_d[tid] = s2;
-        __syncthreads();
-        if (part == 0 && c < C) for (int r = 1; r < parts; ++r) t2 += sred_d[r * C + c];
+        if (part == 0 && c < C)
+          for (int r = 1; r < parts; ++r) {
+            t1 += red_d[r * C + c]; t2 += red_d[kFT + r * C + c]; mm = fmaxf(mm, red_f[4 * kFT + r * C + c]);
+          }
         __syncthreads();
       }
       if (part == 0 && c < C) {
@@ -783,14 +848,15 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
         }
       }
     }
+    for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
     __syncthreads();
-    sred_f[tid] = gm;
+    if ((tid & 31) == 0) red_f[tid >> 5] = gm;
     __syncthreads();
-    for (int o = kFT / 2; o > 0; o >>= 1) {
-      if (tid < o) sred_f[tid] = fmaxf(sred_f[tid], sred_f[tid + o]);
-      __syncthreads();
+    if (tid == 0) {
+      float g = red_f[0];
+      for (int w = 1; w < kFT / 32; ++w) g = fmaxf(g, red_f[w]);
+      s_gmax = g;
     }
-    if (tid == 0) s_gmax = sred_f[0];
     __syncthreads();
   }
 
@@ -800,37 +866,50 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
 #pragma unroll
     for (int e = 0; e < VE; ++e) k[e] = 0u;
     if (real) {
-      float sg[VE];
+      if constexpr (kPacked) {
+        // |g| > sigma in binary32 is |g| > (sigma truncated to bf16) for a bf16 g; counts of up to
+        // 128 ones are exact in a bf16 accumulator
+        uint32_t thr[4], acc2[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-      for (int e = 0; e < VE; ++e) sg[e] = ch_sigma[c0 + e];
-      for (int i0 = 0; i0 < n_it; i0 += 4) {
-        Raw raw[4];
+        for (int j = 0; j < 4; ++j)
+          thr[j] = (__float_as_uint(ch_sigma[c0 + 2 * j]) >> 16) | (__float_as_uint(ch_sigma[c0 + 2 * j + 1]) & 0xFFFF0000u);
+        int run = 0;
+        auto flush = [&]() {
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const int i = i0 + u;
-          if (i < n_it)
-            raw[u] = i < a.slots ? slab[(size_t)i * kFT + tid] : load_raw<T, VE>(base + (first + (int64_t)i * rpi) * C);
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (i0 + u < n_it) {
-            float v[VE];
-            unpack_raw(raw[u], v, (const T*)nullptr);
-#pragma unroll
-            for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+          for (int j = 0; j < 4; ++j) {
+            k[2 * j] += (uint32_t)__uint_as_float(acc2[j] << 16);
+            k[2 * j + 1] += (uint32_t)__uint_as_float(acc2[j] & 0xFFFF0000u);
+            acc2[j] = 0u;
           }
-        }
+        };
+        auto body = [&](int, const Raw& raw) {
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
+          if (++run == 128) { run = 0; flush(); }
+        };
+        for_each_batched<4, Raw>(0, n_slab, load_slab, body);
+        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
+        flush();
+      } else {
+        float sg[VE];
+#pragma unroll
+        for (int e = 0; e < VE; ++e) sg[e] = ch_sigma[c0 + e];
+        auto body = [&](int, const Raw& raw) {
+          float v[VE];
+          unpack_raw(raw, v, (const T*)nullptr);
+#pragma unroll
+          for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+        };
+        for_each_batched<4, Raw>(0, n_slab, load_slab, body);
+        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
       }
     }
-#pragma unroll
-    for (int e = 0; e < VE; ++e) {
-      const uint32_t tot = column_reduce<uint32_t, false>(k[e], sred_u, Gp, rows_per_warp, rpi);
-      if (tid < G && tot) atomicAdd(a.ws.cnt + tid * VE + e, tot);
-    }
+    column_reduce<VE>(m, Gp, k, red_u, OpAdd(), [&](int c, uint32_t v) { if (c < C && v) atomicAdd(a.ws.cnt + c, v); });
     ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status);
   }
 
-  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------------
+  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------
   if (ok) {
     const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
     for (int c = tid; c < C; c += kFT) {
@@ -855,51 +934,68 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     __syncthreads();
 
     // ---------------- phase 3: both sets of codes -------------------------------------------------
-    if (active && n_it > 0) {
+    if (n_it > 0) {
+      using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
       float inv1[VE];
 #pragma unroll
       for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
       const float inv2 = inv_scale(s_gmax);
       const uint32_t key0 = sr_key(a.seed, 0u);
-      int64_t n = first / a.HW;
-      int64_t hw = first - n * a.HW;
-      for (int i0 = 0; i0 < n_it; i0 += 4) {
-        Raw pre[4];
+      const uint32_t keyx0 = key0 ^ (key0 >> 16);
+      const Idx HWi = (Idx)a.HW;
+      const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
+      const int64_t n0 = first / a.HW;
+      int64_t hw = first - n0 * a.HW;
+      Idx idx0 = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + (Idx)hw;   // NCHW index of (n, c0, hw)
+      int8_t* o1 = a.q1 + first * a.Cp + c0;
+      int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
+      const size_t o_stride = (size_t)rpi * a.Cp;
+      auto body = [&](int i, const Raw& raw) {
+        uint32_t ra[VE], rb[VE];
         if (real) {
+          float v[VE];
+          unpack_raw(raw, v, (const T*)nullptr);
+          Idx idx = idx0;
 #pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const int j = i0 + u;
-            if (j < n_it)
-              pre[u] = j < a.slots ? slab[(size_t)j * kFT + tid] : load_raw<T, VE>(base + (first + (int64_t)j * rpi) * C);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          if (i0 + u >= n_it) break;
-          const int64_t p = first + (int64_t)(i0 + u) * rpi;
-          int qa[VE], qb[VE];
-          if (real) {
-            float v[VE];
-            unpack_raw(pre[u], v, (const T*)nullptr);
-            const uint64_t idx0 = ((uint64_t)n * C + c0) * a.HW + hw;
-#pragma unroll
-            for (int e = 0; e < VE; ++e) {
-              const uint64_t idx = idx0 + (uint64_t)e * a.HW;
+          for (int e = 0; e < VE; ++e) {
+            uint32_t h;
+            if constexpr (IDX32) {
+              h = sr_hash_folded(idx, keyx0);
+            } else {
               const uint32_t hi = (uint32_t)(idx >> 32);
               const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-              const uint32_t h = avalanche32((uint32_t)idx ^ key);
-              qa[e] = quant_stochastic(v[e], inv1[e], sr_uniform(h));
-              qb[e] = DUAL ? quant_stochastic(v[e], inv2, sr_uniform(h * 0x9E3779B1u)) : 0;
+              h = avalanche32((uint32_t)idx ^ key);
             }
-          } else {
-#pragma unroll
-            for (int e = 0; e < VE; ++e) { qa[e] = 0; qb[e] = 0; }
+            ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
+            if constexpr (DUAL) rb[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+            idx += HWi;
           }
-          store_codes<VE>(a.q1 + p * a.Cp + c0, qa);
-          if (DUAL) store_codes<VE>(a.q2 + p * a.Cp + c0, qb);
-          hw += rpi;
-          while (hw >= a.HW) { hw -= a.HW; ++n; }
+        } else {
+#pragma unroll
+          for (int e = 0; e < VE; ++e) { ra[e] = 0u; rb[e] = 0u; }
         }
+        int8_t* d1 = o1 + (size_t)i * o_stride;
+        if constexpr (VE == 8) {
+          *reinterpret_cast<uint2*>(d1) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4], ra[5], ra[6], ra[7]));
+          if constexpr (DUAL)
+            *reinterpret_cast<uint2*>(o2 + (size_t)i * o_stride) =
+                make_uint2(pack_codes4(rb[0], rb[1], rb[2], rb[3]), pack_codes4(rb[4], rb[5], rb[6], rb[7]));
+        } else if constexpr (VE == 4) {
+          *reinterpret_cast<uint32_t*>(d1) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
+          if constexpr (DUAL) *reinterpret_cast<uint32_t*>(o2 + (size_t)i * o_stride) = pack_codes4(rb[0], rb[1], rb[2], rb[3]);
+        } else {
+          *d1 = (int8_t)(ra[0] & 0xFFu);
+          if constexpr (DUAL) *(o2 + (size_t)i * o_stride) = (int8_t)(rb[0] & 0xFFu);
+        }
+        hw += rpi;
+        idx0 += (Idx)rpi;
+        while (hw >= a.HW) { hw -= a.HW; idx0 += wrap; }
+      };
+      if (real) {
+        for_each_batched<2, Raw>(0, n_slab, load_slab, body);
+        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
+      } else {
+        for (int i = 0; i < n_it; ++i) body(i, Raw());
       }
     }
   }
@@ -930,10 +1026,10 @@ const FusedConfig& fused_config() {
   return cfg;
 }
 
-template <typename T, int VE, bool DUAL>
+template <typename T, int VE, bool DUAL, bool IDX32>
 dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   const FusedConfig& cfg = fused_config();
-  const size_t fixed = ((size_t)kFT * 12 + (size_t)a.C * 16 + 15) / 16 * 16;
+  const size_t fixed = (fused_red_bytes(VE) + (size_t)a.C * 16 + 15) / 16 * 16;
   const size_t budget = cfg.smem_max - 1024;   // static shared memory of the kernel
   const size_t slot_bytes = sizeof(typename RawVec<T, VE>::type) * kFT;
   // pixel rows handled per CTA iteration
@@ -942,11 +1038,11 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   if (ctas > cfg.sms) ctas = cfg.sms;
   const int64_t chunk = ceil_div64(a.npix, ctas);
   const int64_t its = ceil_div64(chunk, rpi);
-  int64_t slots = (int64_t)((budget - fixed) / slot_bytes);
+  int64_t slots = budget > fixed ? (int64_t)((budget - fixed) / slot_bytes) : 0;
   if (slots > its) slots = its;
   a.slots = (int)slots;
   const size_t smem = fixed + (size_t)slots * slot_bytes;
-  auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL>;
+  auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL, IDX32>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [&] {
@@ -957,6 +1053,12 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFT), args, smem, st));
   note_launch(1);
   return DAI8_OK;
+}
+
+template <typename T, int VE>
+dai8_status launch_fused_select(const T* dY, FusedArgs& a, bool dual, bool idx32, cudaStream_t st) {
+  if (dual) return idx32 ? launch_fused<T, VE, true, true>(dY, a, st) : launch_fused<T, VE, true, false>(dY, a, st);
+  return idx32 ? launch_fused<T, VE, false, true>(dY, a, st) : launch_fused<T, VE, false, false>(dY, a, st);
 }
 
 struct NhwcGrid {
@@ -1012,8 +1114,9 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
       a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
       if (!a.status) return DAI8_ERR_CUDA;
-      if (vec) return gq ? launch_fused<T, VEfull, true>(dY, a, st) : launch_fused<T, VEfull, false>(dY, a, st);
-      return gq ? launch_fused<T, 1, true>(dY, a, st) : launch_fused<T, 1, false>(dY, a, st);
+      const bool idx32 = npix * C < ((int64_t)1 << 32);   // NCHW element indices fit 32 bits
+      if (vec) return launch_fused_select<T, VEfull>(dY, a, gq != nullptr, idx32, st);
+      return launch_fused_select<T, 1>(dY, a, gq != nullptr, idx32, st);
     }
   }
   if (layout == DAI8_NHWC) {
