@@ -537,34 +537,42 @@ absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Fused NHWC path: the three sweeps in ONE persistent cooperative kernel (one CTA of 512 threads
-// per SM).  Every thread owns the same elements in all three phases (one 16-byte vector of channels
-// of every rpi-th pixel of the CTA's pixel range), so the part of the tensor that fits is parked in
-// shared memory during the first sweep and the later sweeps never touch HBM for it; the rest is
-// re-read (L2 hits for tensors of up to ~100 MB).  Between the phases the CTAs meet at a bounded
-// grid barrier and every CTA finishes the per-channel scalars for itself, in one fixed order, so
-// all of them hold identical sigma, class and clip values.
+// Fused NHWC path: the three sweeps in ONE persistent cooperative kernel, one CTA per SM.
 //
-// The kernel is bound by instruction issue rather than by HBM (two stochastic roundings per
-// element, each with its own hash-derived uniform), so the per-element instruction count is what
-// is optimised: bf16 inputs take |g|max and the density count two elements at a time in packed
-// bf16 arithmetic (both are exact there), codes come out of a magic-number addition instead of a
-// float-to-int conversion, and tensors of fewer than 2^32 elements use 32-bit index arithmetic.
+// A CTA owns a contiguous range of pixels, i.e. a contiguous byte range of dY.  One producer warp
+// streams that range into shared memory with bulk asynchronous copies (cp.async.bulk, completion on
+// mbarriers) in pieces of up to 16 KB; sixteen consumer warps work on the pieces.  As many pieces as
+// fit stay resident for all three phases, the rest cycles through a small ring and is fetched again
+// in the later phases (L2 hits for tensors of up to ~100 MB).  The producer runs ahead across phase
+// boundaries, so the first pieces of the next phase are already in flight while the CTAs meet at a
+// grid barrier.
+//
+// Between phase 1 and 2 the per-CTA partial moments are combined once: channel c is finished by one
+// warp of CTA c mod gridDim.x (fixed order, hence deterministic), and after a second barrier every
+// CTA reads the finished |g|max and sigma.  The density counts are integer atomics.
+//
+// Two things bound this kernel, and neither is HBM.  (1) Instruction issue in phase 3: two
+// stochastic roundings per element, each with its own hash-derived uniform.  So bf16 inputs take
+// |g|max and the density count two elements at a time in packed bf16 arithmetic (both are exact
+// there), codes come out of a magic-number addition instead of a float-to-int conversion, and
+// tensors of fewer than 2^32 elements use 32-bit index arithmetic.  (2) Everything outside the three
+// loops runs exactly once per CTA, straight from a cold instruction cache, at roughly ten cycles per
+// instruction: the code between the loops is therefore kept SMALL rather than fast -- one
+// out-of-line reduction routine with run-time loops serves all four column reductions, binary64
+// division and square root are avoided (reciprocals come from the host), spin loops are out of line.
 // ------------------------------------------------------------------------------------------------
-constexpr int kFT = 512;             // threads per CTA of the fused kernel (one CTA per SM)
+constexpr int kFT = 512;             // consumer threads per CTA (one CTA per SM)
+constexpr int kFusedThreads = kFT + 32;  // plus the producer warp
 constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
-constexpr long long kBarrierTimeoutCycles = 2000000000LL;
-// reduction scratch at the start of the dynamic shared memory: VE arrays of kFT doubles (at least 3)
-__host__ __device__ constexpr size_t fused_red_bytes(int ve) { return (size_t)(ve < 3 ? 3 : ve) * kFT * 8; }
+constexpr int kMaxSlots = 28;        // shared-memory pieces per CTA
+constexpr int kMaxRing = 4;
+constexpr int kPieceBytes = 16384;
+constexpr long long kWaitTimeoutCycles = 2000000000LL;  // about one second
 
-template <typename T, int VE> struct RawVec { using type = uint4; };
-template <typename T> struct RawVec<T, 1> { using type = T; };
+// reduction scratch at the start of the dynamic shared memory: per consumer thread and vector
+// element one float (max) and two doubles (sum, sum of squares)
+__host__ __device__ constexpr size_t fused_red_bytes(int ve) { return (size_t)ve * kFT * 20; }
 
-template <typename T, int VE>
-__device__ __forceinline__ typename RawVec<T, VE>::type load_raw(const T* p) {
-  if constexpr (VE == 1) return *p;
-  else return *reinterpret_cast<const uint4*>(p);
-}
 __device__ __forceinline__ void unpack_raw(const uint4& r, float (&v)[4], const float*) {
   v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
 }
@@ -573,8 +581,6 @@ __device__ __forceinline__ void unpack_raw(const uint4& r, float (&v)[8], const 
 #pragma unroll
   for (int i = 0; i < 4; ++i) { v[2 * i] = __uint_as_float(w[i] << 16); v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u); }
 }
-__device__ __forceinline__ void unpack_raw(const float& r, float (&v)[1], const float*) { v[0] = r; }
-__device__ __forceinline__ void unpack_raw(const bf16_t& r, float (&v)[1], const bf16_t*) { v[0] = to_f32(r); }
 
 // Packed bf16 helpers (two values per 32-bit word).  max and compare are exact in bf16.
 __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
@@ -594,10 +600,61 @@ __device__ __forceinline__ uint32_t bf16x2_add(uint32_t a, uint32_t b) {
   return d;
 }
 
+// ---- mbarrier / bulk-copy wrappers ---------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false if the CTA is giving up (this wait or another one ran out).
+__device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                            unsigned int* status) {
+  const long long t0 = clock64();
+  for (;;) {
+#pragma unroll 1
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitTimeoutCycles) {
+      *abort_flag = 1u;
+      atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
+      return false;
+    }
+  }
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag, status);
+}
+// Contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kFT) : "memory"); }
+
 struct FusedArgs {
   int64_t npix, HW;
+  double inv_M, inv_denom; // 1/M and 1/(M or M-1), from the host
   int C, Cp, G, Gp;        // G input vector columns, Gp output vector columns (>= G, zero padding)
-  int slots;               // vectors per thread kept in shared memory
+  int rows_per_warp, rpi;  // thread tiling, see fused_map
+  int rp;                  // pixel rows per piece (a multiple of rpi)
+  int slots, ring_log2;    // shared-memory pieces per CTA; log2 of how many of them cycle when not all fit
   GvqWs ws;
   uint32_t* gridbar;
   const float* sigma_override;
@@ -613,156 +670,249 @@ struct FusedArgs {
   unsigned int* status;
 };
 
-// All CTAs of a cooperative launch meet here.  Bounded: returns false (in every thread of the CTA)
-// if the others do not arrive in time, after recording DAI8_ERR_TIMEOUT.
-__device__ __forceinline__ bool grid_barrier(uint32_t* counter, uint32_t target, unsigned int* status) {
-  __shared__ uint32_t s_ok;
-  __syncthreads();
+// All consumer threads of all CTAs of a cooperative launch meet here.  Bounded: returns false (in
+// every consumer thread of the CTA) if the others do not arrive in time, after recording
+// DAI8_ERR_TIMEOUT.
+__device__ __noinline__ bool grid_barrier(uint32_t* counter, uint32_t target, unsigned int* status,
+                                          volatile uint32_t* abort_flag, uint32_t* s_ok) {
+  consumer_sync();
   if (threadIdx.x == 0) {
     __threadfence();
     atomicAdd(counter, 1u);
-    uint32_t ok = 1u;
+    uint32_t ok = *abort_flag ? 0u : 1u;
     const long long t0 = clock64();
-    while (*reinterpret_cast<volatile uint32_t*>(counter) < target) {
-      if (clock64() - t0 > kBarrierTimeoutCycles) {
+    while (ok && *reinterpret_cast<volatile uint32_t*>(counter) < target) {
+      if (clock64() - t0 > kWaitTimeoutCycles) {
         atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
+        *abort_flag = 1u;
         ok = 0u;
-        break;
       }
     }
     __threadfence();
-    s_ok = ok;
+    *s_ok = ok;
   }
-  __syncthreads();
-  return s_ok != 0u;
+  consumer_sync();
+  return *reinterpret_cast<volatile uint32_t*>(s_ok) != 0u;
 }
 
-// How the 512 threads of a CTA tile (pixel row, vector column) pairs.
-struct FusedMap {
-  int rows_per_warp;  // > 0 when a warp holds whole rows (Gp <= 32)
-  int rpi;            // pixel rows per CTA iteration
-  int col, rl;        // this thread's vector column and row lane
-  int nrows_smem;     // rows that reach shared memory in a column reduction
-  int row_smem;       // this thread's row there
-  bool active;
-};
+// How the 512 consumer threads of a CTA tile (pixel row, vector column) pairs: with Gp <= 32 vector
+// columns a warp holds rows_per_warp = 32/Gp whole rows, otherwise the CTA holds rpi = 512/Gp rows.
+__host__ __device__ inline int fused_rows_per_iteration(int Gp) { return Gp <= 32 ? (kFT / 32) * (32 / Gp) : kFT / Gp; }
 
-__device__ __forceinline__ FusedMap fused_map(int Gp) {
-  FusedMap m;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (Gp <= 32) {
-    m.rows_per_warp = 32 / Gp;
-    m.rpi = (kFT / 32) * m.rows_per_warp;
-    m.col = lane % Gp;
-    m.rl = warp * m.rows_per_warp + lane / Gp;
-    m.active = lane < m.rows_per_warp * Gp;
-    m.nrows_smem = kFT / 32;
-    m.row_smem = warp;
-  } else {
-    m.rows_per_warp = 0;
-    m.rpi = kFT / Gp;
-    m.col = tid % Gp;
-    m.rl = tid / Gp;
-    m.active = m.rl < m.rpi;
-    m.nrows_smem = m.rpi;
-    m.row_smem = m.rl;
-  }
-  return m;
+// Combines, in a fixed order, what the consumer threads have stored per (vector element e, pixel
+// row lane, vector column) at index e*kFT + row*Gp + col over the row lanes, and writes the result for
+// channel c = col*VE + e (c < C).  First `parts` interleaved subsets of the rows are combined in
+// place by all threads, then the subsets.  Ends with a consumer barrier, after which the scratch may
+// be rewritten.  Out of line, with run-time loops: it runs once per call and is kept small.
+struct RedIndex { int total0, parts, NV; };
+__device__ __forceinline__ RedIndex red_index(int rows, int Gp, int VE) {
+  RedIndex r;
+  r.NV = VE * Gp;
+  r.parts = r.NV >= kFT ? 1 : kFT / r.NV;
+  if (r.parts > rows) r.parts = rows;
+  r.total0 = r.NV * r.parts;
+  return r;
 }
 
-struct OpAdd { template <typename V> __device__ __forceinline__ V operator()(V a, V b) const { return a + b; } };
-struct OpMax { template <typename V> __device__ __forceinline__ V operator()(V a, V b) const { return a > b ? a : b; } };
-
-// Combines val[e] over the row lanes of the CTA for every (column, e), in a fixed order.  The result
-// for channel col*VE + e is handed to out(channel, value) by thread e*Gp + col.  `red` holds
-// VE * kFT values.  Two __syncthreads; `red` may be reused after the call returns.
-template <int VE, typename V, typename Op, typename Out>
-__device__ __forceinline__ void column_reduce(const FusedMap& m, int Gp, V (&val)[VE], V* red, Op op, Out out) {
-  const int tid = threadIdx.x, lane = tid & 31;
-  if (m.rows_per_warp > 1) {
-#pragma unroll
-    for (int e = 0; e < VE; ++e) {
-      V acc = val[e];
-      for (int k = 1; k < m.rows_per_warp; ++k) acc = op(acc, __shfl_sync(0xFFFFFFFFu, val[e], (lane + k * Gp) & 31));
-      val[e] = acc;
+// max (float) and two sums (double) at once: the statistics of phase 1
+__device__ __noinline__ void column_reduce_stats(float* smax, double* ssum, double* sss, int rows, int Gp, int VE,
+                                                 int C, float* out_max, double* out_sum, double* out_ss) {
+  const int tid = threadIdx.x;
+  const RedIndex ri = red_index(rows, Gp, VE);
+  consumer_sync();
+#pragma unroll 1
+  for (int idx = tid; idx < ri.total0; idx += kFT) {
+    const int p = idx / ri.NV, j = idx - p * ri.NV;
+    const int e = j / Gp, col = j - e * Gp;
+    const int cell = e * kFT + p * Gp + col;
+    float m = smax[cell];
+    double s1 = ssum[cell], s2 = sss[cell];
+#pragma unroll 4
+    for (int r = p + ri.parts; r < rows; r += ri.parts) {
+      const int o = cell + (r - p) * Gp;
+      m = fmaxf(m, smax[o]); s1 += ssum[o]; s2 += sss[o];
     }
+    smax[cell] = m; ssum[cell] = s1; sss[cell] = s2;
   }
-  const bool writer = m.rows_per_warp > 0 ? lane < Gp : m.active;
-  if (writer) {
-#pragma unroll
-    for (int e = 0; e < VE; ++e) red[e * kFT + m.row_smem * Gp + m.col] = val[e];
+  consumer_sync();
+#pragma unroll 1
+  for (int j = tid; j < ri.NV; j += kFT) {
+    const int e = j / Gp, col = j - e * Gp;
+    const int cell = e * kFT + col;
+    float m = smax[cell];
+    double s1 = ssum[cell], s2 = sss[cell];
+#pragma unroll 4
+    for (int p = 1; p < ri.parts; ++p) {
+      const int o = cell + p * Gp;
+      m = fmaxf(m, smax[o]); s1 += ssum[o]; s2 += sss[o];
+    }
+    const int c = col * VE + e;
+    if (c < C) { out_max[c] = m; out_sum[c] = s1; out_ss[c] = s2; }
   }
-  __syncthreads();
-  for (int t = tid; t < VE * Gp; t += kFT) {
-    const int e = t / Gp, col = t - e * Gp;
-    V acc = red[e * kFT + col];
-    for (int r = 1; r < m.nrows_smem; ++r) acc = op(acc, red[e * kFT + r * Gp + col]);
-    out(col * VE + e, acc);
-  }
-  __syncthreads();
+  consumer_sync();
 }
 
-// Runs f(i, raw) for i in [begin, end), loading U vectors ahead of the work on them.
-template <int U, typename Raw, typename Load, typename F>
-__device__ __forceinline__ void for_each_batched(int begin, int end, Load load, F f) {
-  int i = begin;
-  for (; i + U <= end; i += U) {
-    Raw r[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) r[u] = load(i + u);
-#pragma unroll
-    for (int u = 0; u < U; ++u) f(i + u, r[u]);
+// counts of phase 2, added to the global per-channel counters
+__device__ __noinline__ void column_reduce_counts(uint32_t* scnt, int rows, int Gp, int VE, int C, uint32_t* out) {
+  const int tid = threadIdx.x;
+  const RedIndex ri = red_index(rows, Gp, VE);
+  consumer_sync();
+#pragma unroll 1
+  for (int idx = tid; idx < ri.total0; idx += kFT) {
+    const int p = idx / ri.NV, j = idx - p * ri.NV;
+    const int e = j / Gp, col = j - e * Gp;
+    const int cell = e * kFT + p * Gp + col;
+    uint32_t n = scnt[cell];
+#pragma unroll 4
+    for (int r = p + ri.parts; r < rows; r += ri.parts) n += scnt[cell + (r - p) * Gp];
+    scnt[cell] = n;
   }
-  for (; i < end; ++i) f(i, load(i));
+  consumer_sync();
+#pragma unroll 1
+  for (int j = tid; j < ri.NV; j += kFT) {
+    const int e = j / Gp, col = j - e * Gp;
+    const int cell = e * kFT + col;
+    uint32_t n = scnt[cell];
+#pragma unroll 4
+    for (int p = 1; p < ri.parts; ++p) n += scnt[cell + p * Gp];
+    const int c = col * VE + e;
+    if (c < C && n) atomicAdd(out + c, n);
+  }
+  consumer_sync();
 }
+
+// The rare sigma whose square leaves the binary32 range.
+__device__ __noinline__ float sigma_wide(double var_over_denom) { return (float)sqrt(var_over_denom); }
 
 template <typename T, int VE, bool DUAL, bool IDX32>
-__global__ void __launch_bounds__(kFT, 1)
+__global__ void __launch_bounds__(kFusedThreads, 1)
 gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
-  using Raw = typename RawVec<T, VE>::type;
   constexpr bool kPacked = VE == 8;  // bf16 vectors: packed max / compare
-  extern __shared__ __align__(16) uint8_t fsmem[];
-  double* red_d = reinterpret_cast<double*>(fsmem);                      // [VE][kFT]
-  float* red_f = reinterpret_cast<float*>(fsmem);
-  uint32_t* red_u = reinterpret_cast<uint32_t*>(fsmem);
-  float* ch_absmax = reinterpret_cast<float*>(fsmem + fused_red_bytes(VE));      // [C]
-  float* ch_sigma = ch_absmax + a.C;                                     // [C]
-  float* ch_sprev = ch_sigma + a.C;                                      // [C]
-  float* ch_inv = ch_sprev + a.C;                                        // [C]
-  Raw* slab = reinterpret_cast<Raw*>(fsmem + ((fused_red_bytes(VE) + (size_t)a.C * 16 + 15) / 16) * 16);
-  __shared__ float s_gmax;
+  extern __shared__ __align__(128) uint8_t fsmem[];
+  __shared__ uint64_t full_bar[kMaxSlots], empty_bar[kMaxRing];
+  __shared__ volatile uint32_t s_abort;
+  __shared__ uint32_t s_ok;
 
-  const int tid = threadIdx.x;
+  double* red_sum = reinterpret_cast<double*>(fsmem);                    // [VE][kFT]
+  double* red_ss = red_sum + (size_t)VE * kFT;                           // [VE][kFT]
+  float* red_max = reinterpret_cast<float*>(red_ss + (size_t)VE * kFT);  // [VE][kFT]
+  uint32_t* red_cnt = reinterpret_cast<uint32_t*>(fsmem);                // [VE][kFT]
+  float* ch_absmax = reinterpret_cast<float*>(fsmem + fused_red_bytes(VE));  // [C + 1], last = layer |g|max
+  float* ch_sigma = ch_absmax + a.C + 1;                                 // [C]
+  float* ch_sprev = ch_sigma + a.C;                                      // [C]
+  float* ch_inv = ch_sprev + a.C;                                        // [C + 1], last = layer scale
+  uint8_t* pieces = fsmem + ((fused_red_bytes(VE) + (size_t)a.C * 16 + 8 + 127) / 128) * 128;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int C = a.C, Gp = a.Gp, G = a.G;
-  const FusedMap m = fused_map(Gp);
-  const int rpi = m.rpi, col = m.col;
-  const bool real = m.active && col < G;     // has input; columns >= G are code padding
-  const int c0 = col * VE;
+  const int rb = C * (int)sizeof(T);                 // bytes per pixel row
+  const int rp = a.rp;
+  const uint32_t piece_stride = (uint32_t)rp * (uint32_t)rb;   // bytes per shared-memory piece
   const int64_t chunk = (a.npix + gridDim.x - 1) / gridDim.x;
   const int64_t p0 = (int64_t)blockIdx.x * chunk;
   const int64_t p1 = min(a.npix, p0 + chunk);
-  const int64_t first = p0 + m.rl;
-  const int n_it = (m.active && first < p1) ? (int)((p1 - first + rpi - 1) / rpi) : 0;
-  const int n_slab = min(n_it, a.slots);
-  const T* base = x + c0 + first * C;
-  const size_t it_stride = (size_t)rpi * C;
-  auto load_global = [&](int i) { return load_raw<T, VE>(base + (size_t)i * it_stride); };
-  auto load_slab = [&](int i) { return slab[(size_t)i * kFT + tid]; };
+  const int rows_total = p1 > p0 ? (int)(p1 - p0) : 0;
+  const int K = (rows_total + rp - 1) / rp;          // pieces of this CTA
+  const int ring = 1 << a.ring_log2;
+  const int R = K <= a.slots ? K : a.slots - ring;   // pieces that stay resident
+  const int NS = K - R;                              // pieces streamed again in every phase
 
-  // ---------------- phase 1: statistics, parking the slab in shared memory ----------------------
+  if (tid == 0) {
+    s_abort = 0u;
+#pragma unroll 1
+    for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full_bar[s], 1);
+#pragma unroll 1
+    for (int r = 0; r < kMaxRing; ++r) mbar_init(&empty_bar[r], kFT / 32);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  // ---------------- producer warp ------------------------------------------------------------------
+  if (warp == kFT / 32) {
+    if (lane == 0) {
+      const uint8_t* src = reinterpret_cast<const uint8_t*>(x) + (size_t)p0 * rb;
+      // resident pieces once, then three passes (phase 1, 2, 3) over the streamed ones
+      const int items = R + 3 * NS;
+      int k = 0;
+#pragma unroll 1
+      for (int i = 0; i < items; ++i) {
+        int slot = i;
+        if (i >= R) {
+          const int t = i - R, r = t & (ring - 1);
+          slot = R + r;
+          if (t >= ring && !mbar_wait(&empty_bar[r], (uint32_t)((t >> a.ring_log2) - 1) & 1u, &s_abort, a.status)) break;
+        }
+        const uint32_t bytes = (uint32_t)min(rp, rows_total - k * rp) * (uint32_t)rb;
+        mbar_expect_tx(&full_bar[slot], bytes);
+        bulk_load(pieces + (size_t)slot * piece_stride, src + (size_t)k * piece_stride, bytes, &full_bar[slot]);
+        if (++k == K) k = R;
+      }
+    }
+    return;
+  }
+
+  // ---------------- consumers ----------------------------------------------------------------------
+  int col, rl;
+  bool active;
+  if (a.rows_per_warp > 0) {       // Gp <= 32: a warp holds rows_per_warp whole rows
+    const int r = lane / Gp;
+    col = lane - r * Gp;
+    rl = warp * a.rows_per_warp + r;
+    active = r < a.rows_per_warp;
+  } else {
+    rl = tid / Gp;
+    col = tid - rl * Gp;
+    active = rl < a.rpi;
+  }
+  const int rpi = a.rpi;
+  const bool real = active && col < G;       // has input; columns >= G are code padding
+  const int c0 = col * VE;
+  const int pos = rl * Gp + col;             // this thread's cell in the reduction scratch
+  int t_cons = 0;                            // streamed pieces consumed so far (all phases)
+  bool ok = true;
+
+  // Runs f(shared-memory piece, rows in it) over the CTA's pieces from `first_piece` on, in order:
+  // the resident ones wait for their one and only fill, the others for the current fill of their
+  // ring slot.  After phase 1 the resident pieces are one contiguous run of rows_res rows.
+  auto for_each_piece = [&](int first_piece, auto&& f) {
+#pragma unroll 1
+    for (int j = first_piece; j < K && ok; ++j) {
+      int slot = j, r = 0;
+      uint32_t parity = 0u;
+      if (j >= R) {
+        const int t = t_cons + (j - R);
+        r = t & (ring - 1);
+        slot = R + r;
+        parity = (uint32_t)(t >> a.ring_log2) & 1u;
+      }
+      ok = mbar_wait(&full_bar[slot], parity, &s_abort, a.status);
+      if (ok) f(pieces + (size_t)slot * piece_stride, min(rp, rows_total - j * rp));
+      if (j >= R) {
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[r]);
+      }
+    }
+    t_cons += NS;
+  };
+  const int rows_res = min(rows_total, R * rp);
+  auto vec_at = [&](const uint8_t* piece, int row) {
+    return *reinterpret_cast<const uint4*>(piece + ((uint32_t)row * (uint32_t)G + (uint32_t)col) * 16u);
+  };
+
+  // ---------------- phase 1: statistics -----------------------------------------------------------
   {
     float amax[VE], fs[VE], fss[VE], piv[VE];
-    uint32_t amax2[VE / 2 + 1];
+    uint32_t amax2[4] = {0u, 0u, 0u, 0u};
     double ds[VE], dss[VE];
 #pragma unroll
     for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; ds[e] = 0.0; dss[e] = 0.0; piv[e] = 0.f; }
-#pragma unroll
-    for (int j = 0; j < VE / 2 + 1; ++j) amax2[j] = 0u;
-    if (real) {
-      load_vec<T, VE>(x + c0, piv);  // pixel 0 of these channels
-      int run = 0;
-      auto body = [&](int i, const Raw& raw) {
-        if (i < n_slab) slab[(size_t)i * kFT + tid] = raw;
+    if (real) load_vec<T, VE>(x + c0, piv);  // pixel 0 of these channels
+    int run = 0;
+    for_each_piece(0, [&](const uint8_t* piece, int rows) {
+      if (!real) return;
+#pragma unroll 1
+      for (int row = rl; row < rows; row += rpi) {
+        const uint4 raw = vec_at(piece, row);
         float v[VE];
         unpack_raw(raw, v, (const T*)nullptr);
         if constexpr (kPacked) {
@@ -782,82 +932,89 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
 #pragma unroll
           for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
         }
-      };
-      for_each_batched<4, Raw>(0, n_it, load_global, body);
+      }
+    });
+    if constexpr (kPacked) {
 #pragma unroll
-      for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; }
-      if constexpr (kPacked) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          amax[2 * j] = __uint_as_float(amax2[j] << 16);
-          amax[2 * j + 1] = __uint_as_float(amax2[j] & 0xFFFF0000u);
-        }
+      for (int j = 0; j < 4; ++j) {
+        amax[2 * j] = __uint_as_float(amax2[j] << 16);
+        amax[2 * j + 1] = __uint_as_float(amax2[j] & 0xFFFF0000u);
       }
     }
+    // per-CTA partials of every channel: [blockIdx][C] rows of the workspace
     const size_t prow = (size_t)blockIdx.x * C;
-    column_reduce<VE>(m, Gp, amax, red_f, OpMax(), [&](int c, float v) { if (c < C) a.ws.pmax[prow + c] = v; });
-    column_reduce<VE>(m, Gp, ds, red_d, OpAdd(), [&](int c, double v) { if (c < C) a.ws.psum[prow + c] = v; });
-    column_reduce<VE>(m, Gp, dss, red_d, OpAdd(), [&](int c, double v) { if (c < C) a.ws.pss[prow + c] = v; });
+    if (active) {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) {
+        red_max[e * kFT + pos] = amax[e];
+        red_sum[e * kFT + pos] = ds[e] + (double)fs[e];
+        red_ss[e * kFT + pos] = dss[e] + (double)fss[e];
+      }
+    }
+    column_reduce_stats(red_max, red_sum, red_ss, rpi, Gp, VE, C, a.ws.pmax + prow, a.ws.psum + prow, a.ws.pss + prow);
   }
-  // previous clip values are read before the barrier after which CTA 0 overwrites them
+  // previous clip values are read before the barriers after which CTA 0 overwrites them
+#pragma unroll 1
   for (int c = tid; c < C; c += kFT) ch_sprev[c] = a.has_prev ? a.s_state[c] : 0.f;
-  bool ok = grid_barrier(a.gridbar, gridDim.x, a.status);
+  ok = grid_barrier(a.gridbar, gridDim.x, a.status, &s_abort, &s_ok) && ok;
 
-  // every CTA combines the per-CTA partials of every channel, in the same fixed order
+  // channel c is finished by one warp of CTA (c mod gridDim.x): fixed order over the CTAs' partials
   if (ok) {
     const int nblk = gridDim.x;
-    const int parts = C >= kFT ? 1 : kFT / C;
-    float gm = 0.f;
-    for (int cb = 0; cb < C; cb += kFT) {
-      const int c = parts == 1 ? cb + tid : tid % C;
-      const int part = parts == 1 ? 0 : tid / C;
+#pragma unroll 1
+    for (int c = blockIdx.x + nblk * warp; c < C; c += nblk * (kFT / 32)) {
       float mx = 0.f;
       double s1 = 0.0, s2 = 0.0;
-      if (c < C && part < parts) {
-        for (int b = part; b < nblk; b += parts) {
-          const size_t idx = (size_t)b * C + c;
-          mx = fmaxf(mx, __ldcg(a.ws.pmax + idx));
-          s1 += __ldcg(a.ws.psum + idx);
-          s2 += __ldcg(a.ws.pss + idx);
+      const double pivot = (double)to_f32(x[c]);
+#pragma unroll 1
+      for (int b0 = lane; b0 < nblk; b0 += 32 * 5) {   // five independent partials per round trip
+        float pm[5];
+        double p1[5], p2[5];
+#pragma unroll
+        for (int u = 0; u < 5; ++u) {
+          const int b = b0 + 32 * u;
+          const size_t idx = (size_t)(b < nblk ? b : b0) * C + c;
+          pm[u] = __ldcg(a.ws.pmax + idx); p1[u] = __ldcg(a.ws.psum + idx); p2[u] = __ldcg(a.ws.pss + idx);
         }
+#pragma unroll
+        for (int u = 0; u < 5; ++u)
+          if (b0 + 32 * u < nblk) { mx = fmaxf(mx, pm[u]); s1 += p1[u]; s2 += p2[u]; }
       }
-      float mm = mx; double t1 = s1, t2 = s2;
-      if (parts > 1) {   // combine the parts through shared memory: [0,kFT) s1, [kFT,2kFT) s2, then max
-        __syncthreads();
-        red_d[tid] = s1; red_d[kFT + tid] = s2; red_f[4 * kFT + tid] = mx;  // floats behind the two double arrays
-        __syncthreads();
-        if (part == 0 && c < C)
-          for (int r = 1; r < parts; ++r) {
-            t1 += red_d[r * C + c]; t2 += red_d[kFT + r * C + c]; mm = fmaxf(mm, red_f[4 * kFT + r * C + c]);
-          }
-        __syncthreads();
+#pragma unroll 1
+      for (int o = 16; o > 0; o >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+        s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
       }
-      if (part == 0 && c < C) {
-        float mean, sigma;
-        finish_moments((double)to_f32(x[c]), t1, t2, a.npix, a.mp, &mean, &sigma);
-        ch_absmax[c] = mm;
-        ch_sigma[c] = a.sigma_override ? a.sigma_override[c] : sigma;
-        gm = fmaxf(gm, mm);
-        if (blockIdx.x == 0) {
-          a.ws.absmax[c] = mm; a.ws.mean[c] = mean; a.ws.sigma[c] = sigma;
-          if (a.stats_out) {
-            a.stats_out[c * 4 + DAI8_STAT_ABSMAX] = mm;
-            a.stats_out[c * 4 + DAI8_STAT_MEAN] = mean;
-            a.stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
-          }
+      if (lane == 0) {
+        // mean and sigma from the moments of d = g - pivot; the pivot (the channel's first element)
+        // keeps sum d^2 - (sum d)^2/M free of cancellation when |mean| >> sigma
+        const double md = s1 * a.inv_M;
+        double var = a.mp.center_mean ? (s2 - s1 * md)
+                                      : (s2 + 2.0 * pivot * s1 + pivot * pivot * (double)a.npix);
+        var = fmax(var, 0.0) * a.inv_denom;
+        const float vf = (float)var;
+        const float sigma = (vf > 1e-30f || var == 0.0) ? sqrtf(vf) : sigma_wide(var);
+        const float mean = (float)(pivot + md);
+        a.ws.absmax[c] = mx; a.ws.mean[c] = mean; a.ws.sigma[c] = sigma;
+        if (a.stats_out) {
+          a.stats_out[c * 4 + DAI8_STAT_ABSMAX] = mx;
+          a.stats_out[c * 4 + DAI8_STAT_MEAN] = mean;
+          a.stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
         }
+        if (mx > 0.f) atomicMax(a.ws.gmax_bits, __float_as_uint(mx));  // non-negative floats order like their bits
       }
     }
-    for (int o = 16; o > 0; o >>= 1) gm = fmaxf(gm, __shfl_xor_sync(0xFFFFFFFFu, gm, o));
-    __syncthreads();
-    if ((tid & 31) == 0) red_f[tid >> 5] = gm;
-    __syncthreads();
-    if (tid == 0) {
-      float g = red_f[0];
-      for (int w = 1; w < kFT / 32; ++w) g = fmaxf(g, red_f[w]);
-      s_gmax = g;
+  }
+  ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
+  if (ok) {
+#pragma unroll 1
+    for (int c = tid; c < C; c += kFT) {
+      ch_absmax[c] = __ldcg(a.ws.absmax + c);
+      ch_sigma[c] = a.sigma_override ? a.sigma_override[c] : __ldcg(a.ws.sigma + c);
     }
-    __syncthreads();
+    if (tid == 0) ch_absmax[C] = __uint_as_float(__ldcg(a.ws.gmax_bits));
+    consumer_sync();
   }
 
   // ---------------- phase 2: density count -----------------------------------------------------
@@ -865,139 +1022,167 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     uint32_t k[VE];
 #pragma unroll
     for (int e = 0; e < VE; ++e) k[e] = 0u;
-    if (real) {
-      if constexpr (kPacked) {
-        // |g| > sigma in binary32 is |g| > (sigma truncated to bf16) for a bf16 g; counts of up to
-        // 128 ones are exact in a bf16 accumulator
-        uint32_t thr[4], acc2[4] = {0u, 0u, 0u, 0u};
+    if constexpr (kPacked) {
+      // |g| > sigma in binary32 is |g| > (sigma truncated to bf16) for a bf16 g; counts of up to
+      // 128 ones are exact in a bf16 accumulator
+      uint32_t thr[4] = {0u, 0u, 0u, 0u}, acc2[4] = {0u, 0u, 0u, 0u};
+      if (real) {
 #pragma unroll
         for (int j = 0; j < 4; ++j)
           thr[j] = (__float_as_uint(ch_sigma[c0 + 2 * j]) >> 16) | (__float_as_uint(ch_sigma[c0 + 2 * j + 1]) & 0xFFFF0000u);
-        int run = 0;
-        auto flush = [&]() {
-#pragma unroll
-          for (int j = 0; j < 4; ++j) {
-            k[2 * j] += (uint32_t)__uint_as_float(acc2[j] << 16);
-            k[2 * j + 1] += (uint32_t)__uint_as_float(acc2[j] & 0xFFFF0000u);
-            acc2[j] = 0u;
-          }
-        };
-        auto body = [&](int, const Raw& raw) {
-          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-          for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
-          if (++run == 128) { run = 0; flush(); }
-        };
-        for_each_batched<4, Raw>(0, n_slab, load_slab, body);
-        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
-        flush();
-      } else {
-        float sg[VE];
-#pragma unroll
-        for (int e = 0; e < VE; ++e) sg[e] = ch_sigma[c0 + e];
-        auto body = [&](int, const Raw& raw) {
-          float v[VE];
-          unpack_raw(raw, v, (const T*)nullptr);
-#pragma unroll
-          for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
-        };
-        for_each_batched<4, Raw>(0, n_slab, load_slab, body);
-        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
       }
+      int run = 0;
+      auto flush = [&]() {   // move the packed counts into the 32-bit counters
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          k[2 * j] += (uint32_t)__uint_as_float(acc2[j] << 16);
+          k[2 * j + 1] += (uint32_t)__uint_as_float(acc2[j] & 0xFFFF0000u);
+          acc2[j] = 0u;
+        }
+      };
+      auto body = [&](const uint4& raw) {
+        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
+        if (++run == 128) { run = 0; flush(); }
+      };
+      if (real) {
+#pragma unroll 4
+        for (int row = rl; row < rows_res; row += rpi) body(vec_at(pieces, row));
+      }
+      for_each_piece(R, [&](const uint8_t* piece, int rows) {
+        if (!real) return;
+#pragma unroll 1
+        for (int row = rl; row < rows; row += rpi) body(vec_at(piece, row));
+      });
+      flush();
+    } else {
+      float sg[VE];
+#pragma unroll
+      for (int e = 0; e < VE; ++e) sg[e] = real ? ch_sigma[c0 + e] : 0.f;
+      auto body = [&](const uint4& raw) {
+        float v[VE];
+        unpack_raw(raw, v, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+      };
+      if (real) {
+#pragma unroll 4
+        for (int row = rl; row < rows_res; row += rpi) body(vec_at(pieces, row));
+      }
+      for_each_piece(R, [&](const uint8_t* piece, int rows) {
+        if (!real) return;
+#pragma unroll 1
+        for (int row = rl; row < rows; row += rpi) body(vec_at(piece, row));
+      });
     }
-    column_reduce<VE>(m, Gp, k, red_u, OpAdd(), [&](int c, uint32_t v) { if (c < C && v) atomicAdd(a.ws.cnt + c, v); });
-    ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status);
+    if (active) {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) red_cnt[e * kFT + pos] = k[e];
+    }
+    column_reduce_counts(red_cnt, rpi, Gp, VE, C, a.ws.cnt);
   }
+  ok = grid_barrier(a.gridbar, 3u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
 
   // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------
   if (ok) {
     const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
-    for (int c = tid; c < C; c += kFT) {
-      const uint32_t cnt = __ldcg(a.ws.cnt + c);
+    const double thr = (double)a.mp.lambda * (double)a.npix;
+#pragma unroll 1
+    for (int c = tid; c <= C; c += kFT) {     // entry C: the layer-wide scale
       const float gmax = ch_absmax[c];
-      const bool bell = (double)cnt > (double)a.mp.lambda * (double)a.npix;
-      float s;
-      if (bell) {
-        s = gmax;
-      } else {
-        const float s_prev = a.has_prev ? ch_sprev[c] : gmax;
-        s = __fadd_rn(__fmul_rn(tcoef, s_prev), __fmul_rn(a.mp.A, gmax));
+      float s = gmax;
+      if (c < C) {
+        const uint32_t cnt = __ldcg(a.ws.cnt + c);
+        const bool bell = (double)cnt > thr;
+        if (!bell) {
+          const float s_prev = a.has_prev ? ch_sprev[c] : gmax;
+          s = __fadd_rn(__fmul_rn(tcoef, s_prev), __fmul_rn(a.mp.A, gmax));
+        }
+        if (blockIdx.x == 0) {
+          a.s_state[c] = s;
+          if (a.cls) a.cls[c] = bell ? 1 : 0;
+          if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt * a.inv_M);
+        }
+      } else if (blockIdx.x == 0) {
+        *a.gmax_layer = gmax;
       }
       ch_inv[c] = inv_scale(s);
-      if (blockIdx.x == 0) {
-        a.s_state[c] = s;
-        if (a.cls) a.cls[c] = bell ? 1 : 0;
-        if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt / (double)a.npix);
-      }
     }
-    if (blockIdx.x == 0 && tid == 0) *a.gmax_layer = s_gmax;
-    __syncthreads();
+    consumer_sync();
 
     // ---------------- phase 3: both sets of codes -------------------------------------------------
-    if (n_it > 0) {
-      using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
-      float inv1[VE];
+    using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
+    float inv1[VE];
 #pragma unroll
-      for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
-      const float inv2 = inv_scale(s_gmax);
-      const uint32_t key0 = sr_key(a.seed, 0u);
-      const uint32_t keyx0 = key0 ^ (key0 >> 16);
-      const Idx HWi = (Idx)a.HW;
-      const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
-      const int64_t n0 = first / a.HW;
-      int64_t hw = first - n0 * a.HW;
-      Idx idx0 = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + (Idx)hw;   // NCHW index of (n, c0, hw)
-      int8_t* o1 = a.q1 + first * a.Cp + c0;
-      int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
-      const size_t o_stride = (size_t)rpi * a.Cp;
-      auto body = [&](int i, const Raw& raw) {
-        uint32_t ra[VE], rb[VE];
-        if (real) {
-          float v[VE];
-          unpack_raw(raw, v, (const T*)nullptr);
-          Idx idx = idx0;
-#pragma unroll
-          for (int e = 0; e < VE; ++e) {
-            uint32_t h;
-            if constexpr (IDX32) {
-              h = sr_hash_folded(idx, keyx0);
-            } else {
-              const uint32_t hi = (uint32_t)(idx >> 32);
-              const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-              h = avalanche32((uint32_t)idx ^ key);
-            }
-            ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
-            if constexpr (DUAL) rb[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
-            idx += HWi;
-          }
-        } else {
-#pragma unroll
-          for (int e = 0; e < VE; ++e) { ra[e] = 0u; rb[e] = 0u; }
-        }
-        int8_t* d1 = o1 + (size_t)i * o_stride;
-        if constexpr (VE == 8) {
-          *reinterpret_cast<uint2*>(d1) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4], ra[5], ra[6], ra[7]));
-          if constexpr (DUAL)
-            *reinterpret_cast<uint2*>(o2 + (size_t)i * o_stride) =
-                make_uint2(pack_codes4(rb[0], rb[1], rb[2], rb[3]), pack_codes4(rb[4], rb[5], rb[6], rb[7]));
-        } else if constexpr (VE == 4) {
-          *reinterpret_cast<uint32_t*>(d1) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
-          if constexpr (DUAL) *reinterpret_cast<uint32_t*>(o2 + (size_t)i * o_stride) = pack_codes4(rb[0], rb[1], rb[2], rb[3]);
-        } else {
-          *d1 = (int8_t)(ra[0] & 0xFFu);
-          if constexpr (DUAL) *(o2 + (size_t)i * o_stride) = (int8_t)(rb[0] & 0xFFu);
-        }
-        hw += rpi;
-        idx0 += (Idx)rpi;
-        while (hw >= a.HW) { hw -= a.HW; idx0 += wrap; }
-      };
+    for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
+    const float inv2 = ch_inv[C];
+    const uint32_t key0 = sr_key(a.seed, 0u);
+    const uint32_t keyx0 = key0 ^ (key0 >> 16);
+    const Idx HWi = (Idx)a.HW;
+    const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
+    const int64_t first = p0 + rl;                 // this thread's first pixel
+    int64_t n0;
+    if constexpr (IDX32) n0 = (int64_t)((uint32_t)first / (uint32_t)a.HW);   // fewer than 2^32 elements
+    else n0 = first / a.HW;
+    Idx hw = (Idx)(first - n0 * a.HW);
+    Idx idx0 = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + hw;   // NCHW index of (n, c0, hw)
+    int8_t* o1 = a.q1 + first * a.Cp + c0;
+    int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
+    const size_t o_stride = (size_t)rpi * a.Cp;
+    auto body = [&](const uint8_t* piece, int row) {
+      uint32_t ra[VE], rb2[VE];
       if (real) {
-        for_each_batched<2, Raw>(0, n_slab, load_slab, body);
-        for_each_batched<4, Raw>(n_slab, n_it, load_global, body);
+        float v[VE];
+        unpack_raw(vec_at(piece, row), v, (const T*)nullptr);
+        Idx idx = idx0;
+#pragma unroll
+        for (int e = 0; e < VE; ++e) {
+          uint32_t h;
+          if constexpr (IDX32) {
+            h = sr_hash_folded(idx, keyx0);
+          } else {
+            const uint32_t hi = (uint32_t)(idx >> 32);
+            const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
+            h = avalanche32((uint32_t)idx ^ key);
+          }
+          ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
+          if constexpr (DUAL) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+          idx += HWi;
+        }
       } else {
-        for (int i = 0; i < n_it; ++i) body(i, Raw());
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { ra[e] = 0u; rb2[e] = 0u; }
       }
+      if constexpr (VE == 8) {
+        *reinterpret_cast<uint2*>(o1) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4], ra[5], ra[6], ra[7]));
+        if constexpr (DUAL)
+          *reinterpret_cast<uint2*>(o2) = make_uint2(pack_codes4(rb2[0], rb2[1], rb2[2], rb2[3]), pack_codes4(rb2[4], rb2[5], rb2[6], rb2[7]));
+      } else {
+        *reinterpret_cast<uint32_t*>(o1) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
+        if constexpr (DUAL) *reinterpret_cast<uint32_t*>(o2) = pack_codes4(rb2[0], rb2[1], rb2[2], rb2[3]);
+      }
+      o1 += o_stride;
+      if constexpr (DUAL) o2 += o_stride;
+      hw += (Idx)rpi;
+      idx0 += (Idx)rpi;
+      while (hw >= HWi) { hw -= HWi; idx0 += wrap; }
+    };
+    if (active) {
+#pragma unroll 1
+      for (int row = rl; row < rows_res; row += rpi) body(pieces, row);
     }
+    for_each_piece(R, [&](const uint8_t* piece, int rows) {
+      if (!active) return;
+#pragma unroll 1
+      for (int row = rl; row < rows; row += rpi) body(piece, row);
+    });
+  }
+
+  if (s_abort) {
+    // a wait ran out: give copies that may still be in flight time to land before the CTA ends
+#pragma unroll 1
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
   }
 }
 
@@ -1029,19 +1214,33 @@ const FusedConfig& fused_config() {
 template <typename T, int VE, bool DUAL, bool IDX32>
 dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   const FusedConfig& cfg = fused_config();
-  const size_t fixed = (fused_red_bytes(VE) + (size_t)a.C * 16 + 15) / 16 * 16;
+  const size_t fixed = (fused_red_bytes(VE) + (size_t)a.C * 16 + 8 + 127) / 128 * 128;
   const size_t budget = cfg.smem_max - 1024;   // static shared memory of the kernel
-  const size_t slot_bytes = sizeof(typename RawVec<T, VE>::type) * kFT;
-  // pixel rows handled per CTA iteration
-  const int rpi = a.Gp <= 32 ? (kFT / 32) * (32 / a.Gp) : kFT / a.Gp;
+  const int rb = a.C * (int)sizeof(T);
+  const int rpi = fused_rows_per_iteration(a.Gp);
+  a.rpi = rpi;
+  a.rows_per_warp = a.Gp <= 32 ? 32 / a.Gp : 0;
+  int mult = kPieceBytes / (rpi * rb);
+  if (mult < 1) mult = 1;
+  a.rp = rpi * mult;
+  const size_t piece_bytes = (size_t)a.rp * rb;
   int64_t ctas = ceil_div64(a.npix, rpi);
   if (ctas > cfg.sms) ctas = cfg.sms;
   const int64_t chunk = ceil_div64(a.npix, ctas);
-  const int64_t its = ceil_div64(chunk, rpi);
-  int64_t slots = budget > fixed ? (int64_t)((budget - fixed) / slot_bytes) : 0;
-  if (slots > its) slots = its;
+  const int64_t pieces = ceil_div64(chunk, a.rp);       // of the largest CTA
+  if (budget < fixed + 2 * piece_bytes) return DAI8_ERR_UNSUPPORTED;
+  int64_t slots = (int64_t)((budget - fixed) / piece_bytes);
+  if (slots > kMaxSlots) slots = kMaxSlots;
+  if (slots > pieces) slots = pieces;
   a.slots = (int)slots;
-  const size_t smem = fixed + (size_t)slots * slot_bytes;
+  a.ring_log2 = slots >= 8 ? 2 : (slots >= 4 ? 1 : 0);   // 4, 2 or 1 cycling pieces
+  {
+    const double M = (double)a.npix;
+    const double denom = a.mp.std_unbiased ? M - 1.0 : M;
+    a.inv_M = 1.0 / M;
+    a.inv_denom = denom > 0.0 ? 1.0 / denom : 0.0;
+  }
+  const size_t smem = fixed + (size_t)slots * piece_bytes;
   auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL, IDX32>;
   static std::once_flag once;
   static cudaError_t attr_err = cudaSuccess;
@@ -1050,7 +1249,7 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   });
   if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
   void* args[] = {(void*)&dY, (void*)&a};
-  DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFT), args, smem, st));
+  DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFusedThreads), args, smem, st));
   note_launch(1);
   return DAI8_OK;
 }
@@ -1104,20 +1303,16 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
   const float* sigma = sigma_override ? sigma_override : ws.sigma;
-  if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC) {
-    const bool vec = C % VEfull == 0;
-    const int ve = vec ? VEfull : 1;
-    if (Cp / ve <= kFT) {
-      FusedArgs a;
-      a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / ve; a.Gp = Cp / ve; a.slots = 0;
-      a.ws = ws; a.gridbar = ws.gridbar; a.sigma_override = sigma_override; a.mp = mp;
-      a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
-      a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
-      if (!a.status) return DAI8_ERR_CUDA;
-      const bool idx32 = npix * C < ((int64_t)1 << 32);   // NCHW element indices fit 32 bits
-      if (vec) return launch_fused_select<T, VEfull>(dY, a, gq != nullptr, idx32, st);
-      return launch_fused_select<T, 1>(dY, a, gq != nullptr, idx32, st);
-    }
+  if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
+    FusedArgs a;
+    a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Cp / VEfull;
+    a.rp = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0;
+    a.ws = ws; a.gridbar = ws.gridbar; a.sigma_override = sigma_override; a.mp = mp;
+    a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
+    a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
+    if (!a.status) return DAI8_ERR_CUDA;
+    const bool idx32 = npix * C < ((int64_t)1 << 32);   // NCHW element indices fit 32 bits
+    return launch_fused_select<T, VEfull>(dY, a, gq != nullptr, idx32, st);
   }
   if (layout == DAI8_NHWC) {
     if (C % VEfull == 0) {
