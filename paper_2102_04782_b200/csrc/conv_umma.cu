@@ -15,6 +15,7 @@
 // and a wait that expires records DAI8_ERR_TIMEOUT in the device status word instead of hanging.
 #include <cuda.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "conv_internal.cuh"
@@ -41,7 +42,10 @@ unsigned int* device_status_address() {
 namespace {
 
 constexpr int kBM = 128;                      // output pixels per tile (MMA M)
-constexpr int kThreadsIgemm = 192;
+constexpr int kThreadsIgemm = 192;      // weight-gradient kernel: TMA warp, MMA warp, 4 epilogue warps
+constexpr int kEpiWarps = 8;             // persistent kernel: two epilogue warps per tensor-memory lane quarter
+constexpr int kThreadsPersist = 64 + 32 * kEpiWarps;
+constexpr int kOutBlockBytes = 32 * 128; // epilogue staging block: 32 pixel rows x 128 bytes of channels
 constexpr long long kTimeoutCycles = 2000000000LL;  // about one second
 
 // ---------------------------------------------------------------------------------------------
@@ -100,10 +104,62 @@ __device__ __forceinline__ void tma_load_tile_3d(const CUtensorMap* map, uint64_
       ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
       : "memory");
 }
+// Shared -> global tile store (2D), tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void tma_store_tile_2d(const CUtensorMap* map, const void* src, int c0, int c1) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
 
+// Variants for the single-thread issue loops: shared-memory addresses are passed as 32-bit values
+// computed once, so that no generic-to-shared conversion or 64-bit arithmetic sits between two
+// issues (these loops are latency chains of one thread).
+__device__ __forceinline__ void mbar_expect_tx_a(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_4d_a(uint64_t map, uint32_t bar, uint32_t dst, int c, int w, int h,
+                                                     int n, uint16_t off_w, uint16_t off_h) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_tile_3d_a(uint64_t map, uint32_t bar, uint32_t dst, int c0, int c1, int c2) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4, %5}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_a(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// The 64-bit matrix descriptor of a K-major tile is a constant high word and a low word that holds
+// the 16-byte-granular address: stepping through chunks and K slices is a 32-bit addition.
+__device__ __forceinline__ uint32_t kmajor_desc_hi(int kc_bytes) {
+  const uint32_t layout = kc_bytes == 128 ? 2u : (kc_bytes == 64 ? 4u : 6u);
+  const uint32_t sbo = (uint32_t)(8 * kc_bytes) >> 4;
+  return sbo | (1u << 14) | (layout << 29);
+}
+__device__ __forceinline__ uint32_t kmajor_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
+__device__ __forceinline__ void mma_i8_parts(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
                "r"(ncols) : "memory");
@@ -161,19 +217,29 @@ struct IgemmParams {
   int G;                 // chunks per pipeline stage
   int k_iters;           // ceil(R*S*chunks_per_tap / G)
   int BN;                // output channels per tile (multiple of 16, <= 256)
-  int tmem_cols;         // power of two >= max(32, BN)
+  int tmem_cols;         // power of two >= max(32, 2*BN): two accumulator buffers
   int stages;
+  int m_tiles, n_tiles;  // tiles of 128 pixels x BN channels; tile t = m_tile*n_tiles + n_tile
+  int b_resident;        // the CTA's whole weight tile stays in shared memory (loaded once)
+  int tma_store;         // NHWC output rows are staged in shared memory and written with tile stores
+  int out_elem_bytes;    // 2 (bf16) or 4 (fp32, int32)
   int sh, sw, lower_h, lower_w;  // pixel (p,q) reads input (lower_h + p*sh + r, lower_w + q*sw + s)
   ConvOut out;
   const float* sa;
   const float* sb;
 };
 
-__global__ void __launch_bounds__(kThreadsIgemm, 1)
+// Persistent: a CTA walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The operand
+// ring keeps filling across tile boundaries and the accumulator is double-buffered in tensor
+// memory, so the epilogue of one tile overlaps the loads and MMAs of the next.  When the weight
+// tile of the CTA fits (it does for every ResNet / MobileNet layer with up to ~100 KB of weights per
+// BN output channels) it is loaded once and only activations stream; gridDim.x is then a multiple
+// of n_tiles so that a CTA always works on the same output channels.
+__global__ void __launch_bounds__(kThreadsPersist, 1)
 igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapB,
-                    const IgemmParams prm) {
+                    const __grid_constant__ CUtensorMap mapC, const IgemmParams prm) {
   extern __shared__ uint8_t smem_raw[];
-  __shared__ uint64_t full_bar[8], empty_bar[8], acc_bar;
+  __shared__ uint64_t full_bar[8], empty_bar[8], acc_full[2], acc_empty[2], b_full;
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
 
@@ -181,18 +247,19 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int a_chunk_bytes = kBM * prm.kc_bytes;
   const int b_chunk_bytes = prm.BN * prm.kc_bytes;
-  const int stage_bytes = prm.G * (a_chunk_bytes + b_chunk_bytes);
   const int total_chunks = prm.R * prm.S * prm.chunks_per_tap;
-
-  // the last tile is shifted back so that every tile covers 128 existing pixels
-  int m0 = blockIdx.x * kBM;
-  if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
-  const int n0 = blockIdx.y * prm.BN;
+  const int b_res_bytes = prm.b_resident ? total_chunks * b_chunk_bytes : 0;
+  const int chunk_pair_bytes = a_chunk_bytes + (prm.b_resident ? 0 : b_chunk_bytes);   // per chunk of a stage
+  const int stage_bytes = prm.G * chunk_pair_bytes;
+  uint8_t* stage_out = smem + ((b_res_bytes + 1023) & ~1023);   // [kEpiWarps][2][4 KB] when tma_store
+  uint8_t* ring = stage_out + (prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0);
+  const int num_tiles = prm.m_tiles * prm.n_tiles;
 
   if (threadIdx.x == 0) {
     abort_flag = 0u;
     for (int s = 0; s < prm.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    mbar_init(&acc_bar, 1);
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpiWarps); }
+    mbar_init(&b_full, 1);
     fence_mbar_init();
   }
   if (warp == 1) {
@@ -208,107 +275,240 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     if (lane == 0) {
       tma_prefetch_desc(&mapA);
       tma_prefetch_desc(&mapB);
-      const int q0 = m0 % prm.Q;
-      const int t = m0 / prm.Q;
-      const int p0 = t % prm.P, img = t / prm.P;
-      const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
-      for (int it = 0; it < prm.k_iters; ++it) {
-        const int s = it % prm.stages;
-        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag)) break;
-        const int c_begin = it * prm.G;
-        const int c_end = min(total_chunks, c_begin + prm.G);
-        mbar_expect_tx(&full_bar[s], (uint32_t)((c_end - c_begin) * (a_chunk_bytes + b_chunk_bytes)));
-        uint8_t* sa = smem + (size_t)s * stage_bytes;
-        uint8_t* sb = sa + prm.G * a_chunk_bytes;
-        for (int c = c_begin; c < c_end; ++c) {
+      if (prm.tma_store) tma_prefetch_desc(&mapC);
+      if (prm.b_resident) {
+        const int n0 = (blockIdx.x % prm.n_tiles) * prm.BN;
+        mbar_expect_tx(&b_full, (uint32_t)b_res_bytes);
+        for (int c = 0; c < total_chunks; ++c) {
           const int tap = c / prm.chunks_per_tap;
           const int k0 = (c - tap * prm.chunks_per_tap) * prm.kc_bytes;
-          const int r = tap / prm.S, ss = tap - r * prm.S;
-          tma_load_im2col_4d(&mapA, &full_bar[s], sa + (c - c_begin) * a_chunk_bytes, k0, cw, ch, img,
-                             (uint16_t)ss, (uint16_t)r);
-          tma_load_tile_3d(&mapB, &full_bar[s], sb + (c - c_begin) * b_chunk_bytes, k0, tap, n0);
+          tma_load_tile_3d(&mapB, &b_full, smem + (size_t)c * b_chunk_bytes, k0, tap, n0);
         }
+      }
+      // A single thread drives the copy engine, so this loop is a latency chain: no integer
+      // divisions (ring stage, tile position and filter tap are running counters) and only 32-bit
+      // shared-memory addresses computed up front.
+      const uint64_t pa = reinterpret_cast<uint64_t>(&mapA), pb = reinterpret_cast<uint64_t>(&mapB);
+      const uint32_t ring_a = smem_u32(ring), full_a = smem_u32(&full_bar[0]);
+      const int G = prm.G, S = prm.S, cpt = prm.chunks_per_tap, kc = prm.kc_bytes, nst = prm.stages, kit = prm.k_iters;
+      const bool resident = prm.b_resident != 0;
+      int stage = 0;
+      uint32_t phase = 0;            // parity of the current pass over the ring
+      bool first_pass = true;        // nothing to wait for until the ring has wrapped once
+      bool ok = true;
+      int t = blockIdx.x;
+      int m_tile = t / prm.n_tiles, n_tile = t - m_tile * prm.n_tiles;
+      const int dm = gridDim.x / prm.n_tiles, dn = gridDim.x - dm * prm.n_tiles;   // tile step of this CTA
+      for (; t < num_tiles && ok; t += gridDim.x) {
+        const int n0 = n_tile * prm.BN;
+        // the last tile is shifted back so that every tile covers 128 existing pixels
+        int m0 = m_tile * kBM;
+        if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
+        const int tq = m0 / prm.Q;               // one division pair per tile (not per load)
+        const int q0 = m0 - tq * prm.Q;
+        const int img = tq / prm.P, p0 = tq - img * prm.P;
+        const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
+        int c = 0, k0 = 0, kchunk = 0, r = 0, ss = 0;    // chunk, its channel offset, tap row and column
+        for (int it = 0; it < kit; ++it) {
+          if (!first_pass && !mbar_wait(&empty_bar[stage], phase ^ 1u, &abort_flag)) { ok = false; break; }
+          const int nch = min(total_chunks - c, G);
+          const uint32_t bar = full_a + 8u * (uint32_t)stage;
+          mbar_expect_tx_a(bar, (uint32_t)(nch * chunk_pair_bytes));
+          uint32_t sa = ring_a + (uint32_t)(stage * stage_bytes);
+          uint32_t sb = sa + (uint32_t)(G * a_chunk_bytes);
+          for (int j = 0; j < nch; ++j, ++c) {
+            tma_load_im2col_4d_a(pa, bar, sa, k0, cw, ch, img, (uint16_t)ss, (uint16_t)r);
+            if (!resident) tma_load_tile_3d_a(pb, bar, sb, k0, r * S + ss, n0);
+            sa += (uint32_t)a_chunk_bytes; sb += (uint32_t)b_chunk_bytes;
+            k0 += kc;
+            if (++kchunk == cpt) { kchunk = 0; k0 = 0; if (++ss == S) { ss = 0; ++r; } }
+          }
+          if (++stage == nst) { stage = 0; phase ^= 1u; first_pass = false; }
+        }
+        m_tile += dm; n_tile += dn;
+        if (n_tile >= prm.n_tiles) { n_tile -= prm.n_tiles; ++m_tile; }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
       const uint32_t idesc = idesc_i8_kmajor(prm.BN);
-      uint32_t accumulate = 0;
-      bool ok = true;
-      for (int it = 0; it < prm.k_iters && ok; ++it) {
-        const int s = it % prm.stages;
-        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag);
+      bool ok = !prm.b_resident || mbar_wait(&b_full, 0, &abort_flag);
+      int stage = 0, tile_i = 0;
+      uint32_t phase = 0;
+      const int kk_n = prm.kc_bytes / 32, G = prm.G, nst = prm.stages, kit = prm.k_iters;
+      const bool resident = prm.b_resident != 0;
+      const uint32_t dhi = kmajor_desc_hi(prm.kc_bytes);
+      const uint32_t ring_lo = kmajor_desc_lo(smem_u32(ring)), bres_lo = kmajor_desc_lo(smem_u32(smem));
+      const uint32_t stage_step = (uint32_t)stage_bytes >> 4, a_step = (uint32_t)a_chunk_bytes >> 4,
+                     b_step = (uint32_t)b_chunk_bytes >> 4;
+      const uint32_t empty_a = smem_u32(&empty_bar[0]);
+      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_i) {
+        const int buf = tile_i & 1;
+        if (tile_i >= 2) ok = mbar_wait(&acc_empty[buf], ((tile_i >> 1) - 1) & 1, &abort_flag);
         if (!ok) break;
         tc_fence_after();
-        const int c_begin = it * prm.G;
-        const int c_end = min(total_chunks, c_begin + prm.G);
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t sb = sa + prm.G * a_chunk_bytes;
-        for (int c = 0; c < c_end - c_begin; ++c) {
-          const uint64_t ad = kmajor_desc(sa + c * a_chunk_bytes, prm.kc_bytes);
-          const uint64_t bd = kmajor_desc(sb + c * b_chunk_bytes, prm.kc_bytes);
-          for (int kk = 0; kk < prm.kc_bytes / 32; ++kk) {
-            mma_i8(tmem_base, ad + (uint64_t)(kk * 2), bd + (uint64_t)(kk * 2), idesc, accumulate);
-            accumulate = 1;
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * prm.BN);
+        uint32_t accumulate = 0;
+        int c = 0;
+        uint32_t bres = bres_lo;                 // descriptor low word of the next resident weight chunk
+        for (int it = 0; it < kit; ++it) {
+          ok = mbar_wait(&full_bar[stage], phase, &abort_flag);
+          if (!ok) break;
+          tc_fence_after();
+          const int nch = min(total_chunks - c, G);
+          uint32_t a_lo = ring_lo + (uint32_t)stage * stage_step;
+          uint32_t b_lo = resident ? bres : a_lo + (uint32_t)G * a_step;
+          for (int j = 0; j < nch; ++j) {
+            for (int kk = 0; kk < kk_n; ++kk) {
+              mma_i8_parts(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, dhi, idesc, accumulate);
+              accumulate = 1;
+            }
+            a_lo += a_step; b_lo += b_step;
           }
+          c += nch;
+          bres += (uint32_t)nch * b_step;
+          tc_commit_a(empty_a + 8u * (uint32_t)stage);   // frees the stage once these MMAs have read it
+          if (++stage == nst) { stage = 0; phase ^= 1u; }
         }
-        tc_commit(&empty_bar[s]);   // frees the stage once these MMAs have read it
+        if (ok) tc_commit(&acc_full[buf]);  // accumulator of this tile complete
       }
-      if (ok) tc_commit(&acc_bar);  // accumulator complete
     }
   } else {
-    // epilogue: warp w may touch tensor-memory lanes 32*(w%4) .. 32*(w%4)+31
+    // epilogue: warp w may touch tensor-memory lanes 32*(w%4) .. 32*(w%4)+31; the two warps of a
+    // lane quarter take alternate groups of 32 accumulator columns
     const int quarter = warp & 3;
-    const bool ok = mbar_wait(&acc_bar, 0, &abort_flag);
-    tc_fence_after();
-    if (ok) {
+    const int half = (warp - 2) >> 2;
+    const bool nhwc = prm.out.layout == DAI8_NHWC;
+    const bool vec_ok = nhwc && (prm.Nout & 15) == 0;
+    const size_t plane = (size_t)prm.P * prm.Q;
+    const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
+    int tile_i = 0, n_store = 0;
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++tile_i) {
+      const int buf = tile_i & 1;
+      if (!mbar_wait(&acc_full[buf], (tile_i >> 1) & 1, &abort_flag)) break;
+      tc_fence_after();
+      const int m_tile = t / prm.n_tiles;
+      const int n0 = (t - m_tile * prm.n_tiles) * prm.BN;
+      int m0 = m_tile * kBM;
+      if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
       const int m = m0 + quarter * 32 + lane;
-      const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
       const int q = m % prm.Q;
-      const int t = m / prm.Q;
-      const int p = t % prm.P, img = t / prm.P;
-      const bool nhwc = prm.out.layout == DAI8_NHWC;
+      const int tq = m / prm.Q;
+      const int p = tq % prm.P, img = tq / prm.P;
       const size_t pix_base = nhwc ? (size_t)m * prm.Nout : 0;
-      const size_t plane = (size_t)prm.P * prm.Q;
-      for (int cg = 0; cg < prm.BN / 16; ++cg) {
-        int v[16];
-        tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cg * 16), v);
-        tmem_ld_wait();
-        const int j0 = n0 + cg * 16;
-        if (j0 >= prm.Nout) break;
-        if (nhwc && j0 + 16 <= prm.Nout && (prm.Nout & 15) == 0) {
-          if (prm.out.dtype == DAI8_F32) {
-            float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.out.ptr) + pix_base + j0);
+      const uint32_t t_tmem = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * prm.BN);
+      if (prm.tma_store) {
+        // Rows of this warp's 32 pixels go through a 128-byte-swizzled staging block and leave as one
+        // tile store per 128 bytes of channels: the copy engine writes whole row segments, where
+        // per-lane stores would scatter 16-byte pieces over 32 rows.
+        const int cols_per_block = 128 / prm.out_elem_bytes;          // 32 (fp32, int32) or 64 (bf16)
+        const int row_bytes = prm.BN * prm.out_elem_bytes;
+        uint8_t* my_stage = stage_out + (size_t)(warp - 2) * 2 * kOutBlockBytes;
+        for (int blk = half; blk * 128 < row_bytes; blk += 2) {
+          const int col = blk * cols_per_block;
+          if (n0 + col >= prm.Nout) break;
+          uint8_t* st = my_stage + (size_t)(n_store & 1) * kOutBlockBytes;
+          if (lane == 0 && n_store >= 2) bulk_wait_read<1>();   // the store that last used this block has read it
+          __syncwarp();
+          uint8_t* row = st + lane * 128;
+#pragma unroll 1
+          for (int sub = 0; sub * 32 < cols_per_block; ++sub) {
+            int va[2][16];
+            tmem_ld16(t_tmem + (uint32_t)(col + sub * 32), va[0]);
+            tmem_ld16(t_tmem + (uint32_t)(col + sub * 32 + 16), va[1]);
+            tmem_ld_wait();
+            if (prm.out.dtype == DAI8_BF16) {
+              // 32 columns -> 64 bytes = chunks 4*sub .. 4*sub+3 of the row
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
-              dst[i] = make_float4(__fmul_rn(__int2float_rn(v[4 * i]), scale), __fmul_rn(__int2float_rn(v[4 * i + 1]), scale),
-                                   __fmul_rn(__int2float_rn(v[4 * i + 2]), scale), __fmul_rn(__int2float_rn(v[4 * i + 3]), scale));
-          } else if (prm.out.dtype == DAI8_BF16) {
-            uint32_t w[8];
+              for (int g = 0; g < 2; ++g) {
+                uint32_t w[8];
 #pragma unroll
-            for (int i = 0; i < 8; ++i)
-              w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i]), scale)) |
-                     ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i + 1]), scale)) << 16);
-            uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(prm.out.ptr) + pix_base + j0);
-            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
-          } else {
-            int4* dst = reinterpret_cast<int4*>(static_cast<int*>(prm.out.ptr) + pix_base + j0);
+                for (int i = 0; i < 8; ++i)
+                  w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(va[g][2 * i]), scale)) |
+                         ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(va[g][2 * i + 1]), scale)) << 16);
+                const int c0 = sub * 4 + g * 2;
+                *reinterpret_cast<uint4*>(row + (((c0) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+                *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ (lane & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
+              }
+            } else {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) dst[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              for (int g = 0; g < 2; ++g)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  uint4 o;
+                  if (prm.out.dtype == DAI8_F32) {
+                    o.x = __float_as_uint(__fmul_rn(__int2float_rn(va[g][4 * i]), scale));
+                    o.y = __float_as_uint(__fmul_rn(__int2float_rn(va[g][4 * i + 1]), scale));
+                    o.z = __float_as_uint(__fmul_rn(__int2float_rn(va[g][4 * i + 2]), scale));
+                    o.w = __float_as_uint(__fmul_rn(__int2float_rn(va[g][4 * i + 3]), scale));
+                  } else {
+                    o = make_uint4((uint32_t)va[g][4 * i], (uint32_t)va[g][4 * i + 1], (uint32_t)va[g][4 * i + 2], (uint32_t)va[g][4 * i + 3]);
+                  }
+                  *reinterpret_cast<uint4*>(row + (((g * 4 + i) ^ (lane & 7)) << 4)) = o;
+                }
+            }
           }
-        } else {
+          fence_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_tile_2d(&mapC, st, (n0 + col) * prm.out_elem_bytes, m0 + quarter * 32);
+            bulk_commit();
+          }
+          ++n_store;
+        }
+      } else
+      for (int cg2 = half; cg2 * 32 < prm.BN; cg2 += 2) {
+        const int col = cg2 * 32;
+        if (n0 + col >= prm.Nout) break;
+        const bool second = col + 16 < prm.BN && n0 + col + 16 < prm.Nout;
+        int va[2][16];
+        tmem_ld16(t_tmem + (uint32_t)col, va[0]);           // both loads in flight, one wait
+        if (second) tmem_ld16(t_tmem + (uint32_t)(col + 16), va[1]);
+        tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            const int j = j0 + i;
-            if (j < prm.Nout) {
-              const size_t idx = nhwc ? pix_base + j : ((size_t)img * prm.Nout + j) * plane + (size_t)p * prm.Q + q;
-              store_result(prm.out.ptr, prm.out.dtype, idx, v[i], scale);
+        for (int g = 0; g < 2; ++g) {
+          if (g == 1 && !second) break;
+          const int (&v)[16] = va[g];
+          const int j0 = n0 + col + g * 16;
+          if (vec_ok && j0 + 16 <= prm.Nout) {
+            if (prm.out.dtype == DAI8_F32) {
+              float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.out.ptr) + pix_base + j0);
+#pragma unroll
+              for (int i = 0; i < 4; ++i)
+                dst[i] = make_float4(__fmul_rn(__int2float_rn(v[4 * i]), scale), __fmul_rn(__int2float_rn(v[4 * i + 1]), scale),
+                                     __fmul_rn(__int2float_rn(v[4 * i + 2]), scale), __fmul_rn(__int2float_rn(v[4 * i + 3]), scale));
+            } else if (prm.out.dtype == DAI8_BF16) {
+              uint32_t w[8];
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i]), scale)) |
+                       ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i + 1]), scale)) << 16);
+              uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(prm.out.ptr) + pix_base + j0);
+              dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+              dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+            } else {
+              int4* dst = reinterpret_cast<int4*>(static_cast<int*>(prm.out.ptr) + pix_base + j0);
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dst[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              const int j = j0 + i;
+              if (j < prm.Nout) {
+                const size_t idx = nhwc ? pix_base + j : ((size_t)img * prm.Nout + j) * plane + (size_t)p * prm.Q + q;
+                store_result(prm.out.ptr, prm.out.dtype, idx, v[i], scale);
+              }
             }
           }
         }
       }
+      // this warp has read its lanes of the buffer: hand it back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&acc_empty[buf]);
     }
+    if (prm.tma_store && lane == 0) bulk_wait_read<0>();   // staging blocks must outlive their stores
   }
 
   // teardown: everything this CTA issued must have drained before tensor memory is released
@@ -388,6 +588,19 @@ bool igemm_supported(const IgemmProblem& pb) {
   return true;
 }
 
+int sm_count() {
+  static int cached = 0;
+  if (cached == 0) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      cached = sms;
+    else
+      return 148;
+  }
+  return cached;
+}
+
 dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* sb, const ConvOut& out,
                          cudaStream_t st) {
   if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
@@ -404,17 +617,38 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   prm.BN = noutp < 256 ? noutp : 256;
   if (noutp > 256 && noutp % 256 != 0 && noutp % 128 == 0) prm.BN = 128;
   prm.tmem_cols = 32;
-  while (prm.tmem_cols < prm.BN) prm.tmem_cols *= 2;
-  const int stage_bytes = prm.G * (kBM + prm.BN) * prm.kc_bytes;
-  int stages = (200 * 1024) / stage_bytes;
+  while (prm.tmem_cols < 2 * prm.BN) prm.tmem_cols *= 2;
+  prm.m_tiles = (prm.Mtot + kBM - 1) / kBM;
+  prm.n_tiles = (noutp + prm.BN - 1) / prm.BN;
+  const int smem_budget = 227 * 1024 - 2048 - 1024;   // opt-in limit minus static and alignment slack
+  const int a_chunk = kBM * prm.kc_bytes, b_chunk = prm.BN * prm.kc_bytes;
+  const int b_res = (total_chunks * b_chunk + 1023) & ~1023;
+  const int out_es = out.dtype == DAI8_BF16 ? 2 : 4;
+  prm.out_elem_bytes = out_es;
+  prm.tma_store = (out.layout == DAI8_NHWC && (pb.Nout * out_es) % 16 == 0 && pb.Nout * out_es >= 128) ? 1 : 0;
+  const int stage_out_bytes = prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0;
+  prm.b_resident = b_res <= 96 * 1024 ? 1 : 0;
+  const int stage_bytes = prm.G * (a_chunk + (prm.b_resident ? 0 : b_chunk));
+  int stages = (smem_budget - stage_out_bytes - (prm.b_resident ? b_res : 0)) / stage_bytes;
   if (stages > 8) stages = 8;
-  if (stages > prm.k_iters) stages = prm.k_iters;
-  if (stages < 1) return DAI8_ERR_UNSUPPORTED;
+  if (stages < 2) return DAI8_ERR_UNSUPPORTED;
   prm.stages = stages;
   prm.sh = pb.sh; prm.sw = pb.sw; prm.lower_h = pb.lower_h; prm.lower_w = pb.lower_w;
   prm.out = out; prm.sa = sa; prm.sb = sb;
 
-  CUtensorMap mapA, mapB;
+  CUtensorMap mapA, mapB, mapC;
+  memset(&mapC, 0, sizeof(mapC));
+  if (prm.tma_store) {
+    // output viewed as bytes: [pixels][Nout*es], stored in boxes of 32 rows x 128 bytes
+    const cuuint64_t dims[2] = {(cuuint64_t)pb.Nout * out_es, (cuuint64_t)prm.Mtot};
+    const cuuint64_t strides[1] = {(cuuint64_t)pb.Nout * out_es};
+    const cuuint32_t box[2] = {128, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, out.ptr, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  }
   {
     const cuuint64_t dims[4] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.Wi, (cuuint64_t)pb.Hi, (cuuint64_t)pb.N};
     const cuuint64_t strides[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.Wi * pb.Kc, (cuuint64_t)pb.Hi * pb.Wi * pb.Kc};
@@ -438,15 +672,19 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
-  const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
+  const size_t smem_bytes = (size_t)(prm.b_resident ? b_res : 0) + stage_out_bytes + (size_t)stages * stage_bytes + 1024;
   static std::once_flag attr_once;
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [] {
     attr_err = cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
   });
   if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
-  const dim3 grid((unsigned)((prm.Mtot + kBM - 1) / kBM), (unsigned)((noutp + prm.BN - 1) / prm.BN), 1);
-  igemm_kmajor_kernel<<<grid, kThreadsIgemm, smem_bytes, st>>>(mapA, mapB, prm);
+  // one persistent CTA per SM; with resident weights a CTA keeps its output-channel tile
+  const int num_tiles = prm.m_tiles * prm.n_tiles;
+  int ctas = sm_count();
+  if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
+  if (ctas > num_tiles) ctas = num_tiles;
+  igemm_kmajor_kernel<<<dim3((unsigned)ctas), kThreadsPersist, smem_bytes, st>>>(mapA, mapB, mapC, prm);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
@@ -578,8 +816,12 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128, N = Nw
-      const uint32_t idesc = idesc_i8_kmajor(Nw) | (1u << 15) | (1u << 16);
+      // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128.  The
+      // boxes of consecutive taps lie side by side in shared memory and in tensor memory, so one
+      // MMA covers as many of them as fit N <= 256: an instruction costs about the same whether it
+      // is 64 or 256 columns wide (the 128-row operand is fetched once per instruction).
+      const int nbox = ntap * prm.nb;              // boxes of bw channels in this CTA's stage
+      const int per_mma = 256 / prm.bw;            // boxes per MMA
       bool ok = true;
       for (int it = 0; it < k_iters && ok; ++it) {
         const int s = it % prm.stages;
@@ -589,10 +831,12 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         const uint32_t sb = sa + a_bytes;
         const uint64_t ad = mnmajor_desc(sa, 128, (uint32_t)a_bytes);
-        for (int tl = 0; tl < ntap; ++tl) {
-          const uint64_t bd = mnmajor_desc(sb + tl * prm.nb * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
+        for (int b0 = 0; b0 < nbox; b0 += per_mma) {
+          const int cnt = min(per_mma, nbox - b0);
+          const uint32_t idesc = idesc_i8_kmajor(cnt * prm.bw) | (1u << 15) | (1u << 16);
+          const uint64_t bd = mnmajor_desc(sb + b0 * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
           for (int kk = 0; kk < kKP / 32; ++kk)
-            mma_i8(tmem_base + (uint32_t)(tl * Nw), ad + (uint64_t)((kk * 32 * 128) >> 4),
+            mma_i8(tmem_base + (uint32_t)(b0 * prm.bw), ad + (uint64_t)((kk * 32 * 128) >> 4),
                    bd + (uint64_t)((kk * 32 * prm.bw) >> 4), idesc, (it > 0 || kk > 0) ? 1u : 0u);
         }
         tc_commit(&empty_bar[s]);

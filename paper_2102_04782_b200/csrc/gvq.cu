@@ -1358,6 +1358,52 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   return DAI8_OK;
 }
 
+// Small tensors (weights): one CTA finds max|x| and writes the codes, so the call is a single
+// launch instead of memset + reduction + quantization.
+constexpr int kSmallThreads = 1024;
+constexpr int64_t kSmallTensorElems = 131072;
+
+template <typename T, bool NHWC_IN>
+__global__ void __launch_bounds__(kSmallThreads)
+quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int absmax_mode, int stochastic,
+                      uint32_t seed, float* __restrict__ scale, int8_t* __restrict__ q) {
+  __shared__ float s_part[kSmallThreads / 32];
+  __shared__ float s_scale;
+  const int tid = threadIdx.x;
+  const int total = N * C * HW;
+  if (absmax_mode) {
+    float m = 0.f;
+    for (int i = tid; i < total; i += kSmallThreads) m = fmaxf(m, fabsf(to_f32(x[i])));
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    if ((tid & 31) == 0) s_part[tid >> 5] = m;
+    __syncthreads();
+    if (tid < 32) {
+      m = s_part[tid];
+      for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+      if (tid == 0) { s_scale = m; *scale = m; }
+    }
+  } else if (tid == 0) {
+    s_scale = *scale;
+  }
+  __syncthreads();
+  const float inv = inv_scale(s_scale);
+  const uint32_t key0 = sr_key(seed, 0u);
+  const int codes = N * HW * Cp;
+  for (int o = tid; o < codes; o += kSmallThreads) {     // o = (n*HW + hw)*Cp + c
+    const int c = o % Cp;
+    const int pix = o / Cp;
+    int code = 0;
+    if (c < C) {
+      const int n = pix / HW, hw = pix - n * HW;
+      const int idx = (n * C + c) * HW + hw;               // NCHW index: the generator's counter
+      const float v = to_f32(x[NHWC_IN ? pix * C + c : idx]);
+      code = stochastic ? quant_stochastic(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key0)))
+                        : quant_nearest(v, inv);
+    }
+    q[o] = (int8_t)code;
+  }
+}
+
 template <typename T>
 dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, int H, int W,
                                   dai8_scale_mode mode, float* scale, dai8_round round,
@@ -1367,6 +1413,16 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
   const int64_t total = npix * C;
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
+  if (npix * Cp <= kSmallTensorElems) {
+    const int am = mode == DAI8_SCALE_ABSMAX ? 1 : 0, sr = round == DAI8_ROUND_STOCHASTIC ? 1 : 0;
+    if (layout == DAI8_NHWC)
+      quantize_small_kernel<T, true><<<1, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+    else
+      quantize_small_kernel<T, false><<<1, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+    note_launch(1);
+    DAI8_RETURN_IF_CUDA(cudaGetLastError());
+    return DAI8_OK;
+  }
   if (mode == DAI8_SCALE_ABSMAX) {
     DAI8_RETURN_IF_CUDA(cudaMemsetAsync(scale, 0, sizeof(float), st));
     uint32_t* bits = reinterpret_cast<uint32_t*>(scale);
