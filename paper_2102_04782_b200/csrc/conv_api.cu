@@ -37,7 +37,11 @@ extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geo
   switch (op) {
     case DAI8_OP_FWD: return 256;
     case DAI8_OP_BWD_DATA: return (wt_bytes(cs) + 255) / 256 * 256 + 256;
-    case DAI8_OP_BWD_FILTER: return (dw_acc_bytes(cs) + 255) / 256 * 256 + 256;
+    case DAI8_OP_BWD_FILTER: {
+      // one int32 image, or one per pixel slice of the tensor-core kernel
+      const int splits = umma_bwd_filter_splits(cs);
+      return (dw_acc_bytes(cs) * (size_t)(splits > 1 ? splits : 1) + 255) / 256 * 256 + 256;
+    }
   }
   return 0;
 }
@@ -105,12 +109,17 @@ extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, 
   const ConvShape cs = make_shape(*geom);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int* acc = static_cast<int*>(ws);
-  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(acc, 0, dw_acc_bytes(cs), st));
   const int mode = g_backend.load();
+  int splits = 1;
   dai8_status r;
-  if (mode != 1 && umma_bwd_filter_supported(cs)) r = umma_bwd_filter_acc(qX, vq, cs, acc, st);
-  else if (mode == 2) return DAI8_ERR_UNSUPPORTED;
-  else r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
+  if (mode != 1 && umma_bwd_filter_supported(cs)) {
+    r = umma_bwd_filter_acc(qX, vq, cs, acc, &splits, st);   // every slice writes its whole image
+  } else if (mode == 2) {
+    return DAI8_ERR_UNSUPPORTED;
+  } else {
+    DAI8_RETURN_IF_CUDA(cudaMemsetAsync(acc, 0, dw_acc_bytes(cs), st));
+    r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
+  }
   if (r != DAI8_OK) return r;
-  return finalize_bwd_filter(acc, sX, s, cs, dW, out_dtype, st);
+  return finalize_bwd_filter(acc, splits, sX, s, cs, dW, out_dtype, st);
 }

@@ -198,20 +198,41 @@ repack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int8_t* __res
 }
 
 __global__ void __launch_bounds__(kThreads)
-finalize_bwd_filter_kernel(const int* __restrict__ acc, const float* __restrict__ sX,
+finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                            const float* __restrict__ s, ConvShape cs, void* __restrict__ dW,
                            dai8_dtype dtype) {
-  const int64_t total = (int64_t)cs.Cout * cs.Cin * cs.R * cs.S;
-  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (t >= total) return;
-  const int ss = (int)(t % cs.S);
-  int64_t m = t / cs.S;
-  const int r = (int)(m % cs.R); m /= cs.R;
-  const int ci = (int)(m % cs.Cin);
-  const int co = (int)(m / cs.Cin);
-  const int a = acc[(((int64_t)co * cs.R + r) * cs.S + ss) * cs.Cinp + ci];
+  // A block sums 32 consecutive accumulators [co][r][s][ci] over the partial images: 8 groups of
+  // 32 threads take every 8th image (coalesced 128-byte reads, several in flight), shared memory
+  // combines the groups in a fixed order.  Integer sums: exact whatever the order.
+  __shared__ int part[8][32];
+  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  const int64_t per_image = (int64_t)cs.Coutp * cs.R * cs.S * cs.Cinp;
+  const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
+  const int64_t e = (int64_t)blockIdx.x * 32 + lane;     // index into one partial image
+  int a = 0;
+  if (e < valid) {
+    const int* src = acc + e;
+    int k = grp;
+    for (; k + 24 < splits; k += 32) {
+      const int v0 = src[(size_t)k * per_image], v1 = src[(size_t)(k + 8) * per_image];
+      const int v2 = src[(size_t)(k + 16) * per_image], v3 = src[(size_t)(k + 24) * per_image];
+      a += v0 + v1 + v2 + v3;
+    }
+    for (; k < splits; k += 8) a += src[(size_t)k * per_image];
+  }
+  part[grp][lane] = a;
+  __syncthreads();
+  if (grp != 0 || e >= valid) return;
+#pragma unroll
+  for (int g = 1; g < 8; ++g) a += part[g][lane];
+  const int ci = (int)(e % cs.Cinp);
+  if (ci >= cs.Cin) return;                                // padding channel
+  int64_t m = e / cs.Cinp;
+  const int ss = (int)(m % cs.S); m /= cs.S;
+  const int r = (int)(m % cs.R);
+  const int co = (int)(m / cs.R);
   const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
-  store_result(dW, dtype, (size_t)t, a, scale);
+  store_result(dW, dtype, (((size_t)co * cs.Cin + ci) * cs.R + r) * cs.S + ss, a, scale);
 }
 
 unsigned blocks_for(int64_t total) { return (unsigned)ceil_div64(total, kThreads); }
@@ -262,10 +283,11 @@ dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int
   return DAI8_OK;
 }
 
-dai8_status finalize_bwd_filter(const int* acc, const float* sX, const float* s, const ConvShape& cs,
-                                void* dW, dai8_dtype dtype, cudaStream_t st) {
-  const int64_t total = (int64_t)cs.Cout * cs.Cin * cs.R * cs.S;
-  finalize_bwd_filter_kernel<<<blocks_for(total), kThreads, 0, st>>>(acc, sX, s, cs, dW, dtype);
+dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, const float* s,
+                                const ConvShape& cs, void* dW, dai8_dtype dtype, cudaStream_t st) {
+  static_assert(kThreads == 256, "the finalize kernel tiles a block as 8 groups of 32 threads");
+  const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
+  finalize_bwd_filter_kernel<<<(unsigned)ceil_div64(valid, 32), kThreads, 0, st>>>(acc, splits, sX, s, cs, dW, dtype);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;

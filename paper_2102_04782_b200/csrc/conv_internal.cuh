@@ -63,9 +63,10 @@ dai8_status direct_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const Conv
 // [Cout][R][S][Cinp] -> [Cinp][R][S][Coutp]; flip != 0 also mirrors the taps (r,s) -> (R-1-r,S-1-s).
 dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int8_t* wT, int flip,
                                       cudaStream_t st);
-// acc[Cout][R][S][Cinp] -> dW (Cout,Cin,R,S), scaled by (sX/127)(s[co]/127) unless dtype is I32.
-dai8_status finalize_bwd_filter(const int* acc, const float* sX, const float* s, const ConvShape& cs,
-                                void* dW, dai8_dtype dtype, cudaStream_t st);
+// sum over `splits` partial images acc[split][Cout][R][S][Cinp] -> dW (Cout,Cin,R,S), scaled by
+// (sX/127)(s[co]/127) unless dtype is I32.
+dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, const float* s,
+                                const ConvShape& cs, void* dW, dai8_dtype dtype, cudaStream_t st);
 
 // ---- tensor-core (tcgen05) kernels: see conv_umma.cu for the geometries covered ------------------
 bool umma_fwd_supported(const ConvShape& cs);
@@ -75,7 +76,10 @@ dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const 
                      const ConvShape& cs, const ConvOut& out, cudaStream_t st);
 dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* gmax, const float* sW,
                           const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+// writes *splits partial images acc[split][Cout][R][S][Cinp] (no zeroing needed), to be added up by
+// finalize_bwd_filter; umma_bwd_filter_splits gives their number for sizing the workspace
 dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc,
-                                cudaStream_t st);
+                                int* splits, cudaStream_t st);
+int umma_bwd_filter_splits(const ConvShape& cs);
 
 }  // namespace dai8

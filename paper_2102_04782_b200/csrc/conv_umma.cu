@@ -716,7 +716,9 @@ IgemmProblem bwd_data_problem(const int8_t* gq, const int8_t* wTflip, const Conv
 // index is contiguous, the contraction index strided): the paper's X -> X', G -> G' dimension
 // transformation is just the major-ness bit of the MMA descriptors, no transposed copy is made.
 // A CTA owns 128 output channels x (a group of taps) x (up to 256 input channels) in tensor memory
-// and a slice of the pixels; slices are combined with integer atomics (exact in any order).
+// and a slice of the pixels.  Every slice writes its own partial image with plain stores and the
+// de-quantizing kernel adds the slices in a fixed order: a hundred-odd CTAs adding into one small
+// image with atomics took longer to drain in L2 than the whole contraction.
 // ---------------------------------------------------------------------------------------------
 constexpr int kKP = 128;  // pixels per pipeline stage (4 MMAs of K = 32)
 
@@ -730,7 +732,8 @@ struct WgradParams {
   int ci_tiles;
   int chunks_total, chunks_per_split;
   int stages, tmem_cols;
-  int* acc;              // [Cout][R*S][Cinp]
+  int* acc;              // [splits][Cout][R*S][Cinp]: one partial image per slice of the pixels
+  size_t acc_stride;     // elements per partial image
 };
 
 __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t saddr, int width_bytes, uint32_t lbo_bytes) {
@@ -849,6 +852,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
     tc_fence_after();
     if (ok) {
       int (*trw)[33] = tr[warp - 2];
+      int* part = prm.acc + (size_t)blockIdx.x * prm.acc_stride;   // this pixel slice's partial sums
       for (int tl = 0; tl < ntap; ++tl) {
         const int tap = tap_begin + tl;
         for (int cg = 0; cg < Nw / 32; ++cg) {
@@ -866,8 +870,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
             for (int rr = 0; rr < 32; ++rr) {
               const int co = co0 + quarter * 32 + rr;
               if (co >= prm.Cout) break;
-              const int val = trw[rr][lane];
-              if (val != 0) atomicAdd(prm.acc + ((size_t)co * T + tap) * prm.Cinp + ci, val);
+              part[((size_t)co * T + tap) * prm.Cinp + ci] = trw[rr][lane];
             }
           }
         }
@@ -895,9 +898,9 @@ bool wgrad_supported(const ConvShape& cs) {
   return true;
 }
 
-dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, cudaStream_t st) {
-  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
-  WgradParams prm;
+// Tiling of the weight gradient: fills everything of `prm` that depends on the geometry only and
+// returns the number of pixel slices (partial images), or 0 if the kernel does not take the shape.
+int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_tiles_out) {
   prm.npix = cs.N * cs.P * cs.Q;
   prm.P = cs.P; prm.Q = cs.Q; prm.Cout = cs.Cout; prm.Cinp = cs.Cinp; prm.R = cs.R; prm.S = cs.S;
   prm.sh = cs.sh; prm.sw = cs.sw; prm.lower_h = -cs.ph; prm.lower_w = -cs.pw;
@@ -916,7 +919,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   int tg_max = 512 / Nw;
   const int tg_smem = (100 * 1024 - kKP * 128) / b_tap_bytes;
   if (tg_max > tg_smem) tg_max = tg_smem;
-  if (tg_max < 1) return DAI8_ERR_UNSUPPORTED;
+  if (tg_max < 1) return 0;
   const int ngroups = (T + tg_max - 1) / tg_max;
   prm.tg = (T + ngroups - 1) / ngroups;
   prm.tmem_cols = 32;
@@ -927,15 +930,31 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   prm.chunks_total = (prm.npix + kKP - 1) / kKP;
   const int co_tiles = (cs.Cout + kBM - 1) / kBM;
   const int tiles = ngroups * prm.ci_tiles * co_tiles;
-  int ksplit = 148 / tiles;
+  int ksplit = sm_count() / tiles;
   if (ksplit < 1) ksplit = 1;
   if (ksplit > prm.chunks_total) ksplit = prm.chunks_total;
   prm.chunks_per_split = (prm.chunks_total + ksplit - 1) / ksplit;
   ksplit = (prm.chunks_total + prm.chunks_per_split - 1) / prm.chunks_per_split;
   if (stages > prm.chunks_per_split) stages = prm.chunks_per_split;
-  if (stages < 1) return DAI8_ERR_UNSUPPORTED;
+  if (stages < 1) return 0;
   prm.stages = stages;
+  prm.acc_stride = (size_t)cs.Coutp * T * cs.Cinp;
+  *ngroups_out = ngroups;
+  *co_tiles_out = co_tiles;
+  return ksplit;
+}
+
+dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, int* splits_out,
+                         cudaStream_t st) {
+  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
+  WgradParams prm;
+  int ngroups = 0, co_tiles = 0;
+  const int ksplit = plan_wgrad(cs, prm, &ngroups, &co_tiles);
+  if (ksplit < 1) return DAI8_ERR_UNSUPPORTED;
   prm.acc = acc;
+  *splits_out = ksplit;
+  const int stages = prm.stages;
+  const int stage_bytes = kKP * 128 + prm.tg * prm.nb * kKP * prm.bw;
 
   CUtensorMap mapG, mapX;
   {
@@ -985,7 +1004,7 @@ bool umma_bwd_data_supported(const ConvShape& cs) {
   return igemm_supported(bwd_data_problem(nullptr, nullptr, cs));
 }
 
-bool umma_bwd_filter_supported(const ConvShape& cs) { return wgrad_supported(cs); }
+bool umma_bwd_filter_supported(const ConvShape& cs) { return umma_bwd_filter_splits(cs) > 0; }
 
 dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW, const ConvShape& cs,
                      const ConvOut& out, cudaStream_t st) {
@@ -997,8 +1016,16 @@ dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* g
   return launch_igemm(bwd_data_problem(gq, wTflip, cs), gmax, sW, out, st);
 }
 
-dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, cudaStream_t st) {
-  return launch_wgrad(qX, vq, cs, acc, st);
+dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, int* splits,
+                                cudaStream_t st) {
+  return launch_wgrad(qX, vq, cs, acc, splits, st);
+}
+
+int umma_bwd_filter_splits(const ConvShape& cs) {
+  if (!wgrad_supported(cs)) return 0;
+  WgradParams prm;
+  int ngroups = 0, co_tiles = 0;
+  return plan_wgrad(cs, prm, &ngroups, &co_tiles);
 }
 
 }  // namespace dai8
