@@ -384,6 +384,91 @@ def run_dai8(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# Per-layer report over one of the network configurations (not the contract line: that is
+# run_dai8 on the conv2_x block).  `python bench.py --layers resnet50|mobilenetv2|vgg16 [--batch N]`
+# prints one JSON object with, per layer, the device time of the gradient quantization and of the
+# three convolutions, and totals as TOPS / GB/s against the measured peaks.
+# ------------------------------------------------------------------------------------------------
+def run_layer_report(args):
+    import torch
+    from paper_2102_04782_b200 import api, synth
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    api.lib()
+    table = {"resnet50": (synth.resnet50_convs, 64), "mobilenetv2": (synth.mobilenetv2_pointwise, 128),
+             "vgg16": (synth.vgg16_convs, 64), "conv2x": (synth.resnet50_conv2x_block, 64)}
+    fn, batch = table[args.layers]
+    N = args.batch or batch
+    peaks = measured_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    bf = torch.bfloat16
+    rows, seen = [], {}
+    tot = {"fwd": [0.0, 0], "bwd_data": [0.0, 0], "bwd_filter": [0.0, 0], "quantize_grad": [0.0, 0]}
+
+    def timed(call, reps=3):
+        best = None
+        for _ in range(reps + 1):
+            flush.zero_()
+            e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(); call(); e1.record(); torch.cuda.synchronize()
+            t = e0.elapsed_time(e1)
+            best = t if best is None else min(best, t)
+        return best
+
+    for L in fn():
+        key = (L.Cin, L.Cout, L.H, L.W, L.R, L.S, L.stride, L.pad)
+        if key not in seen:
+            g = api.ConvGeom(N, L.Cin, L.Cout, L.H, L.W, L.R, L.S, L.stride, L.stride, L.pad, L.pad)
+            Cip, Cop = api.padded_channels(L.Cin), api.padded_channels(L.Cout)
+            qX = torch.randint(-127, 128, (N, L.H, L.W, Cip), dtype=torch.int8, device=dev)
+            qW = torch.randint(-127, 128, (L.Cout, L.R, L.S, Cip), dtype=torch.int8, device=dev)
+            dY = (torch.randn((N, L.P, L.Q, L.Cout), device=dev) * 1e-4).to(bf)
+            vq = torch.empty((N, L.P, L.Q, Cop), dtype=torch.int8, device=dev)
+            gq = torch.empty_like(vq)
+            Y = torch.empty((N, L.P, L.Q, L.Cout), dtype=bf, device=dev)
+            dX = torch.empty((N, L.H, L.W, L.Cin), dtype=bf, device=dev)
+            dW = torch.empty((L.Cout, L.Cin, L.R, L.S), dtype=torch.float32, device=dev)
+            one = torch.ones(1, device=dev); gm = torch.zeros(1, device=dev)
+            s_c = torch.zeros(L.Cout, device=dev)
+            ws_g = torch.empty(api.quantize_grad_workspace_bytes(L.Cout), dtype=torch.uint8, device=dev)
+            ws_d = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_DATA, g)), dtype=torch.uint8, device=dev)
+            ws_w = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_FILTER, g)), dtype=torch.uint8, device=dev)
+            t = {
+                "quantize_grad": timed(lambda: api.quantize_grad(dY, api.NHWC, N, L.Cout, L.P, L.Q, None, s_c, False, gm,
+                                                                 None, None, vq, gq, 1, ws_g)),
+                "fwd": timed(lambda: api.conv_fwd(qX, qW, one, one, g, Y, api.NHWC, None)),
+                "bwd_filter": timed(lambda: api.conv_bwd_filter(qX, vq, one, s_c, g, dW, ws_w)),
+                "bwd_data": timed(lambda: api.conv_bwd_data(gq, qW, gm, one, g, dX, api.NHWC, ws_d)),
+            }
+            npix_o, npix_i = N * L.P * L.Q, N * L.H * L.W
+            seen[key] = (t, 2 * L.macs(N), npix_o * (2 * L.Cout + 2 * Cop))
+            del qX, qW, dY, vq, gq, Y, dX, dW
+        t, ops, gvq_bytes = seen[key]
+        rows.append({"layer": L.name, "shape": f"{L.Cin}->{L.Cout} {L.R}x{L.S}/{L.stride} @{L.H}",
+                     "ms": {k: round(v, 4) for k, v in t.items()},
+                     "tops": {k: round(ops / t[k] / 1e9, 1) for k in ("fwd", "bwd_data", "bwd_filter")},
+                     "gvq_gbs": round(gvq_bytes / t["quantize_grad"] / 1e6, 1)})
+        for k in ("fwd", "bwd_data", "bwd_filter"):
+            tot[k][0] += t[k]; tot[k][1] += ops
+        tot["quantize_grad"][0] += t["quantize_grad"]; tot["quantize_grad"][1] += gvq_bytes
+    assert api.get_device_status() == api.OK
+    int8_peak = INT8_OVER_BF16 * peaks["bf16_burst"]
+    bwd_ms = tot["bwd_data"][0] + tot["bwd_filter"][0]
+    bwd_ops = tot["bwd_data"][1] + tot["bwd_filter"][1]
+    out = {"layers_config": args.layers, "batch": N, "timing": "best of 3 per call, L2 flushed before each call",
+           "totals": {
+               "fwd_ms": round(tot["fwd"][0], 3), "fwd_tops": round(tot["fwd"][1] / tot["fwd"][0] / 1e9, 1),
+               "bwd_ms": round(bwd_ms, 3), "bwd_tops": round(bwd_ops / bwd_ms / 1e9, 1),
+               "bwd_frac_int8_peak": round(bwd_ops / bwd_ms / 1e9 / int8_peak, 4),
+               "gvq_ms": round(tot["quantize_grad"][0], 3),
+               "gvq_gbs": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6, 1),
+               "gvq_frac_hbm": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6 / peaks["hbm_gbs"], 4),
+               "int8_peak_tops": int8_peak, "hbm_peak_gbs": peaks["hbm_gbs"]},
+           "layers": rows}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -391,8 +476,13 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dai8", choices=["dai8", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers", default=None, choices=["conv2x", "resnet50", "mobilenetv2", "vgg16"],
+                    help="print a per-layer report for a network configuration instead of the benchmark line")
+    ap.add_argument("--batch", type=int, default=0)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.layers:
+        run_layer_report(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_dai8(args)
