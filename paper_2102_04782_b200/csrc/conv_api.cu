@@ -83,11 +83,7 @@ extern "C" dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, co
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   int8_t* wT = static_cast<int8_t*>(ws);
   const int mode = g_backend.load();
-  if (mode != 1 && umma_bwd_data_supported(cs)) {
-    dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/1, st);
-    if (r != DAI8_OK) return r;
-    return umma_bwd_data(gq, wT, gmax, sW, cs, out, st);
-  }
+  if (mode != 1 && umma_bwd_data_supported(cs)) return umma_bwd_data(gq, qW, wT, gmax, sW, cs, out, st);
   if (mode == 2) return DAI8_ERR_UNSUPPORTED;
   dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/0, st);
   if (r != DAI8_OK) return r;

@@ -198,6 +198,25 @@ repack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int8_t* __res
 }
 
 __global__ void __launch_bounds__(kThreads)
+repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, DgradClasses dc, int8_t* __restrict__ wT) {
+  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;   // the classes partition the taps
+  int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  int k = 0;
+  while (k + 1 < dc.n && t >= dc.cls[k + 1].w_off) ++k;
+  const DgradClass& c = dc.cls[k];
+  int64_t m = t - c.w_off;
+  const int co = (int)(m % cs.Coutp); m /= cs.Coutp;
+  const int ts = (int)(m % c.Ts); m /= c.Ts;
+  const int tr = (int)(m % c.Tr);
+  const int ci = (int)(m / c.Tr);
+  const int r = c.r0 + cs.sh * (c.Tr - 1 - tr), s = c.s0 + cs.sw * (c.Ts - 1 - ts);   // mirrored order
+  int8_t v = 0;
+  if (co < cs.Cout) v = qW[(((int64_t)co * cs.R + r) * cs.S + s) * cs.Cinp + ci];  // ci >= Cin holds 0
+  wT[t] = v;
+}
+
+__global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                            const float* __restrict__ s, ConvShape cs, void* __restrict__ dW,
                            dai8_dtype dtype) {
@@ -278,6 +297,15 @@ dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int
                                       cudaStream_t st) {
   const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;
   repack_weights_kernel<<<blocks_for(total), kThreads, 0, st>>>(qW, cs, wT, flip);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const DgradClasses& dc, int8_t* wT,
+                                   cudaStream_t st) {
+  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;
+  repack_weights_classes_kernel<<<blocks_for(total), kThreads, 0, st>>>(qW, cs, dc, wT);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;

@@ -39,6 +39,13 @@ __device__ __forceinline__ uint16_t f32_to_bf16_bits(float f) {
   return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);                  // nearest even
 }
 
+// Two fp32 values -> packed bfloat16 pair (lo in bits 0-15), round to nearest even, one instruction.
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
 // Writes one output element: the raw accumulator, or float(acc)*scale as fp32 / bf16.
 __device__ __forceinline__ void store_result(void* out, dai8_dtype dtype, size_t idx, int acc, float scale) {
   if (dtype == DAI8_I32) {
@@ -49,6 +56,19 @@ __device__ __forceinline__ void store_result(void* out, dai8_dtype dtype, size_t
     else static_cast<uint16_t*>(out)[idx] = f32_to_bf16_bits(v);
   }
 }
+
+// Residue classes of the input gradient (see conv_umma.cu): class (a, b) owns the output pixels with
+// h mod stride_h = a, w mod stride_w = b and the filter taps r = r0 + stride_h*j, s = s0 + stride_w*j.
+struct DgradClass {
+  int a, b, r0, s0, Tr, Ts;      // Tr*Ts taps; 0 when the class has none
+  int Ha, Wb;                    // output pixels of the class per image
+  int lower_h, lower_w;          // first q(G) row / column read by output (0, 0) of the class
+  long long w_off;               // offset of the class's weights [Cinp][Tr][Ts][Coutp] in the repacked buffer
+};
+struct DgradClasses {
+  DgradClass cls[16];
+  int n, any_empty;
+};
 
 // ---- direct (CUDA-core, dp4a) kernels: every geometry --------------------------------------------
 dai8_status direct_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
@@ -74,8 +94,12 @@ bool umma_bwd_data_supported(const ConvShape& cs);
 bool umma_bwd_filter_supported(const ConvShape& cs);
 dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
                      const ConvShape& cs, const ConvOut& out, cudaStream_t st);
-dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* gmax, const float* sW,
+// wT: workspace of Cinp*R*S*Coutp bytes for the class-ordered weights
+dai8_status umma_bwd_data(const int8_t* gq, const int8_t* qW, int8_t* wT, const float* gmax, const float* sW,
                           const ConvShape& cs, const ConvOut& out, cudaStream_t st);
+// [Cout][R][S][Cinp] -> for every class [Cinp][Tr][Ts][Coutp] with the class's taps mirrored
+dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const DgradClasses& dc, int8_t* wT,
+                                   cudaStream_t st);
 // writes *splits partial images acc[split][Cout][R][S][Cinp] (no zeroing needed), to be added up by
 // finalize_bwd_filter; umma_bwd_filter_splits gives their number for sizing the workspace
 dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc,

@@ -224,6 +224,9 @@ struct IgemmParams {
   int tma_store;         // NHWC output rows are staged in shared memory and written with tile stores
   int out_elem_bytes;    // 2 (bf16) or 4 (fp32, int32)
   int sh, sw, lower_h, lower_w;  // pixel (p,q) reads input (lower_h + p*sh + r, lower_w + q*sw + s)
+  // tile pixel (img, p, q) is written to pixel (img, oh_off + p*oh_step, ow_off + q*ow_step) of an
+  // oH x oW output image (identity for the forward and stride-1 input-gradient convolutions)
+  int oH, oW, oh_step, oh_off, ow_step, ow_off;
   ConvOut out;
   const float* sa;
   const float* sb;
@@ -380,7 +383,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const int half = (warp - 2) >> 2;
     const bool nhwc = prm.out.layout == DAI8_NHWC;
     const bool vec_ok = nhwc && (prm.Nout & 15) == 0;
-    const size_t plane = (size_t)prm.P * prm.Q;
+    const size_t plane = (size_t)prm.oH * prm.oW;
     const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
     int tile_i = 0, n_store = 0;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++tile_i) {
@@ -395,7 +398,8 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       const int q = m % prm.Q;
       const int tq = m / prm.Q;
       const int p = tq % prm.P, img = tq / prm.P;
-      const size_t pix_base = nhwc ? (size_t)m * prm.Nout : 0;
+      const size_t opix = (size_t)(prm.oh_off + p * prm.oh_step) * prm.oW + (size_t)(prm.ow_off + q * prm.ow_step);   // within the image
+      const size_t pix_base = nhwc ? ((size_t)img * plane + opix) * prm.Nout : 0;
       const uint32_t t_tmem = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * prm.BN);
       if (prm.tma_store) {
         // Rows of this warp's 32 pixels go through a 128-byte-swizzled staging block and leave as one
@@ -424,8 +428,8 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 uint32_t w[8];
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
-                  w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(va[g][2 * i]), scale)) |
-                         ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(va[g][2 * i + 1]), scale)) << 16);
+                  w[i] = pack_bf16x2(__fmul_rn(__int2float_rn(va[g][2 * i]), scale),
+                                     __fmul_rn(__int2float_rn(va[g][2 * i + 1]), scale));
                 const int c0 = sub * 4 + g * 2;
                 *reinterpret_cast<uint4*>(row + (((c0) ^ (lane & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
                 *reinterpret_cast<uint4*>(row + (((c0 + 1) ^ (lane & 7)) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
@@ -481,8 +485,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
               uint32_t w[8];
 #pragma unroll
               for (int i = 0; i < 8; ++i)
-                w[i] = (uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i]), scale)) |
-                       ((uint32_t)f32_to_bf16_bits(__fmul_rn(__int2float_rn(v[2 * i + 1]), scale)) << 16);
+                w[i] = pack_bf16x2(__fmul_rn(__int2float_rn(v[2 * i]), scale), __fmul_rn(__int2float_rn(v[2 * i + 1]), scale));
               uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(prm.out.ptr) + pix_base + j0);
               dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
               dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
@@ -496,7 +499,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
             for (int i = 0; i < 16; ++i) {
               const int j = j0 + i;
               if (j < prm.Nout) {
-                const size_t idx = nhwc ? pix_base + j : ((size_t)img * prm.Nout + j) * plane + (size_t)p * prm.Q + q;
+                const size_t idx = nhwc ? pix_base + j : ((size_t)img * prm.Nout + j) * plane + opix;
                 store_result(prm.out.ptr, prm.out.dtype, idx, v[i], scale);
               }
             }
@@ -574,6 +577,7 @@ struct IgemmProblem {
   const int8_t* B;  // [Brows][R*S][Kc]
   int N, Hi, Wi, Kc, Brows;
   int P, Q, Nout, R, S, sh, sw, lower_h, lower_w;
+  int oH, oW, oh_step, oh_off, ow_step, ow_off;   // output placement, see IgemmParams
 };
 
 bool igemm_supported(const IgemmProblem& pb) {
@@ -625,7 +629,8 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   const int b_res = (total_chunks * b_chunk + 1023) & ~1023;
   const int out_es = out.dtype == DAI8_BF16 ? 2 : 4;
   prm.out_elem_bytes = out_es;
-  prm.tma_store = (out.layout == DAI8_NHWC && (pb.Nout * out_es) % 16 == 0 && pb.Nout * out_es >= 128) ? 1 : 0;
+  const bool identity_place = pb.oH == pb.P && pb.oW == pb.Q && pb.oh_step == 1 && pb.ow_step == 1 && pb.oh_off == 0 && pb.ow_off == 0;
+  prm.tma_store = (identity_place && out.layout == DAI8_NHWC && (pb.Nout * out_es) % 16 == 0 && pb.Nout * out_es >= 128) ? 1 : 0;
   const int stage_out_bytes = prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0;
   prm.b_resident = b_res <= 96 * 1024 ? 1 : 0;
   const int stage_bytes = prm.G * (a_chunk + (prm.b_resident ? 0 : b_chunk));
@@ -634,6 +639,8 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   if (stages < 2) return DAI8_ERR_UNSUPPORTED;
   prm.stages = stages;
   prm.sh = pb.sh; prm.sw = pb.sw; prm.lower_h = pb.lower_h; prm.lower_w = pb.lower_w;
+  prm.oH = pb.oH; prm.oW = pb.oW; prm.oh_step = pb.oh_step; prm.oh_off = pb.oh_off;
+  prm.ow_step = pb.ow_step; prm.ow_off = pb.ow_off;
   prm.out = out; prm.sa = sa; prm.sb = sb;
 
   CUtensorMap mapA, mapB, mapC;
@@ -696,17 +703,52 @@ IgemmProblem fwd_problem(const int8_t* qX, const int8_t* qW, const ConvShape& cs
   pb.N = cs.N; pb.Hi = cs.H; pb.Wi = cs.W; pb.Kc = cs.Cinp; pb.Brows = cs.Cout;
   pb.P = cs.P; pb.Q = cs.Q; pb.Nout = cs.Cout; pb.R = cs.R; pb.S = cs.S;
   pb.sh = cs.sh; pb.sw = cs.sw; pb.lower_h = -cs.ph; pb.lower_w = -cs.pw;
+  pb.oH = cs.P; pb.oW = cs.Q; pb.oh_step = 1; pb.oh_off = 0; pb.ow_step = 1; pb.ow_off = 0;
   return pb;
 }
 
-// Input gradient at stride 1: a forward convolution of q(G) with the mirrored, transposed filter
-// and padding R-1-pad.
-IgemmProblem bwd_data_problem(const int8_t* gq, const int8_t* wTflip, const ConvShape& cs) {
+// Input gradient (Eq. 3) as stride-1 forward convolutions of q(G).  Output pixel (h, w) receives
+// G[p, q] * W[r, s] for h = p*sh + r - ph, w = q*sw + s - pw.  Fixing the residues a = h mod sh,
+// b = w mod sw fixes which taps contribute (r = r0 + sh*j with r0 = (a + ph) mod sh) and makes the
+// rest dense: with h = a + sh*h', row p = h' + e - j, e = (a + ph - r0)/sh.  So each residue class
+// is one implicit GEMM over q(G) with the class's taps in mirrored order, padding lower = e - (Tr-1),
+// written to every sh-th row / sw-th column of dX.  Stride 1 is the single class a = b = 0 (the
+// mirrored filter with padding R-1-pad); at stride 2 a 3x3 filter splits into 1, 2, 2 and 4 taps,
+// so no multiply is spent on inserted zeros.  A class without taps (1x1 filter, stride 2) leaves
+// zeros, written by a memset.
+int plan_dgrad(const ConvShape& cs, DgradClasses& dc) {
+  int n = 0;
+  size_t off = 0;
+  dc.any_empty = 0;
+  for (int a = 0; a < cs.sh; ++a)
+    for (int b = 0; b < cs.sw; ++b) {
+      DgradClass& c = dc.cls[n++];
+      c.a = a; c.b = b;
+      c.r0 = (a + cs.ph) % cs.sh; c.s0 = (b + cs.pw) % cs.sw;
+      c.Tr = c.r0 < cs.R ? (cs.R - c.r0 + cs.sh - 1) / cs.sh : 0;
+      c.Ts = c.s0 < cs.S ? (cs.S - c.s0 + cs.sw - 1) / cs.sw : 0;
+      c.Ha = a < cs.H ? (cs.H - a + cs.sh - 1) / cs.sh : 0;
+      c.Wb = b < cs.W ? (cs.W - b + cs.sw - 1) / cs.sw : 0;
+      c.lower_h = (a + cs.ph - c.r0) / cs.sh - (c.Tr - 1);
+      c.lower_w = (b + cs.pw - c.s0) / cs.sw - (c.Ts - 1);
+      c.w_off = (long long)off;
+      if (c.Tr * c.Ts == 0 || c.Ha * c.Wb == 0) {
+        if (c.Ha * c.Wb != 0) dc.any_empty = 1;
+        c.Tr = c.Ts = 0;
+      }
+      off += (size_t)cs.Cinp * c.Tr * c.Ts * cs.Coutp;
+    }
+  dc.n = n;
+  return n;
+}
+
+IgemmProblem dgrad_class_problem(const int8_t* gq, const int8_t* wT, const ConvShape& cs, const DgradClass& c) {
   IgemmProblem pb;
-  pb.A = gq; pb.B = wTflip;
+  pb.A = gq; pb.B = wT + c.w_off;
   pb.N = cs.N; pb.Hi = cs.P; pb.Wi = cs.Q; pb.Kc = cs.Coutp; pb.Brows = cs.Cinp;
-  pb.P = cs.H; pb.Q = cs.W; pb.Nout = cs.Cin; pb.R = cs.R; pb.S = cs.S;
-  pb.sh = 1; pb.sw = 1; pb.lower_h = -(cs.R - 1 - cs.ph); pb.lower_w = -(cs.S - 1 - cs.pw);
+  pb.P = c.Ha; pb.Q = c.Wb; pb.Nout = cs.Cin; pb.R = c.Tr; pb.S = c.Ts;
+  pb.sh = 1; pb.sw = 1; pb.lower_h = c.lower_h; pb.lower_w = c.lower_w;
+  pb.oH = cs.H; pb.oW = cs.W; pb.oh_step = cs.sh; pb.oh_off = c.a; pb.ow_step = cs.sw; pb.ow_off = c.b;
   return pb;
 }
 
@@ -999,9 +1041,12 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
 bool umma_fwd_supported(const ConvShape& cs) { return igemm_supported(fwd_problem(nullptr, nullptr, cs)); }
 
 bool umma_bwd_data_supported(const ConvShape& cs) {
-  if (cs.sh != 1 || cs.sw != 1) return false;
-  if (cs.ph > cs.R - 1 || cs.pw > cs.S - 1) return false;
-  return igemm_supported(bwd_data_problem(nullptr, nullptr, cs));
+  if (cs.sh > 4 || cs.sw > 4) return false;
+  DgradClasses dc;
+  plan_dgrad(cs, dc);
+  for (int i = 0; i < dc.n; ++i)
+    if (dc.cls[i].Tr > 0 && !igemm_supported(dgrad_class_problem(nullptr, nullptr, cs, dc.cls[i]))) return false;
+  return true;
 }
 
 bool umma_bwd_filter_supported(const ConvShape& cs) { return umma_bwd_filter_splits(cs) > 0; }
@@ -1011,9 +1056,22 @@ dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const 
   return launch_igemm(fwd_problem(qX, qW, cs), sX, sW, out, st);
 }
 
-dai8_status umma_bwd_data(const int8_t* gq, const int8_t* wTflip, const float* gmax, const float* sW,
+dai8_status umma_bwd_data(const int8_t* gq, const int8_t* qW, int8_t* wT, const float* gmax, const float* sW,
                           const ConvShape& cs, const ConvOut& out, cudaStream_t st) {
-  return launch_igemm(bwd_data_problem(gq, wTflip, cs), gmax, sW, out, st);
+  DgradClasses dc;
+  plan_dgrad(cs, dc);
+  if (dc.any_empty) {   // positions no tap reaches
+    const size_t es = out.dtype == DAI8_BF16 ? 2 : 4;
+    DAI8_RETURN_IF_CUDA(cudaMemsetAsync(out.ptr, 0, (size_t)cs.N * cs.H * cs.W * cs.Cin * es, st));
+  }
+  dai8_status r = repack_weights_classes(qW, cs, dc, wT, st);
+  if (r != DAI8_OK) return r;
+  for (int i = 0; i < dc.n; ++i) {
+    if (dc.cls[i].Tr == 0) continue;
+    r = launch_igemm(dgrad_class_problem(gq, wT, cs, dc.cls[i]), gmax, sW, out, st);
+    if (r != DAI8_OK) return r;
+  }
+  return DAI8_OK;
 }
 
 dai8_status umma_bwd_filter_acc(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, int* splits,

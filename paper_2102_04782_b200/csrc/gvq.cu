@@ -1358,8 +1358,9 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   return DAI8_OK;
 }
 
-// Small tensors (weights): one CTA finds max|x| and writes the codes, so the call is a single
-// launch instead of memset + reduction + quantization.
+// Small tensors (weights): a single launch instead of memset + reduction + quantization.  Every CTA
+// finds max|x| of the whole tensor for itself (it is small and sits in L2), so no CTA waits for
+// another, and writes its share of the codes.
 constexpr int kSmallThreads = 1024;
 constexpr int64_t kSmallTensorElems = 131072;
 
@@ -1373,6 +1374,7 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
   const int total = N * C * HW;
   if (absmax_mode) {
     float m = 0.f;
+#pragma unroll 4
     for (int i = tid; i < total; i += kSmallThreads) m = fmaxf(m, fabsf(to_f32(x[i])));
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if ((tid & 31) == 0) s_part[tid >> 5] = m;
@@ -1380,7 +1382,7 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
     if (tid < 32) {
       m = s_part[tid];
       for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-      if (tid == 0) { s_scale = m; *scale = m; }
+      if (tid == 0) { s_scale = m; if (blockIdx.x == 0) *scale = m; }
     }
   } else if (tid == 0) {
     s_scale = *scale;
@@ -1389,7 +1391,7 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
   const float inv = inv_scale(s_scale);
   const uint32_t key0 = sr_key(seed, 0u);
   const int codes = N * HW * Cp;
-  for (int o = tid; o < codes; o += kSmallThreads) {     // o = (n*HW + hw)*Cp + c
+  for (int o = blockIdx.x * kSmallThreads + tid; o < codes; o += gridDim.x * kSmallThreads) {   // o = (n*HW + hw)*Cp + c
     const int c = o % Cp;
     const int pix = o / Cp;
     int code = 0;
@@ -1415,10 +1417,12 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
   constexpr int VEfull = vec_elems<T>();
   if (npix * Cp <= kSmallTensorElems) {
     const int am = mode == DAI8_SCALE_ABSMAX ? 1 : 0, sr = round == DAI8_ROUND_STOCHASTIC ? 1 : 0;
+    int small_ctas = (int)ceil_div64(npix * Cp, 4 * kSmallThreads);
+    if (small_ctas > 32) small_ctas = 32;
     if (layout == DAI8_NHWC)
-      quantize_small_kernel<T, true><<<1, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+      quantize_small_kernel<T, true><<<small_ctas, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
     else
-      quantize_small_kernel<T, false><<<1, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+      quantize_small_kernel<T, false><<<small_ctas, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
     note_launch(1);
     DAI8_RETURN_IF_CUDA(cudaGetLastError());
     return DAI8_OK;
