@@ -432,12 +432,13 @@ def run_layer_report(args):
             one = torch.ones(1, device=dev); gm = torch.zeros(1, device=dev)
             s_c = torch.zeros(L.Cout, device=dev)
             ws_g = torch.empty(api.quantize_grad_workspace_bytes(L.Cout), dtype=torch.uint8, device=dev)
+            ws_f = torch.empty(max(16, api.conv_workspace_bytes(api.OP_FWD, g)), dtype=torch.uint8, device=dev)
             ws_d = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_DATA, g)), dtype=torch.uint8, device=dev)
             ws_w = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_FILTER, g)), dtype=torch.uint8, device=dev)
             t = {
                 "quantize_grad": timed(lambda: api.quantize_grad(dY, api.NHWC, N, L.Cout, L.P, L.Q, None, s_c, False, gm,
                                                                  None, None, vq, gq, 1, ws_g)),
-                "fwd": timed(lambda: api.conv_fwd(qX, qW, one, one, g, Y, api.NHWC, None)),
+                "fwd": timed(lambda: api.conv_fwd(qX, qW, one, one, g, Y, api.NHWC, ws_f)),
                 "bwd_filter": timed(lambda: api.conv_bwd_filter(qX, vq, one, s_c, g, dW, ws_w)),
                 "bwd_data": timed(lambda: api.conv_bwd_data(gq, qW, gm, one, g, dX, api.NHWC, ws_d)),
             }

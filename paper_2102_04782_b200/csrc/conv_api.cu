@@ -23,6 +23,24 @@ bool bad_layout(dai8_layout l) { return l != DAI8_NCHW && l != DAI8_NHWC; }
 
 size_t wt_bytes(const ConvShape& cs) { return (size_t)cs.Cinp * cs.R * cs.S * cs.Coutp; }
 size_t dw_acc_bytes(const ConvShape& cs) { return (size_t)cs.Coutp * cs.R * cs.S * cs.Cinp * sizeof(int); }
+size_t up256(size_t b) { return (b + 255) / 256 * 256; }
+
+// Packed pointwise form of a layer with at most 16 input channels, if the tensor-core kernels take it.
+int packed_fwd(const ConvShape& cs, ConvShape* pw) {
+  ConvShape tmp;
+  const int Kp = packed_small_cin(cs, &tmp);
+  if (Kp == 0 || !umma_fwd_supported(tmp)) return 0;
+  if (pw) *pw = tmp;
+  return Kp;
+}
+int packed_bwd_filter(const ConvShape& cs, ConvShape* pw) {
+  ConvShape tmp;
+  const int Kp = packed_small_cin(cs, &tmp);
+  if (Kp == 0 || !umma_bwd_filter_supported(tmp)) return 0;
+  if (pw) *pw = tmp;
+  return Kp;
+}
+size_t packed_a_bytes(const ConvShape& cs, int Kp) { return up256((size_t)cs.N * cs.P * cs.Q * Kp); }
 
 }  // namespace
 }  // namespace dai8
@@ -35,10 +53,16 @@ extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geo
   if (check_geom(geom) != DAI8_OK) return 0;
   const ConvShape cs = make_shape(*geom);
   switch (op) {
-    case DAI8_OP_FWD: return 256;
+    case DAI8_OP_FWD: {
+      const int Kp = umma_fwd_supported(cs) ? 0 : packed_fwd(cs, nullptr);
+      return Kp ? packed_a_bytes(cs, Kp) + up256((size_t)cs.Coutp * Kp) + 256 : 256;
+    }
     case DAI8_OP_BWD_DATA: return (wt_bytes(cs) + 255) / 256 * 256 + 256;
     case DAI8_OP_BWD_FILTER: {
       // one int32 image, or one per pixel slice of the tensor-core kernel
+      ConvShape pw;
+      const int Kp = umma_bwd_filter_supported(cs) ? 0 : packed_bwd_filter(cs, &pw);
+      if (Kp) return up256(dw_acc_bytes(pw) * (size_t)umma_bwd_filter_splits(pw)) + packed_a_bytes(cs, Kp) + 256;
       const int splits = umma_bwd_filter_splits(cs);
       return (dw_acc_bytes(cs) * (size_t)(splits > 1 ? splits : 1) + 255) / 256 * 256 + 256;
     }
@@ -49,7 +73,6 @@ extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geo
 extern "C" dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
                                      const dai8_conv_geom* geom, void* Y, dai8_dtype out_dtype,
                                      dai8_layout out_layout, void* ws, size_t ws_bytes, void* stream) {
-  (void)ws; (void)ws_bytes;
   dai8_status g = check_geom(geom);
   if (g != DAI8_OK) return g;
   if (!qX || !qW || !Y || bad_out(out_dtype) || bad_layout(out_layout)) return DAI8_ERR_INVALID_ARG;
@@ -62,7 +85,18 @@ extern "C" dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const f
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const int mode = g_backend.load();
   if (mode != 1 && umma_fwd_supported(cs)) return umma_fwd(qX, qW, sX, sW, cs, out, st);
-  if (mode == 2) return DAI8_ERR_UNSUPPORTED;
+  ConvShape pw;
+  const int Kp = mode != 1 ? packed_fwd(cs, &pw) : 0;
+  if (Kp && ws && aligned16(ws) && ws_bytes >= dai8_conv_workspace_bytes(DAI8_OP_FWD, geom)) {
+    // few input channels: gather the real channels of all taps, then a pointwise convolution
+    int8_t* A = static_cast<int8_t*>(ws);
+    int8_t* Wp = A + packed_a_bytes(cs, Kp);
+    dai8_status r = pack_small_cin(qX, cs, Kp, A, st);
+    if (r == DAI8_OK) r = pack_small_cin_weights(qW, cs, Kp, Wp, st);
+    if (r != DAI8_OK) return r;
+    return umma_fwd(A, Wp, sX, sW, pw, out, st);
+  }
+  if (mode == 2) return Kp ? DAI8_ERR_WORKSPACE : DAI8_ERR_UNSUPPORTED;
   return direct_fwd(qX, qW, sX, sW, cs, out, st);
 }
 
@@ -108,8 +142,16 @@ extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, 
   const int mode = g_backend.load();
   int splits = 1;
   dai8_status r;
+  ConvShape pw;
   if (mode != 1 && umma_bwd_filter_supported(cs)) {
     r = umma_bwd_filter_acc(qX, vq, cs, acc, &splits, st);   // every slice writes its whole image
+  } else if (const int Kp = mode != 1 ? packed_bwd_filter(cs, &pw) : 0) {
+    // few input channels: the weight gradient of the packed pointwise form, unpacked by finalize
+    int8_t* A = static_cast<int8_t*>(ws) + up256(dw_acc_bytes(pw) * (size_t)umma_bwd_filter_splits(pw));
+    r = pack_small_cin(qX, cs, Kp, A, st);
+    if (r == DAI8_OK) r = umma_bwd_filter_acc(A, vq, pw, acc, &splits, st);
+    if (r != DAI8_OK) return r;
+    return finalize_bwd_filter(acc, splits, sX, s, pw, &cs, dW, out_dtype, st);
   } else if (mode == 2) {
     return DAI8_ERR_UNSUPPORTED;
   } else {
@@ -117,5 +159,5 @@ extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, 
     r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
   }
   if (r != DAI8_OK) return r;
-  return finalize_bwd_filter(acc, splits, sX, s, cs, dW, out_dtype, st);
+  return finalize_bwd_filter(acc, splits, sX, s, cs, nullptr, dW, out_dtype, st);
 }

@@ -197,6 +197,55 @@ repack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int8_t* __res
   wT[t] = v;
 }
 
+// Layers with at most 16 input channels (network stems) would leave the tensor core's K = 32
+// mostly empty.  Their activations are gathered once into a matrix A'[pixel][k'], k' = (r*S+s)*Cin + ci
+// over the REAL channels, padded with zeros to Kp (a multiple of 32); forward and weight-gradient
+// convolutions then run as pointwise convolutions with Kp input channels on the tensor-core kernels.
+__global__ void __launch_bounds__(kThreads)
+pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* __restrict__ A) {
+  const int groups = Kp / 16;                                   // 16-byte groups per pixel row of A'
+  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * groups;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int kg = (int)(t % groups);
+  int64_t m = t / groups;
+  const int q = (int)(m % cs.Q); m /= cs.Q;
+  const int p = (int)(m % cs.P);
+  const int n = (int)(m / cs.P);
+  const int Kreal = cs.R * cs.S * cs.Cin;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+  int k = kg * 16;
+  int tap = k / cs.Cin, ci = k - tap * cs.Cin;
+  int r = tap / cs.S, s = tap - r * cs.S;
+#pragma unroll
+  for (int j = 0; j < 16; ++j, ++k) {
+    if (k < Kreal) {
+      const int h = p * cs.sh + r - cs.ph, x = q * cs.sw + s - cs.pw;
+      if (h >= 0 && h < cs.H && x >= 0 && x < cs.W) {
+        const uint32_t v = (uint8_t)qX[(((int64_t)n * cs.H + h) * cs.W + x) * cs.Cinp + ci];
+        w[j >> 2] |= v << (8 * (j & 3));
+      }
+      if (++ci == cs.Cin) { ci = 0; if (++s == cs.S) { s = 0; ++r; } }
+    }
+  }
+  reinterpret_cast<uint4*>(A)[t] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// [Cout][R][S][Cinp] -> [Cout][Kp] in the same k' order.
+__global__ void __launch_bounds__(kThreads)
+pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t* __restrict__ Wp) {
+  const int64_t total = (int64_t)cs.Cout * Kp;
+  const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
+  if (t >= total) return;
+  const int k = (int)(t % Kp), co = (int)(t / Kp);
+  int8_t v = 0;
+  if (k < cs.R * cs.S * cs.Cin) {
+    const int tap = k / cs.Cin, ci = k - tap * cs.Cin;
+    v = qW[((int64_t)co * cs.R * cs.S + tap) * cs.Cinp + ci];
+  }
+  Wp[t] = v;
+}
+
 __global__ void __launch_bounds__(kThreads)
 repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, DgradClasses dc, int8_t* __restrict__ wT) {
   const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;   // the classes partition the taps
@@ -218,8 +267,8 @@ repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, Dgrad
 
 __global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
-                           const float* __restrict__ s, ConvShape cs, void* __restrict__ dW,
-                           dai8_dtype dtype) {
+                           const float* __restrict__ s, ConvShape cs, int pack_cin, int pack_R, int pack_S,
+                           void* __restrict__ dW, dai8_dtype dtype) {
   // A block sums 32 consecutive accumulators [co][r][s][ci] over the partial images: 8 groups of
   // 32 threads take every 8th image (coalesced 128-byte reads, several in flight), shared memory
   // combines the groups in a fixed order.  Integer sums: exact whatever the order.
@@ -244,14 +293,23 @@ finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float*
   if (grp != 0 || e >= valid) return;
 #pragma unroll
   for (int g = 1; g < 8; ++g) a += part[g][lane];
-  const int ci = (int)(e % cs.Cinp);
+  int ci = (int)(e % cs.Cinp);
   if (ci >= cs.Cin) return;                                // padding channel
   int64_t m = e / cs.Cinp;
-  const int ss = (int)(m % cs.S); m /= cs.S;
-  const int r = (int)(m % cs.R);
+  int ss = (int)(m % cs.S); m /= cs.S;
+  int r = (int)(m % cs.R);
   const int co = (int)(m / cs.R);
+  int Cin = cs.Cin, R = cs.R, S = cs.S;
+  if (pack_cin > 0) {
+    // the images come from the packed pointwise form: `ci` is k' = (r*S + s)*Cin + ci of the real filter
+    const int k = ci;
+    if (k >= pack_R * pack_S * pack_cin) return;
+    const int tap = k / pack_cin;
+    ci = k - tap * pack_cin; r = tap / pack_S; ss = tap - r * pack_S;
+    Cin = pack_cin; R = pack_R; S = pack_S;
+  }
   const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
-  store_result(dW, dtype, (((size_t)co * cs.Cin + ci) * cs.R + r) * cs.S + ss, a, scale);
+  store_result(dW, dtype, (((size_t)co * Cin + ci) * R + r) * S + ss, a, scale);
 }
 
 unsigned blocks_for(int64_t total) { return (unsigned)ceil_div64(total, kThreads); }
@@ -311,11 +369,28 @@ dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const 
   return DAI8_OK;
 }
 
+dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st) {
+  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
+  pack_im2col_kernel<<<blocks_for(total), kThreads, 0, st>>>(qX, cs, Kp, A);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
+dai8_status pack_small_cin_weights(const int8_t* qW, const ConvShape& cs, int Kp, int8_t* Wp, cudaStream_t st) {
+  pack_weights_kernel<<<blocks_for((int64_t)cs.Cout * Kp), kThreads, 0, st>>>(qW, cs, Kp, Wp);
+  note_launch();
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+
 dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, const float* s,
-                                const ConvShape& cs, void* dW, dai8_dtype dtype, cudaStream_t st) {
+                                const ConvShape& cs, const ConvShape* packed_from, void* dW, dai8_dtype dtype,
+                                cudaStream_t st) {
   static_assert(kThreads == 256, "the finalize kernel tiles a block as 8 groups of 32 threads");
   const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
-  finalize_bwd_filter_kernel<<<(unsigned)ceil_div64(valid, 32), kThreads, 0, st>>>(acc, splits, sX, s, cs, dW, dtype);
+  const int pc = packed_from ? packed_from->Cin : 0, pr = packed_from ? packed_from->R : 0, ps = packed_from ? packed_from->S : 0;
+  finalize_bwd_filter_kernel<<<(unsigned)ceil_div64(valid, 32), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;

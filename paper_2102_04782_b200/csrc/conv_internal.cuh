@@ -85,8 +85,28 @@ dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int
                                       cudaStream_t st);
 // sum over `splits` partial images acc[split][Cout][R][S][Cinp] -> dW (Cout,Cin,R,S), scaled by
 // (sX/127)(s[co]/127) unless dtype is I32.
+// With packed_from != nullptr, `cs` is the pointwise form of the layer *packed_from (see
+// packed_small_cin) and channel k' of the images is element (ci, r, s) of the real filter.
 dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, const float* s,
-                                const ConvShape& cs, void* dW, dai8_dtype dtype, cudaStream_t st);
+                                const ConvShape& cs, const ConvShape* packed_from, void* dW, dai8_dtype dtype,
+                                cudaStream_t st);
+
+// Layers with at most 16 input channels: A'[N*P*Q][Kp] gathers the real channels of all taps
+// (k' = (r*S+s)*Cin + ci, zero padded to Kp = multiple of 32), W'[Cout][Kp] likewise; the layer then
+// is a pointwise convolution with Kp input channels.
+inline int packed_small_cin(const ConvShape& cs, ConvShape* pw) {
+  if (cs.Cinp != 16) return 0;
+  const int Kp = round_up(cs.R * cs.S * cs.Cin, 32);
+  if (Kp > 2048) return 0;
+  if (pw) {
+    *pw = cs;
+    pw->Cin = Kp; pw->Cinp = Kp; pw->H = cs.P; pw->W = cs.Q; pw->R = 1; pw->S = 1;
+    pw->sh = 1; pw->sw = 1; pw->ph = 0; pw->pw = 0;
+  }
+  return Kp;
+}
+dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st);
+dai8_status pack_small_cin_weights(const int8_t* qW, const ConvShape& cs, int Kp, int8_t* Wp, cudaStream_t st);
 
 // ---- tensor-core (tcgen05) kernels: see conv_umma.cu for the geometries covered ------------------
 bool umma_fwd_supported(const ConvShape& cs);

@@ -58,7 +58,7 @@ def test_network_layer_convolutions(key):
     dW = torch.empty((Cout, Cin, R, S), dtype=torch.int32, device="cuda")
     dqX, dqW, dqG = codes_from_nchw(qX), weights_dev(qW), codes_from_nchw(qG)
     one = scalar(1.0)
-    api.conv_fwd(dqX, dqW, one, one, gg, Y, api.NHWC, None)
+    api.conv_fwd(dqX, dqW, one, one, gg, Y, api.NHWC, ws_bytes(api.conv_workspace_bytes(api.OP_FWD, gg)))
     api.conv_bwd_data(dqG, dqW, one, one, gg, dX, api.NHWC, ws_bytes(api.conv_workspace_bytes(api.OP_BWD_DATA, gg)))
     api.conv_bwd_filter(dqX, dqG, one, torch.ones(Cout, device="cuda"), gg, dW,
                         ws_bytes(api.conv_workspace_bytes(api.OP_BWD_FILTER, gg)))
