@@ -113,6 +113,26 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# Multi-GPU: replicas only.  Every rank runs the whole workload on its own GPU; the only exchange
+# is the timing itself (max over ranks) and rank 0 prints the aggregate.  These two helpers hold
+# that logic so that it can be exercised with the gloo backend on CPU.
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(ms, dist=None, device="cpu"):
+    """Slowest rank's time in milliseconds (the job is as slow as its slowest replica)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_value(ops_per_step_per_rank, ms_per_step, world):
+    """Whole-job TOPS of `world` replicas that each do ops_per_step_per_rank in ms_per_step."""
+    return world * ops_per_step_per_rank / (ms_per_step * 1e-3) / 1e12
+
+
+# ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
 class LayerBuffers:
@@ -259,12 +279,8 @@ def run_dai8(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    def max_over_ranks(ms):
-        if dist is None:
-            return ms
-        t = torch.tensor([ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    def max_ranks(ms):
+        return max_over_ranks(ms, dist, dev)
 
     for _ in range(max(args.warmup, 3)):
         step()
@@ -281,13 +297,13 @@ def run_dai8(args):
         step(records)
     t1.record()
     barrier()
-    total_ms = max_over_ranks(t0.elapsed_time(t1))
+    total_ms = max_ranks(t0.elapsed_time(t1))
     launches = api.launch_count() - launches0
     clocks = sampler.stop() if sampler else None
     assert api.get_device_status() == api.OK
     ms_per_step = total_ms / args.steps
     ops_step = bwd_ops(layers, BATCH)
-    value = world * ops_step / (ms_per_step * 1e-3) / 1e12
+    value = aggregate_value(ops_step, ms_per_step, world)
 
     # ---- end to end: pinned host inputs -> device, results -> pinned host, every step ------------
     def e2e_step():
@@ -307,8 +323,8 @@ def run_dai8(args):
         e2e_step()
     e1.record()
     barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / e2e_steps
-    e2e_value = world * ops_step / (e2e_ms * 1e-3) / 1e12
+    e2e_ms = max_ranks(e0.elapsed_time(e1)) / e2e_steps
+    e2e_value = aggregate_value(ops_step, e2e_ms, world)
 
     if rank != 0:
         if dist is not None:
