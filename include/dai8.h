@@ -110,7 +110,11 @@ dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout la
  *              taken as |g|max,c), out s_{c,t} -- the per-channel clip values used for `vq`
  *   gmax_layer device [1], out: |g|max of the layer, the scale of `gq`
  *   stats      device [C][4] or NULL, out: |g|max,c, mean, sigma, P = #{|g|>sigma}/M
- *   cls        device [C] or NULL, out: 1 = bell-shaped (P > lambda), 0 = Inverted-T
+ *   cls        device [C] or NULL, out: 1 = bell-shaped (P > lambda), 0 = Inverted-T.  When has_prev
+ *              != 0 its previous contents are read as a hint (the classes of the last iteration):
+ *              the fused kernel writes the codes while it counts, with the clip value of the hinted
+ *              class, and redoes only the channels whose class turned out different.  The hint
+ *              affects speed only, never a result.
  *   vq         out, int8 [N][H][W][Cp]: per-channel codes (for dai8_conv_bwd_filter)
  *   gq         out or NULL, int8 [N][H][W][Cp]: layer-wide codes (for dai8_conv_bwd_data)
  *   seed       stochastic-rounding seed; vq uses stream 0, gq stream 1 of the generator

@@ -14,6 +14,7 @@
 // (4 fp32 / 8 bf16) of one pixel and walks down the pixels, so per-channel scalars stay in
 // registers and every load/store instruction of a warp covers contiguous memory.  NCHW inputs are
 // read along H*W per (n, c) row and transposed through shared memory when codes are written.
+#include <cmath>
 #include <mutex>
 #include <type_traits>
 
@@ -537,19 +538,23 @@ absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_
 }
 
 // ------------------------------------------------------------------------------------------------
-// Fused NHWC path: the three sweeps in ONE persistent cooperative kernel, one CTA per SM.
+// Fused NHWC path: statistics, density count, clip update and both code tensors in ONE persistent
+// cooperative kernel, one CTA per SM, in two sweeps over dY (plus a rare partial third).
 //
 // A CTA owns a contiguous range of pixels, i.e. a contiguous byte range of dY.  One producer warp
 // streams that range into shared memory with bulk asynchronous copies (cp.async.bulk, completion on
 // mbarriers) in pieces of up to 16 KB; sixteen consumer warps work on the pieces.  As many pieces as
-// fit stay resident for all three phases, the rest cycles through a small ring and is fetched again
-// in the later phases (L2 hits for tensors of up to ~100 MB).  The producer runs ahead across phase
-// boundaries, so the first pieces of the next phase are already in flight while the CTAs meet at a
+// fit stay resident for all sweeps, the rest cycles through a small ring and is fetched again in the
+// later sweeps (L2 hits for tensors of up to ~100 MB).  The producer runs ahead across sweep
+// boundaries, so the first pieces of the next sweep are already in flight while the CTAs meet at a
 // grid barrier.
 //
-// Between phase 1 and 2 the per-CTA partial moments are combined once: channel c is finished by one
-// warp of CTA c mod gridDim.x (fixed order, hence deterministic), and after a second barrier every
-// CTA reads the finished |g|max and sigma.  The density counts are integer atomics.
+// Sweep 1 takes the statistics.  The per-CTA partial moments are combined once: channel c is
+// finished by one warp of CTA c mod gridDim.x (fixed order, hence deterministic), and after a second
+// barrier every CTA reads the finished |g|max and sigma.  Sweep 2 takes the density count (integer
+// atomics) AND writes the codes, with the clip value of the class it predicts for each channel; the
+// class that the count then yields is the one reported and the one the codes must match, so channels
+// with a wrong prediction are re-quantized in a fix-up sweep that only their threads take part in.
 //
 // Two things bound this kernel, and neither is HBM.  (1) Instruction issue in phase 3: two
 // stochastic roundings per element, each with its own hash-derived uniform.  So bf16 inputs take
@@ -651,6 +656,7 @@ __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;"
 struct FusedArgs {
   int64_t npix, HW;
   double inv_M, inv_denom; // 1/M and 1/(M or M-1), from the host
+  float pred_ratio;        // a channel is predicted bell-shaped when |g|max < pred_ratio * sigma
   int C, Cp, G, Gp;        // G input vector columns, Gp output vector columns (>= G, zero padding)
   int rows_per_warp, rpi;  // thread tiling, see fused_map
   int rp;                  // pixel rows per piece (a multiple of rpi)
@@ -792,6 +798,8 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   __shared__ uint64_t full_bar[kMaxSlots], empty_bar[kMaxRing];
   __shared__ volatile uint32_t s_abort;
   __shared__ uint32_t s_ok;
+  __shared__ volatile uint32_t s_fix;        // 0 undecided, 1 no fix-up pass, 2 fix-up pass
+  __shared__ uint32_t s_any_mis;
 
   double* red_sum = reinterpret_cast<double*>(fsmem);                    // [VE][kFT]
   double* red_ss = red_sum + (size_t)VE * kFT;                           // [VE][kFT]
@@ -801,7 +809,8 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   float* ch_sigma = ch_absmax + a.C + 1;                                 // [C]
   float* ch_sprev = ch_sigma + a.C;                                      // [C]
   float* ch_inv = ch_sprev + a.C;                                        // [C + 1], last = layer scale
-  uint8_t* pieces = fsmem + ((fused_red_bytes(VE) + (size_t)a.C * 16 + 8 + 127) / 128) * 128;
+  uint8_t* ch_pred = reinterpret_cast<uint8_t*>(ch_inv + a.C + 1);       // [C] predicted class; 2 = mispredicted
+  uint8_t* pieces = fsmem + ((fused_red_bytes(VE) + (size_t)a.C * 17 + 8 + 127) / 128) * 128;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int C = a.C, Gp = a.Gp, G = a.G;
@@ -818,7 +827,7 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   const int NS = K - R;                              // pieces streamed again in every phase
 
   if (tid == 0) {
-    s_abort = 0u;
+    s_abort = 0u; s_fix = 0u; s_any_mis = 0u;
 #pragma unroll 1
     for (int s = 0; s < kMaxSlots; ++s) mbar_init(&full_bar[s], 1);
 #pragma unroll 1
@@ -831,21 +840,32 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   if (warp == kFT / 32) {
     if (lane == 0) {
       const uint8_t* src = reinterpret_cast<const uint8_t*>(x) + (size_t)p0 * rb;
-      // resident pieces once, then three passes (phase 1, 2, 3) over the streamed ones
-      const int items = R + 3 * NS;
+      // resident pieces once, then one pass over the streamed ones per sweep: statistics, the
+      // count + quantize sweep, and -- only if a channel's class was mispredicted -- the fix-up sweep
       int k = 0;
+      auto issue = [&](int begin, int end) {
 #pragma unroll 1
-      for (int i = 0; i < items; ++i) {
-        int slot = i;
-        if (i >= R) {
-          const int t = i - R, r = t & (ring - 1);
-          slot = R + r;
-          if (t >= ring && !mbar_wait(&empty_bar[r], (uint32_t)((t >> a.ring_log2) - 1) & 1u, &s_abort, a.status)) break;
+        for (int i = begin; i < end; ++i) {
+          int slot = i;
+          if (i >= R) {
+            const int t = i - R, r = t & (ring - 1);
+            slot = R + r;
+            if (t >= ring && !mbar_wait(&empty_bar[r], (uint32_t)((t >> a.ring_log2) - 1) & 1u, &s_abort, a.status)) return false;
+          }
+          const uint32_t bytes = (uint32_t)min(rp, rows_total - k * rp) * (uint32_t)rb;
+          mbar_expect_tx(&full_bar[slot], bytes);
+          bulk_load(pieces + (size_t)slot * piece_stride, src + (size_t)k * piece_stride, bytes, &full_bar[slot]);
+          if (++k == K) k = R;
         }
-        const uint32_t bytes = (uint32_t)min(rp, rows_total - k * rp) * (uint32_t)rb;
-        mbar_expect_tx(&full_bar[slot], bytes);
-        bulk_load(pieces + (size_t)slot * piece_stride, src + (size_t)k * piece_stride, bytes, &full_bar[slot]);
-        if (++k == K) k = R;
+        return true;
+      };
+      if (issue(0, R + 2 * NS) && NS > 0) {
+        const long long t0 = clock64();
+        while (s_fix == 0u && !s_abort) {          // the consumers decide after the third grid barrier
+          if (clock64() - t0 > kWaitTimeoutCycles) { s_abort = 1u; atomicExch(a.status, (unsigned int)DAI8_ERR_TIMEOUT); }
+          __nanosleep(200);
+        }
+        if (s_fix == 2u && !s_abort) issue(R + 2 * NS, R + 3 * NS);
       }
     }
     return;
@@ -1007,166 +1027,140 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     }
   }
   ok = grid_barrier(a.gridbar, 2u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
-  if (ok) {
-#pragma unroll 1
-    for (int c = tid; c < C; c += kFT) {
-      ch_absmax[c] = __ldcg(a.ws.absmax + c);
-      ch_sigma[c] = a.sigma_override ? a.sigma_override[c] : __ldcg(a.ws.sigma + c);
-    }
-    if (tid == 0) ch_absmax[C] = __uint_as_float(__ldcg(a.ws.gmax_bits));
-    consumer_sync();
-  }
 
-  // ---------------- phase 2: density count -----------------------------------------------------
+  // Every CTA now holds |g|max and sigma of every channel.  The class (Eq. 15) needs one more
+  // sweep for the density count, the codes another one; to save a sweep the class is PREDICTED --
+  // from the caller's classes of the previous iteration if given, else from |g|max / sigma, which
+  // is about sqrt(2 ln M) for a bell-shaped and ln(M)/sqrt(2) for a long-tailed channel -- and the
+  // codes are written with the clip value of the predicted class while the count is taken.  After
+  // the count the true class is known; channels whose prediction was wrong (rare) get their
+  // per-channel codes rewritten in a fix-up sweep, so the result never depends on the prediction.
+  const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
   if (ok) {
-    uint32_t k[VE];
-#pragma unroll
-    for (int e = 0; e < VE; ++e) k[e] = 0u;
-    if constexpr (kPacked) {
-      // |g| > sigma in binary32 is |g| > (sigma truncated to bf16) for a bf16 g; counts of up to
-      // 128 ones are exact in a bf16 accumulator
-      uint32_t thr[4] = {0u, 0u, 0u, 0u}, acc2[4] = {0u, 0u, 0u, 0u};
-      if (real) {
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-          thr[j] = (__float_as_uint(ch_sigma[c0 + 2 * j]) >> 16) | (__float_as_uint(ch_sigma[c0 + 2 * j + 1]) & 0xFFFF0000u);
-      }
-      int run = 0;
-      auto flush = [&]() {   // move the packed counts into the 32-bit counters
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          k[2 * j] += (uint32_t)__uint_as_float(acc2[j] << 16);
-          k[2 * j + 1] += (uint32_t)__uint_as_float(acc2[j] & 0xFFFF0000u);
-          acc2[j] = 0u;
-        }
-      };
-      auto body = [&](const uint4& raw) {
-        const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
-#pragma unroll
-        for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
-        if (++run == 128) { run = 0; flush(); }
-      };
-      if (real) {
-#pragma unroll 4
-        for (int row = rl; row < rows_res; row += rpi) body(vec_at(pieces, row));
-      }
-      for_each_piece(R, [&](const uint8_t* piece, int rows) {
-        if (!real) return;
-#pragma unroll 1
-        for (int row = rl; row < rows; row += rpi) body(vec_at(piece, row));
-      });
-      flush();
-    } else {
-      float sg[VE];
-#pragma unroll
-      for (int e = 0; e < VE; ++e) sg[e] = real ? ch_sigma[c0 + e] : 0.f;
-      auto body = [&](const uint4& raw) {
-        float v[VE];
-        unpack_raw(raw, v, (const T*)nullptr);
-#pragma unroll
-        for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
-      };
-      if (real) {
-#pragma unroll 4
-        for (int row = rl; row < rows_res; row += rpi) body(vec_at(pieces, row));
-      }
-      for_each_piece(R, [&](const uint8_t* piece, int rows) {
-        if (!real) return;
-#pragma unroll 1
-        for (int row = rl; row < rows; row += rpi) body(vec_at(piece, row));
-      });
-    }
-    if (active) {
-#pragma unroll
-      for (int e = 0; e < VE; ++e) red_cnt[e * kFT + pos] = k[e];
-    }
-    column_reduce_counts(red_cnt, rpi, Gp, VE, C, a.ws.cnt);
-  }
-  ok = grid_barrier(a.gridbar, 3u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
-
-  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------
-  if (ok) {
-    const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
-    const double thr = (double)a.mp.lambda * (double)a.npix;
+    const bool hinted = a.has_prev && a.cls != nullptr;
 #pragma unroll 1
     for (int c = tid; c <= C; c += kFT) {     // entry C: the layer-wide scale
-      const float gmax = ch_absmax[c];
-      float s = gmax;
+      float gmax, s;
       if (c < C) {
-        const uint32_t cnt = __ldcg(a.ws.cnt + c);
-        const bool bell = (double)cnt > thr;
-        if (!bell) {
-          const float s_prev = a.has_prev ? ch_sprev[c] : gmax;
-          s = __fadd_rn(__fmul_rn(tcoef, s_prev), __fmul_rn(a.mp.A, gmax));
-        }
-        if (blockIdx.x == 0) {
-          a.s_state[c] = s;
-          if (a.cls) a.cls[c] = bell ? 1 : 0;
-          if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt * a.inv_M);
-        }
-      } else if (blockIdx.x == 0) {
-        *a.gmax_layer = gmax;
+        gmax = __ldcg(a.ws.absmax + c);
+        const float sigma = __ldcg(a.ws.sigma + c);
+        ch_sigma[c] = a.sigma_override ? a.sigma_override[c] : sigma;
+        const bool pred = hinted ? a.cls[c] != 0 : gmax < a.pred_ratio * sigma;
+        ch_pred[c] = pred ? 1 : 0;
+        s = gmax;
+        if (!pred) s = __fadd_rn(__fmul_rn(tcoef, a.has_prev ? ch_sprev[c] : gmax), __fmul_rn(a.mp.A, gmax));
+      } else {
+        gmax = __uint_as_float(__ldcg(a.ws.gmax_bits));
+        s = gmax;
       }
+      ch_absmax[c] = gmax;
       ch_inv[c] = inv_scale(s);
     }
     consumer_sync();
+  }
 
-    // ---------------- phase 3: both sets of codes -------------------------------------------------
-    using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
-    float inv1[VE];
+  // ---------------- sweep 2: density count + both sets of codes --------------------------------------
+  using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
+  const uint32_t key0 = sr_key(a.seed, 0u);
+  const uint32_t keyx0 = key0 ^ (key0 >> 16);
+  const Idx HWi = (Idx)a.HW;
+  const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
+  const int64_t first = p0 + rl;                 // this thread's first pixel
+  int64_t n0;
+  if constexpr (IDX32) n0 = (int64_t)((uint32_t)first / (uint32_t)a.HW);   // fewer than 2^32 elements
+  else n0 = first / a.HW;
+  const Idx hw_first = (Idx)(first - n0 * a.HW);
+  const Idx idx_first = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + hw_first;   // NCHW index of (n, c0, hw)
+  const size_t o_stride = (size_t)rpi * a.Cp;
+  Idx hw = hw_first, idx0 = idx_first;
+  int8_t* o1 = a.q1 + first * a.Cp + c0;
+  int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
+  float inv1[VE];
+  // One pixel's vector of this thread: codes with inv1 (and, if with_gq, the layer-wide ones).
+  auto quantize_row = [&](const uint4& raw, bool with_gq, float inv2) {
+    uint32_t ra[VE], rb2[VE];
+    if (real) {
+      float v[VE];
+      unpack_raw(raw, v, (const T*)nullptr);
+      Idx idx = idx0;
 #pragma unroll
-    for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
-    const float inv2 = ch_inv[C];
-    const uint32_t key0 = sr_key(a.seed, 0u);
-    const uint32_t keyx0 = key0 ^ (key0 >> 16);
-    const Idx HWi = (Idx)a.HW;
-    const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
-    const int64_t first = p0 + rl;                 // this thread's first pixel
-    int64_t n0;
-    if constexpr (IDX32) n0 = (int64_t)((uint32_t)first / (uint32_t)a.HW);   // fewer than 2^32 elements
-    else n0 = first / a.HW;
-    Idx hw = (Idx)(first - n0 * a.HW);
-    Idx idx0 = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + hw;   // NCHW index of (n, c0, hw)
-    int8_t* o1 = a.q1 + first * a.Cp + c0;
-    int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
-    const size_t o_stride = (size_t)rpi * a.Cp;
-    auto body = [&](const uint8_t* piece, int row) {
-      uint32_t ra[VE], rb2[VE];
-      if (real) {
-        float v[VE];
-        unpack_raw(vec_at(piece, row), v, (const T*)nullptr);
-        Idx idx = idx0;
-#pragma unroll
-        for (int e = 0; e < VE; ++e) {
-          uint32_t h;
-          if constexpr (IDX32) {
-            h = sr_hash_folded(idx, keyx0);
-          } else {
-            const uint32_t hi = (uint32_t)(idx >> 32);
-            const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-            h = avalanche32((uint32_t)idx ^ key);
-          }
-          ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
-          if constexpr (DUAL) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
-          idx += HWi;
+      for (int e = 0; e < VE; ++e) {
+        uint32_t h;
+        if constexpr (IDX32) {
+          h = sr_hash_folded(idx, keyx0);
+        } else {
+          const uint32_t hi = (uint32_t)(idx >> 32);
+          const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
+          h = avalanche32((uint32_t)idx ^ key);
         }
-      } else {
+        ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
+        if constexpr (DUAL) {
+          if (with_gq) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+        }
+        idx += HWi;
+      }
+    } else {
 #pragma unroll
-        for (int e = 0; e < VE; ++e) { ra[e] = 0u; rb2[e] = 0u; }
-      }
-      if constexpr (VE == 8) {
-        *reinterpret_cast<uint2*>(o1) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4], ra[5], ra[6], ra[7]));
-        if constexpr (DUAL)
+      for (int e = 0; e < VE; ++e) { ra[e] = 0u; rb2[e] = 0u; }
+    }
+    if constexpr (VE == 8) {
+      *reinterpret_cast<uint2*>(o1) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4], ra[5], ra[6], ra[7]));
+      if constexpr (DUAL)
+        if (with_gq)
           *reinterpret_cast<uint2*>(o2) = make_uint2(pack_codes4(rb2[0], rb2[1], rb2[2], rb2[3]), pack_codes4(rb2[4], rb2[5], rb2[6], rb2[7]));
-      } else {
-        *reinterpret_cast<uint32_t*>(o1) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
-        if constexpr (DUAL) *reinterpret_cast<uint32_t*>(o2) = pack_codes4(rb2[0], rb2[1], rb2[2], rb2[3]);
+    } else {
+      *reinterpret_cast<uint32_t*>(o1) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
+      if constexpr (DUAL)
+        if (with_gq) *reinterpret_cast<uint32_t*>(o2) = pack_codes4(rb2[0], rb2[1], rb2[2], rb2[3]);
+    }
+    o1 += o_stride;
+    if constexpr (DUAL) o2 += o_stride;
+    hw += (Idx)rpi;
+    idx0 += (Idx)rpi;
+    while (hw >= HWi) { hw -= HWi; idx0 += wrap; }
+  };
+
+  if (ok) {
+    uint32_t k[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { k[e] = 0u; inv1[e] = real ? ch_inv[c0 + e] : 0.f; }
+    const float inv2 = ch_inv[C];
+    // density count.  bf16: |g| > sigma in binary32 is |g| > (sigma truncated to bf16) for a bf16 g,
+    // two elements per instruction; counts of up to 128 ones are exact in a bf16 accumulator
+    uint32_t thr[4] = {0u, 0u, 0u, 0u}, acc2[4] = {0u, 0u, 0u, 0u};
+    float sg[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) sg[e] = real ? ch_sigma[c0 + e] : 0.f;
+    if constexpr (kPacked) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) thr[j] = (__float_as_uint(sg[2 * j]) >> 16) | (__float_as_uint(sg[2 * j + 1]) & 0xFFFF0000u);
+    }
+    int run = 0;
+    auto flush = [&]() {   // move the packed counts into the 32-bit counters
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        k[2 * j < VE ? 2 * j : 0] += (uint32_t)__uint_as_float(acc2[j] << 16);
+        k[2 * j + 1 < VE ? 2 * j + 1 : 0] += (uint32_t)__uint_as_float(acc2[j] & 0xFFFF0000u);
+        acc2[j] = 0u;
       }
-      o1 += o_stride;
-      if constexpr (DUAL) o2 += o_stride;
-      hw += (Idx)rpi;
-      idx0 += (Idx)rpi;
-      while (hw >= HWi) { hw -= HWi; idx0 += wrap; }
+    };
+    auto body = [&](const uint8_t* piece, int row) {
+      uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+      if (real) {
+        raw = vec_at(piece, row);
+        if constexpr (kPacked) {
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
+          if (++run == 128) { run = 0; flush(); }
+        } else {
+          float v[VE];
+          unpack_raw(raw, v, (const T*)nullptr);
+#pragma unroll
+          for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+        }
+      }
+      quantize_row(raw, true, inv2);
     };
     if (active) {
 #pragma unroll 1
@@ -1176,6 +1170,62 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
       if (!active) return;
 #pragma unroll 1
       for (int row = rl; row < rows; row += rpi) body(piece, row);
+    });
+    if constexpr (kPacked) flush();
+    if (active) {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) red_cnt[e * kFT + pos] = k[e];
+    }
+    column_reduce_counts(red_cnt, rpi, Gp, VE, C, a.ws.cnt);
+  }
+  ok = grid_barrier(a.gridbar, 3u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
+
+  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------
+  bool fix_mine = false;
+  if (ok) {
+    const double thr = (double)a.mp.lambda * (double)a.npix;
+#pragma unroll 1
+    for (int c = tid; c < C; c += kFT) {
+      const float gmax = ch_absmax[c];
+      const uint32_t cnt = __ldcg(a.ws.cnt + c);
+      const bool bell = (double)cnt > thr;
+      float s = gmax;
+      if (!bell) s = __fadd_rn(__fmul_rn(tcoef, a.has_prev ? ch_sprev[c] : gmax), __fmul_rn(a.mp.A, gmax));
+      if (blockIdx.x == 0) {
+        a.s_state[c] = s;
+        if (a.cls) a.cls[c] = bell ? 1 : 0;
+        if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt * a.inv_M);
+      }
+      if (bell != (ch_pred[c] != 0)) {       // mispredicted: the codes of this channel are redone
+        ch_pred[c] = 2;
+        ch_inv[c] = inv_scale(s);
+        s_any_mis = 1u;
+      }
+    }
+    if (blockIdx.x == 0 && tid == 0) *a.gmax_layer = ch_absmax[C];
+    consumer_sync();
+    if (real) {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) fix_mine = fix_mine || ch_pred[c0 + e] == 2;
+    }
+  }
+  const bool fix_pass = ok && s_any_mis != 0u;
+  if (tid == 0) s_fix = fix_pass ? 2u : 1u;    // tells the producer whether a third sweep is streamed
+
+  // ---------------- fix-up sweep: per-channel codes of the vector columns with a wrong prediction ----
+  if (fix_pass) {
+    hw = hw_first; idx0 = idx_first;
+    o1 = a.q1 + first * a.Cp + c0;
+#pragma unroll
+    for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
+    if (fix_mine) {
+#pragma unroll 1
+      for (int row = rl; row < rows_res; row += rpi) quantize_row(vec_at(pieces, row), false, 0.f);
+    }
+    for_each_piece(R, [&](const uint8_t* piece, int rows) {
+      if (!fix_mine) return;
+#pragma unroll 1
+      for (int row = rl; row < rows; row += rpi) quantize_row(vec_at(piece, row), false, 0.f);
     });
   }
 
@@ -1214,7 +1264,7 @@ const FusedConfig& fused_config() {
 template <typename T, int VE, bool DUAL, bool IDX32>
 dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   const FusedConfig& cfg = fused_config();
-  const size_t fixed = (fused_red_bytes(VE) + (size_t)a.C * 16 + 8 + 127) / 128 * 128;
+  const size_t fixed = (fused_red_bytes(VE) + (size_t)a.C * 17 + 8 + 127) / 128 * 128;
   const size_t budget = cfg.smem_max - 1024;   // static shared memory of the kernel
   const int rb = a.C * (int)sizeof(T);
   const int rpi = fused_rows_per_iteration(a.Gp);
@@ -1239,6 +1289,10 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
     const double denom = a.mp.std_unbiased ? M - 1.0 : M;
     a.inv_M = 1.0 / M;
     a.inv_denom = denom > 0.0 ? 1.0 / denom : 0.0;
+    // expected |g|max / sigma of M samples: sqrt(2 ln M) for a Gaussian, ln(M)/sqrt(2) for a Laplace
+    // density; the midpoint separates the two channel shapes well for the M of real layers
+    const double lnM = std::log(M > 2.0 ? M : 2.0);
+    a.pred_ratio = (float)(0.5 * (std::sqrt(2.0 * lnM) + lnM / std::sqrt(2.0)));
   }
   const size_t smem = fixed + (size_t)slots * piece_bytes;
   auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL, IDX32>;
@@ -1306,7 +1360,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
     FusedArgs a;
     a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Cp / VEfull;
-    a.rp = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0;
+    a.rp = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0; a.pred_ratio = 0.f;
     a.ws = ws; a.gridbar = ws.gridbar; a.sigma_override = sigma_override; a.mp = mp;
     a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
     a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();

@@ -20,11 +20,12 @@ pytestmark = pytest.mark.gpu
 REL = 1e-5
 
 
-def check_grad_quant(g, bf16, layout, seed=5, iters=2, params=None):
+def check_grad_quant(g, bf16, layout, seed=5, iters=2, params=None, later=()):
+    """`later`: tensors for the iterations after the first (default: the same tensor again)."""
     N, C, H, W = g.shape
     M = N * H * W
     gq = GradQuant(N, C, H, W)
-    d = dev_input(g, bf16, layout)
+    tensors = [g] + list(later)
     kw = {}
     if params is not None:
         kw = dict(lam=params.lam, k=params.k, A=params.A)
@@ -32,6 +33,8 @@ def check_grad_quant(g, bf16, layout, seed=5, iters=2, params=None):
     s_prev_e2e = None
     band_ever = np.zeros(C, bool)
     for t in range(iters):
+        g = tensors[min(t, len(tensors) - 1)]
+        d = dev_input(g, bf16, layout)
         gq.run(d, layout, seed + t, has_prev=t > 0, params=params)
         stats = gq.stats.cpu().numpy()
         s_gpu = gq.s_state.cpu().numpy()
@@ -99,6 +102,21 @@ def test_ragged_shapes(shape, layout, bf16):
     if bf16:
         g = synth.round_to_bf16(g)
     check_grad_quant(g, bf16, layout, iters=2)
+
+
+@pytest.mark.parametrize("shape", [(8, 64, 14, 14), (4, 256, 40, 40), (64, 64, 56, 56)])
+def test_classes_change_between_iterations(shape):
+    """The fused kernel writes the codes with the class it predicts (from the previous classes when
+    the caller passes them) and redoes mispredicted channels: feed it tensors whose channels swap
+    between bell-shaped and long-tailed from one iteration to the next, so that about half of the
+    hints are wrong, and check every stage against the oracle as usual."""
+    ga, bell_a, _ = synth.channel_mixed_grad(*shape, seed=21)
+    gb, bell_b, _ = synth.channel_mixed_grad(*shape, seed=22)
+    gc, _, _ = synth.channel_mixed_grad(*shape, seed=23)
+    assert np.any(bell_a != bell_b)
+    rb = synth.round_to_bf16
+    check_grad_quant(rb(ga), True, api.NHWC, iters=3, later=(rb(gb), rb(gc)))
+    check_grad_quant(ga, False, api.NHWC, iters=3, later=(gb, gc))
 
 
 def test_hyper_parameters_and_flags():
