@@ -35,6 +35,9 @@ WORKLOAD = "resnet50_conv2x_bottleneck_N64_56x56_bf16_nhwc"
 BATCH = 64
 SEED = 2024
 INT8_OVER_BF16 = 2.0   # nominal dense ratio 4.5 / 2.25 PFLOP/s
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant call's kernel, from the ncu
+# capture summarised in profiles/gvq_fused_nhwc_bf16_conv2x.md (bytes; None once the kernel changes)
+NCU_TRAFFIC = {"quantize_grad @ conv2_x.1x1b": 188.58e6 + 59.36e6}
 
 
 def measured_peaks():
@@ -392,7 +395,8 @@ def run_dai8(args):
     else:
         achieved, peak, unit = alg[dkey]["bytes"] / dms / 1e6, peaks["hbm_gbs"], "GB/s"
     roofline = {"bound": dent["bound"], "achieved": round(achieved, 2), "peak": peak, "unit": unit,
-                "frac": round(achieved / peak, 4), "traffic": None,
+                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC.get(f"{dkey[1]} @ {dkey[0]}"),
+                "algorithmic_bytes": alg[dkey]["bytes"],
                 "kernel": f"{dkey[1]} @ {dkey[0]}", "peak_source": peaks["source"],
                 "peak_kind": ("int8 = 2 x bf16 " + ("sustained" if sustained else "burst")) if unit == "TOPS" else "copy"}
     def phase_ms(names):
