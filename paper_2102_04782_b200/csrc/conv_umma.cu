@@ -762,7 +762,7 @@ IgemmProblem dgrad_class_problem(const int8_t* gq, const int8_t* wT, const ConvS
 // de-quantizing kernel adds the slices in a fixed order: a hundred-odd CTAs adding into one small
 // image with atomics took longer to drain in L2 than the whole contraction.
 // ---------------------------------------------------------------------------------------------
-constexpr int kKP = 128;  // pixels per pipeline stage (4 MMAs of K = 32)
+constexpr int kKP = 128;  // pixels per pipeline stage (4 MMAs of K = 32); 256 where the stage is small
 
 struct WgradParams {
   int npix, P, Q;
@@ -774,6 +774,7 @@ struct WgradParams {
   int ci_tiles;
   int chunks_total, chunks_per_split;
   int stages, tmem_cols;
+  int kp;                // pixels per pipeline stage: 128 or 256
   int* acc;              // [splits][Cout][R*S][Cinp]: one partial image per slice of the pixels
   size_t acc_stride;     // elements per partial image
 };
@@ -815,8 +816,8 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
   const int co0 = blockIdx.z * kBM;
   const int tap_begin = grp * prm.tg;
   const int ntap = min(T, tap_begin + prm.tg) - tap_begin;
-  const int a_bytes = kKP * 128;
-  const int b_box_bytes = kKP * prm.bw;
+  const int a_bytes = prm.kp * 128;
+  const int b_box_bytes = prm.kp * prm.bw;
   const int stage_bytes = a_bytes + prm.tg * prm.nb * b_box_bytes;
 
   if (threadIdx.x == 0) {
@@ -841,7 +842,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
       for (int it = 0; it < k_iters; ++it) {
         const int s = it % prm.stages;
         if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag)) break;
-        const int pix0 = (chunk_begin + it) * kKP;
+        const int pix0 = (chunk_begin + it) * prm.kp;
         const int q0 = pix0 % prm.Q;
         const int t = pix0 / prm.Q;
         const int p0 = t % prm.P, img = t / prm.P;
@@ -880,7 +881,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
           const int cnt = min(per_mma, nbox - b0);
           const uint32_t idesc = idesc_i8_kmajor(cnt * prm.bw) | (1u << 15) | (1u << 16);
           const uint64_t bd = mnmajor_desc(sb + b0 * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
-          for (int kk = 0; kk < kKP / 32; ++kk)
+          for (int kk = 0; kk < prm.kp / 32; ++kk)
             mma_i8(tmem_base + (uint32_t)(b0 * prm.bw), ad + (uint64_t)((kk * 32 * 128) >> 4),
                    bd + (uint64_t)((kk * 32 * prm.bw) >> 4), idesc, (it > 0 || kk > 0) ? 1u : 0u);
         }
@@ -966,10 +967,14 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
   prm.tg = (T + ngroups - 1) / ngroups;
   prm.tmem_cols = 32;
   while (prm.tmem_cols < prm.tg * Nw) prm.tmem_cols *= 2;
-  const int stage_bytes = kKP * 128 + prm.tg * b_tap_bytes;
+  // Per-load fixed costs dominate small stages: shapes whose 128-pixel stage is small advance 256
+  // pixels per stage (halving the stage to 64 pixels where it is large made things slower).
+  prm.kp = kKP;
+  int stage_bytes = kKP * 128 + prm.tg * b_tap_bytes;
+  if ((200 * 1024) / (2 * stage_bytes) >= 3 && prm.npix >= 8 * 256) { prm.kp = 256; stage_bytes *= 2; }
   int stages = (200 * 1024) / stage_bytes;
   if (stages > 8) stages = 8;
-  prm.chunks_total = (prm.npix + kKP - 1) / kKP;
+  prm.chunks_total = (prm.npix + prm.kp - 1) / prm.kp;
   const int co_tiles = (cs.Cout + kBM - 1) / kBM;
   const int tiles = ngroups * prm.ci_tiles * co_tiles;
   int ksplit = sm_count() / tiles;
@@ -996,13 +1001,13 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   prm.acc = acc;
   *splits_out = ksplit;
   const int stages = prm.stages;
-  const int stage_bytes = kKP * 128 + prm.tg * prm.nb * kKP * prm.bw;
+  const int stage_bytes = prm.kp * 128 + prm.tg * prm.nb * prm.kp * prm.bw;
 
   CUtensorMap mapG, mapX;
   {
     const cuuint64_t dims[2] = {(cuuint64_t)cs.Coutp, (cuuint64_t)prm.npix};
     const cuuint64_t strides[1] = {(cuuint64_t)cs.Coutp};
-    const cuuint32_t box[2] = {128, (cuuint32_t)kKP};
+    const cuuint32_t box[2] = {128, (cuuint32_t)prm.kp};
     const cuuint32_t estr[2] = {1, 1};
     CUresult r = g_encode_tiled(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1016,7 +1021,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
     const int upper[2] = {-cs.pw + (cs.Q - 1) * cs.sw - (cs.W - 1), -cs.ph + (cs.P - 1) * cs.sh - (cs.H - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)cs.sw, (cuuint32_t)cs.sh, 1};
     CUresult r = g_encode_im2col(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(qX), dims, strides, lower,
-                                 upper, (cuuint32_t)prm.bw, (cuuint32_t)kKP, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                 upper, (cuuint32_t)prm.bw, (cuuint32_t)prm.kp, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  swizzle_for(prm.bw), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
