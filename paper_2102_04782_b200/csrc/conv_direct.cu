@@ -265,34 +265,40 @@ repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, Dgrad
   wT[t] = v;
 }
 
+template <int GROUPS>
 __global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                            const float* __restrict__ s, ConvShape cs, int pack_cin, int pack_R, int pack_S,
                            void* __restrict__ dW, dai8_dtype dtype) {
-  // A block sums 32 consecutive accumulators [co][r][s][ci] over the partial images: 8 groups of
-  // 32 threads take every 8th image (coalesced 128-byte reads, several in flight), shared memory
-  // combines the groups in a fixed order.  Integer sums: exact whatever the order.
-  __shared__ int part[8][32];
-  const int lane = threadIdx.x & 31, grp = threadIdx.x >> 5;
+  // A block sums kThreads/GROUPS consecutive accumulators [co][r][s][ci] over the partial images:
+  // GROUPS groups of threads take every GROUPS-th image (coalesced reads, several in flight), shared
+  // memory combines the groups in a fixed order.  Integer sums: exact whatever the order.  GROUPS is
+  // chosen from the number of images, so that few images do not leave most of a block idle.
+  constexpr int PER = kThreads / GROUPS;
+  __shared__ int part[GROUPS][PER];
+  const int lane = threadIdx.x % PER, grp = threadIdx.x / PER;
   const int64_t per_image = (int64_t)cs.Coutp * cs.R * cs.S * cs.Cinp;
   const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
-  const int64_t e = (int64_t)blockIdx.x * 32 + lane;     // index into one partial image
+  const int64_t e = (int64_t)blockIdx.x * PER + lane;     // index into one partial image
   int a = 0;
   if (e < valid) {
     const int* src = acc + e;
     int k = grp;
-    for (; k + 24 < splits; k += 32) {
-      const int v0 = src[(size_t)k * per_image], v1 = src[(size_t)(k + 8) * per_image];
-      const int v2 = src[(size_t)(k + 16) * per_image], v3 = src[(size_t)(k + 24) * per_image];
+    for (; k + 3 * GROUPS < splits; k += 4 * GROUPS) {
+      const int v0 = src[(size_t)k * per_image], v1 = src[(size_t)(k + GROUPS) * per_image];
+      const int v2 = src[(size_t)(k + 2 * GROUPS) * per_image], v3 = src[(size_t)(k + 3 * GROUPS) * per_image];
       a += v0 + v1 + v2 + v3;
     }
-    for (; k < splits; k += 8) a += src[(size_t)k * per_image];
+    for (; k < splits; k += GROUPS) a += src[(size_t)k * per_image];
   }
-  part[grp][lane] = a;
-  __syncthreads();
-  if (grp != 0 || e >= valid) return;
+  if (GROUPS > 1) {
+    part[grp][lane] = a;
+    __syncthreads();
+    if (grp != 0) return;
 #pragma unroll
-  for (int g = 1; g < 8; ++g) a += part[g][lane];
+    for (int g = 1; g < GROUPS; ++g) a += part[g][lane];
+  }
+  if (e >= valid) return;
   int ci = (int)(e % cs.Cinp);
   if (ci >= cs.Cin) return;                                // padding channel
   int64_t m = e / cs.Cinp;
@@ -310,6 +316,30 @@ finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float*
   }
   const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
   store_result(dW, dtype, (((size_t)co * Cin + ci) * R + r) * S + ss, a, scale);
+}
+
+// Few partial images, large filters: one block per output channel.  The sums are taken in the order
+// of the images ([tap][ci], coalesced reads) into shared memory and written in the order of dW
+// ([ci][tap], one contiguous run per output channel), so both sides move whole cache lines.
+__global__ void __launch_bounds__(kThreads)
+finalize_bwd_filter_rows_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
+                                const float* __restrict__ s, ConvShape cs, void* __restrict__ dW, dai8_dtype dtype) {
+  extern __shared__ int row[];                         // [T][Cinp]
+  const int co = blockIdx.x, T = cs.R * cs.S, n = T * cs.Cinp;
+  const size_t per_image = (size_t)cs.Coutp * n;
+  const int* src = acc + (size_t)co * n;
+  for (int i = threadIdx.x; i < n; i += kThreads) {
+    int a = 0;
+    for (int k = 0; k < splits; ++k) a += src[(size_t)k * per_image + i];
+    row[i] = a;
+  }
+  __syncthreads();
+  const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
+  const size_t out0 = (size_t)co * cs.Cin * T;
+  for (int j = threadIdx.x; j < cs.Cin * T; j += kThreads) {
+    const int ci = j / T, tap = j - ci * T;
+    store_result(dW, dtype, out0 + j, row[tap * cs.Cinp + ci], scale);
+  }
 }
 
 unsigned blocks_for(int64_t total) { return (unsigned)ceil_div64(total, kThreads); }
@@ -387,10 +417,17 @@ dai8_status pack_small_cin_weights(const int8_t* qW, const ConvShape& cs, int Kp
 dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, const float* s,
                                 const ConvShape& cs, const ConvShape* packed_from, void* dW, dai8_dtype dtype,
                                 cudaStream_t st) {
-  static_assert(kThreads == 256, "the finalize kernel tiles a block as 8 groups of 32 threads");
   const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
   const int pc = packed_from ? packed_from->Cin : 0, pr = packed_from ? packed_from->R : 0, ps = packed_from ? packed_from->S : 0;
-  finalize_bwd_filter_kernel<<<(unsigned)ceil_div64(valid, 32), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+  const size_t row_bytes = (size_t)cs.R * cs.S * cs.Cinp * sizeof(int);
+  if (!packed_from && splits <= 16 && row_bytes <= 48 * 1024 && row_bytes >= 4096) {
+    finalize_bwd_filter_rows_kernel<<<(unsigned)cs.Cout, kThreads, row_bytes, st>>>(acc, splits, sX, s, cs, dW, dtype);
+  } else if (splits >= 8)
+    finalize_bwd_filter_kernel<8><<<(unsigned)ceil_div64(valid, kThreads / 8), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+  else if (splits >= 3)
+    finalize_bwd_filter_kernel<2><<<(unsigned)ceil_div64(valid, kThreads / 2), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+  else
+    finalize_bwd_filter_kernel<1><<<(unsigned)ceil_div64(valid, kThreads), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
