@@ -758,7 +758,7 @@ __device__ __noinline__ void column_reduce_stats(float* smax, double* ssum, doub
   consumer_sync();
 }
 
-// counts of phase 2, added to the global per-channel counters
+// counts of phase 2, written to this CTA's row of partial counts
 __device__ __noinline__ void column_reduce_counts(uint32_t* scnt, int rows, int Gp, int VE, int C, uint32_t* out) {
   const int tid = threadIdx.x;
   const RedIndex ri = red_index(rows, Gp, VE);
@@ -782,7 +782,7 @@ __device__ __noinline__ void column_reduce_counts(uint32_t* scnt, int rows, int 
 #pragma unroll 4
     for (int p = 1; p < ri.parts; ++p) n += scnt[cell + p * Gp];
     const int c = col * VE + e;
-    if (c < C && n) atomicAdd(out + c, n);
+    if (c < C) out[c] = n;
   }
   consumer_sync();
 }
@@ -861,7 +861,7 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
       };
       if (issue(0, R + 2 * NS) && NS > 0) {
         const long long t0 = clock64();
-        while (s_fix == 0u && !s_abort) {          // the consumers decide after the third grid barrier
+        while (s_fix == 0u && !s_abort) {          // the consumers decide after the last grid barrier
           if (clock64() - t0 > kWaitTimeoutCycles) { s_abort = 1u; atomicExch(a.status, (unsigned int)DAI8_ERR_TIMEOUT); }
           __nanosleep(200);
         }
@@ -1176,33 +1176,62 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
 #pragma unroll
       for (int e = 0; e < VE; ++e) red_cnt[e * kFT + pos] = k[e];
     }
-    column_reduce_counts(red_cnt, rpi, Gp, VE, C, a.ws.cnt);
+    // the partial maxima are no longer needed: their rows now take the partial counts
+    column_reduce_counts(red_cnt, rpi, Gp, VE, C, reinterpret_cast<uint32_t*>(a.ws.pmax) + (size_t)blockIdx.x * C);
   }
   ok = grid_barrier(a.gridbar, 3u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
 
-  // ---------------- classify + clip (Algorithm 1, Eq. 14/15), identically in every CTA -----------
-  bool fix_mine = false;
+  // ---------------- classify + clip (Algorithm 1, Eq. 14/15) ---------------------------------------
+  // Channel c is classified by one warp of CTA (c mod gridDim.x), which adds the CTAs' partial counts,
+  // writes the channel's outputs and flags the channel if its class was mispredicted.
   if (ok) {
     const double thr = (double)a.mp.lambda * (double)a.npix;
+    const uint32_t* pcnt = reinterpret_cast<const uint32_t*>(a.ws.pmax);
+    const int nblk = gridDim.x;
 #pragma unroll 1
-    for (int c = tid; c < C; c += kFT) {
-      const float gmax = ch_absmax[c];
-      const uint32_t cnt = __ldcg(a.ws.cnt + c);
-      const bool bell = (double)cnt > thr;
-      float s = gmax;
-      if (!bell) s = __fadd_rn(__fmul_rn(tcoef, a.has_prev ? ch_sprev[c] : gmax), __fmul_rn(a.mp.A, gmax));
-      if (blockIdx.x == 0) {
+    for (int c = blockIdx.x + nblk * warp; c < C; c += nblk * (kFT / 32)) {
+      uint32_t cnt = 0u;
+#pragma unroll 1
+      for (int b0 = lane; b0 < nblk; b0 += 32 * 5) {   // five independent partials per round trip
+        uint32_t pc[5];
+#pragma unroll
+        for (int u = 0; u < 5; ++u) {
+          const int b = b0 + 32 * u;
+          pc[u] = b < nblk ? __ldcg(pcnt + (size_t)b * C + c) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 5; ++u) cnt += pc[u];
+      }
+#pragma unroll 1
+      for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
+      if (lane == 0) {
+        const float gmax = ch_absmax[c];
+        const bool bell = (double)cnt > thr;
+        float s = gmax;
+        if (!bell) s = __fadd_rn(__fmul_rn(tcoef, a.has_prev ? ch_sprev[c] : gmax), __fmul_rn(a.mp.A, gmax));
         a.s_state[c] = s;
         if (a.cls) a.cls[c] = bell ? 1 : 0;
         if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt * a.inv_M);
-      }
-      if (bell != (ch_pred[c] != 0)) {       // mispredicted: the codes of this channel are redone
-        ch_pred[c] = 2;
-        ch_inv[c] = inv_scale(s);
-        s_any_mis = 1u;
+        const bool mis = bell != (ch_pred[c] != 0);
+        a.ws.tickets[c] = mis ? 1u : 0u;
+        if (mis) *reinterpret_cast<volatile uint32_t*>(a.ws.ticket2) = 1u;
       }
     }
     if (blockIdx.x == 0 && tid == 0) *a.gmax_layer = ch_absmax[C];
+  }
+  ok = grid_barrier(a.gridbar, 4u * gridDim.x, a.status, &s_abort, &s_ok) && ok;
+
+  // mispredicted channels (rare): their per-channel codes are redone with the right clip value
+  bool fix_mine = false;
+  if (ok && __ldcg(a.ws.ticket2) != 0u) {
+#pragma unroll 1
+    for (int c = tid; c < C; c += kFT) {
+      if (__ldcg(a.ws.tickets + c) != 0u) {
+        ch_pred[c] = 2;
+        ch_inv[c] = inv_scale(__ldcg(a.s_state + c));
+        s_any_mis = 1u;
+      }
+    }
     consumer_sync();
     if (real) {
 #pragma unroll
