@@ -605,6 +605,30 @@ __device__ __forceinline__ uint32_t bf16x2_add(uint32_t a, uint32_t b) {
   return d;
 }
 
+// Two binary32 additions per instruction on a register pair (lower word = first element).  Each
+// half is rounded exactly like the scalar addition of the same rounding mode.  There is no packed
+// multiply here on purpose: the assembler contracts a packed multiply with a packed addition that
+// consumes it into one fused operation (observed: codes that differ from the two-rounding
+// definition about once in 2^21 elements), which it never does with the scalar __fmul_rn.
+__device__ __forceinline__ uint64_t f32x2_pack(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void f32x2_unpack(uint64_t p, uint32_t& lo, uint32_t& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p));
+}
+__device__ __forceinline__ uint64_t f32x2_add_rn(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+__device__ __forceinline__ uint64_t f32x2_add_rd(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 // ---- mbarrier / bulk-copy wrappers ---------------------------------------------------------------
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -660,6 +684,7 @@ struct FusedArgs {
   int C, Cp, G, Gp;        // G input vector columns, Gp output vector columns (>= G, zero padding)
   int rows_per_warp, rpi;  // thread tiling, see fused_map
   int rp;                  // pixel rows per piece (a multiple of rpi)
+  int adv_q, adv_rem;      // rpi / HW and rpi % HW: how the (image, pixel) position advances per iteration
   int slots, ring_log2;    // shared-memory pieces per CTA; log2 of how many of them cycle when not all fit
   GvqWs ws;
   uint32_t* gridbar;
@@ -1072,32 +1097,68 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   const Idx hw_first = (Idx)(first - n0 * a.HW);
   const Idx idx_first = ((Idx)n0 * (Idx)C + (Idx)c0) * HWi + hw_first;   // NCHW index of (n, c0, hw)
   const size_t o_stride = (size_t)rpi * a.Cp;
+  const Idx adv_rem = (Idx)a.adv_rem, adv_idx = (Idx)rpi + (Idx)a.adv_q * wrap;
   Idx hw = hw_first, idx0 = idx_first;
   int8_t* o1 = a.q1 + first * a.Cp + c0;
   int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
   float inv1[VE];
+  auto hash_at = [&](Idx idx) -> uint32_t {
+    if constexpr (IDX32) {
+      return sr_hash_folded(idx, keyx0);
+    } else {
+      const uint32_t hi = (uint32_t)(idx >> 32);
+      const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
+      return avalanche32((uint32_t)idx ^ key);
+    }
+  };
   // One pixel's vector of this thread: codes with inv1 (and, if with_gq, the layer-wide ones).
-  auto quantize_row = [&](const uint4& raw, bool with_gq, float inv2) {
+  // `unclipped` promises |g * inv| <= 126.75 for every element and both scales: then neither clamp of
+  // the stochastic quantizer can act (v + u stays inside (-127.75, 127.75)), so the codes are
+  // floor(fl(fl(g * inv) + u)) and the additions run two elements at a time.
+  auto quantize_row = [&](const uint4& raw, bool with_gq, float inv2, bool unclipped, auto has_input) {
     uint32_t ra[VE], rb2[VE];
-    if (real) {
-      float v[VE];
-      unpack_raw(raw, v, (const T*)nullptr);
+    if constexpr (decltype(has_input)::value) {
       Idx idx = idx0;
+      bool done = false;
+      if constexpr (kPacked) {
+        if (unclipped) {
+          done = true;
+          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+          const uint32_t one_bits = 0xBF800000u, magic_bits = 0x4B400000u;   // -1.0f, 1.5 * 2^23
+          const uint64_t minus1 = f32x2_pack(one_bits, one_bits), magic = f32x2_pack(magic_bits, magic_bits);
 #pragma unroll
-      for (int e = 0; e < VE; ++e) {
-        uint32_t h;
-        if constexpr (IDX32) {
-          h = sr_hash_folded(idx, keyx0);
-        } else {
-          const uint32_t hi = (uint32_t)(idx >> 32);
-          const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-          h = avalanche32((uint32_t)idx ^ key);
+          for (int j = 0; j < 4; ++j) {
+            const uint32_t h0 = hash_at(idx);
+            idx += HWi;
+            const uint32_t h1 = hash_at(idx);
+            idx += HWi;
+            const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
+            const uint64_t v1 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv1[2 * j])), __float_as_uint(__fmul_rn(g1, inv1[2 * j + 1])));
+            const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0, 0x7Fu, 9), __funnelshift_r(h1, 0x7Fu, 9)), minus1);
+            f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v1, u1), magic), ra[2 * j], ra[2 * j + 1]);
+            if constexpr (DUAL) {
+              if (with_gq) {
+                const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0 * 0x9E3779B1u, 0x7Fu, 9),
+                                                            __funnelshift_r(h1 * 0x9E3779B1u, 0x7Fu, 9)), minus1);
+                const uint64_t v2 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv2)), __float_as_uint(__fmul_rn(g1, inv2)));
+                f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v2, u2), magic), rb2[2 * j], rb2[2 * j + 1]);
+              }
+            }
+          }
         }
-        ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
-        if constexpr (DUAL) {
-          if (with_gq) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+      }
+      if (!done) {
+        float v[VE];
+        unpack_raw(raw, v, (const T*)nullptr);
+#pragma unroll
+        for (int e = 0; e < VE; ++e) {
+          const uint32_t h = hash_at(idx);
+          ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
+          if constexpr (DUAL) {
+            if (with_gq) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+          }
+          idx += HWi;
         }
-        idx += HWi;
       }
     } else {
 #pragma unroll
@@ -1115,9 +1176,9 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     }
     o1 += o_stride;
     if constexpr (DUAL) o2 += o_stride;
-    hw += (Idx)rpi;
-    idx0 += (Idx)rpi;
-    while (hw >= HWi) { hw -= HWi; idx0 += wrap; }
+    hw += adv_rem;                      // rpi pixels further: rpi = adv_q * HW + adv_rem
+    idx0 += adv_idx;
+    if (hw >= HWi) { hw -= HWi; idx0 += wrap; }
   };
 
   if (ok) {
@@ -1135,6 +1196,18 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
 #pragma unroll
       for (int j = 0; j < 4; ++j) thr[j] = (__float_as_uint(sg[2 * j]) >> 16) | (__float_as_uint(sg[2 * j + 1]) & 0xFFFF0000u);
     }
+    // packed bf16 bounds below which no clamp of either quantizer can act: 126.6/inv = 0.9969 * scale,
+    // rounded toward zero to bf16, the smaller of the channel's and the layer's
+    uint32_t cthr[4] = {0u, 0u, 0u, 0u};
+    if constexpr (kPacked) {
+      const float lim2 = inv2 > 0.f ? __fdiv_rn(126.6f, inv2) : 3.0e38f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float l0 = fminf(inv1[2 * j] > 0.f ? __fdiv_rn(126.6f, inv1[2 * j]) : 3.0e38f, lim2);
+        const float l1 = fminf(inv1[2 * j + 1] > 0.f ? __fdiv_rn(126.6f, inv1[2 * j + 1]) : 3.0e38f, lim2);
+        cthr[j] = (__float_as_uint(l0) >> 16) | (__float_as_uint(l1) & 0xFFFF0000u);
+      }
+    }
     int run = 0;
     auto flush = [&]() {   // move the packed counts into the 32-bit counters
 #pragma unroll
@@ -1144,33 +1217,39 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
         acc2[j] = 0u;
       }
     };
-    auto body = [&](const uint8_t* piece, int row) {
-      uint4 raw = make_uint4(0u, 0u, 0u, 0u);
+    // the rows of this thread in one contiguous run of `rows` pixel rows starting at `base`
+    const uint32_t pstep = (uint32_t)rpi * (uint32_t)G * 16u;
+    auto sweep_rows = [&](const uint8_t* base, int rows) {
       if (real) {
-        raw = vec_at(piece, row);
-        if constexpr (kPacked) {
-          const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+        const uint8_t* p = base + ((uint32_t)rl * (uint32_t)G + (uint32_t)col) * 16u;
+#pragma unroll 1
+        for (int row = rl; row < rows; row += rpi, p += pstep) {
+          const uint4 raw = *reinterpret_cast<const uint4*>(p);
+          uint32_t over = 0u;     // nonzero if an element is large enough for a clamp to matter
+          if constexpr (kPacked) {
+            const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-          for (int j = 0; j < 4; ++j) acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(w[j] & 0x7FFF7FFFu, thr[j]));
-          if (++run == 128) { run = 0; flush(); }
-        } else {
-          float v[VE];
-          unpack_raw(raw, v, (const T*)nullptr);
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t mag = w[j] & 0x7FFF7FFFu;
+              acc2[j] = bf16x2_add(acc2[j], bf16x2_gt_one(mag, thr[j]));
+              over |= bf16x2_gt_one(mag, cthr[j]);
+            }
+            if (++run == 128) { run = 0; flush(); }
+          } else {
+            float v[VE];
+            unpack_raw(raw, v, (const T*)nullptr);
 #pragma unroll
-          for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+            for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+          }
+          quantize_row(raw, true, inv2, over == 0u, std::true_type{});
         }
+      } else if (active) {        // zero padding of the code rows
+#pragma unroll 1
+        for (int row = rl; row < rows; row += rpi) quantize_row(make_uint4(0u, 0u, 0u, 0u), true, 0.f, false, std::false_type{});
       }
-      quantize_row(raw, true, inv2);
     };
-    if (active) {
-#pragma unroll 1
-      for (int row = rl; row < rows_res; row += rpi) body(pieces, row);
-    }
-    for_each_piece(R, [&](const uint8_t* piece, int rows) {
-      if (!active) return;
-#pragma unroll 1
-      for (int row = rl; row < rows; row += rpi) body(piece, row);
-    });
+    sweep_rows(pieces, rows_res);
+    for_each_piece(R, sweep_rows);
     if constexpr (kPacked) flush();
     if (active) {
 #pragma unroll
@@ -1247,15 +1326,13 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
     o1 = a.q1 + first * a.Cp + c0;
 #pragma unroll
     for (int e = 0; e < VE; ++e) inv1[e] = real ? ch_inv[c0 + e] : 0.f;
-    if (fix_mine) {
-#pragma unroll 1
-      for (int row = rl; row < rows_res; row += rpi) quantize_row(vec_at(pieces, row), false, 0.f);
-    }
-    for_each_piece(R, [&](const uint8_t* piece, int rows) {
+    auto fix_rows = [&](const uint8_t* base, int rows) {
       if (!fix_mine) return;
 #pragma unroll 1
-      for (int row = rl; row < rows; row += rpi) quantize_row(vec_at(piece, row), false, 0.f);
-    });
+      for (int row = rl; row < rows; row += rpi) quantize_row(vec_at(base, row), false, 0.f, false, std::true_type{});
+    };
+    fix_rows(pieces, rows_res);
+    for_each_piece(R, fix_rows);
   }
 
   if (s_abort) {
@@ -1298,6 +1375,8 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   const int rb = a.C * (int)sizeof(T);
   const int rpi = fused_rows_per_iteration(a.Gp);
   a.rpi = rpi;
+  a.adv_q = (int)(rpi / a.HW);
+  a.adv_rem = (int)(rpi % a.HW);
   a.rows_per_warp = a.Gp <= 32 ? 32 / a.Gp : 0;
   int mult = kPieceBytes / (rpi * rb);
   if (mult < 1) mult = 1;
@@ -1389,7 +1468,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
     FusedArgs a;
     a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Cp / VEfull;
-    a.rp = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0; a.pred_ratio = 0.f;
+    a.rp = 0; a.adv_q = 0; a.adv_rem = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0; a.pred_ratio = 0.f;
     a.ws = ws; a.gridbar = ws.gridbar; a.sigma_override = sigma_override; a.mp = mp;
     a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
     a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
