@@ -463,6 +463,7 @@ def run_layer_report(args):
         best = None
         for _ in range(reps + 1):
             flush.zero_()
+            torch.cuda._sleep(200000)   # the host enqueues the call meanwhile, as in a pipelined training step
             e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
             e0.record(); call(); e1.record(); torch.cuda.synchronize()
             t = e0.elapsed_time(e1)
@@ -510,7 +511,7 @@ def run_layer_report(args):
     int8_peak = INT8_OVER_BF16 * peaks["bf16_burst"]
     bwd_ms = tot["bwd_data"][0] + tot["bwd_filter"][0]
     bwd_ops = tot["bwd_data"][1] + tot["bwd_filter"][1]
-    out = {"layers_config": args.layers, "batch": N, "timing": "best of 3 per call, L2 flushed before each call",
+    out = {"layers_config": args.layers, "batch": N, "timing": "best of 3 per call, CUDA events on the device; L2 flushed before each call; the call is enqueued while a delay kernel runs, so host launch latency is not in the time",
            "totals": {
                "fwd_ms": round(tot["fwd"][0], 3), "fwd_tops": round(tot["fwd"][1] / tot["fwd"][0] / 1e9, 1),
                "bwd_ms": round(bwd_ms, 3), "bwd_tops": round(bwd_ops / bwd_ms / 1e9, 1),
