@@ -231,6 +231,47 @@ pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* 
   reinterpret_cast<uint4*>(A)[t] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// The same matrix, one output row (n, p) per block: the R input rows it needs are first compacted to
+// their real channels in shared memory, where the S*Cin bytes of one filter row of one output pixel
+// are contiguous, so every input vector is fetched once per block and the rows of A' leave as
+// full 16-byte stores.
+__global__ void __launch_bounds__(kThreads)
+pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int rowpix, int rowbytes,
+                        int8_t* __restrict__ A) {
+  extern __shared__ uint8_t xrows[];                            // [R][rowbytes]
+  const int p = blockIdx.x % cs.P, n = blockIdx.x / cs.P;
+  for (int i = threadIdx.x; i < cs.R * rowpix; i += kThreads) {
+    const int r = i / rowpix, xi = i - r * rowpix;
+    const int h = p * cs.sh + r - cs.ph, x = xi - cs.pw;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (h >= 0 && h < cs.H && x >= 0 && x < cs.W)
+      v = *reinterpret_cast<const uint4*>(qX + (((int64_t)n * cs.H + h) * cs.W + x) * 16);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    uint8_t* dst = xrows + r * rowbytes + xi * cs.Cin;
+#pragma unroll
+    for (int c = 0; c < 16; ++c)
+      if (c < cs.Cin) dst[c] = (uint8_t)(w[c >> 2] >> (8 * (c & 3)));
+  }
+  __syncthreads();
+  const int groups = Kp / 16, SC = cs.S * cs.Cin, Kreal = cs.R * SC;
+  uint4* out = reinterpret_cast<uint4*>(A) + (int64_t)blockIdx.x * cs.Q * groups;
+  for (int i = threadIdx.x; i < cs.Q * groups; i += kThreads) {
+    const int q = i / groups, kg = i - q * groups;
+    int k = kg * 16;
+    int r = k / SC, off = k - r * SC;
+    const uint8_t* src = xrows + q * cs.sw * cs.Cin;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 16; ++j, ++k) {
+      if (k < Kreal) {
+        w[j >> 2] |= (uint32_t)src[r * rowbytes + off] << (8 * (j & 3));
+        if (++off == SC) { off = 0; ++r; }
+      }
+    }
+    out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+
 // [Cout][R][S][Cinp] -> [Cout][Kp] in the same k' order.
 __global__ void __launch_bounds__(kThreads)
 pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t* __restrict__ Wp) {
@@ -246,76 +287,102 @@ pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t*
   Wp[t] = v;
 }
 
+// One block transposes a 64 (co) x 64 (ci) tile of one filter tap through shared memory: 16-byte reads
+// along ci, 16-byte writes along co.  blockIdx.z runs over the taps in class order.
 __global__ void __launch_bounds__(kThreads)
 repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, DgradClasses dc, int8_t* __restrict__ wT) {
-  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;   // the classes partition the taps
-  int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
-  if (t >= total) return;
-  int k = 0;
-  while (k + 1 < dc.n && t >= dc.cls[k + 1].w_off) ++k;
+  __shared__ __align__(16) uint8_t tile[64][80];              // [co][ci], rows padded against bank conflicts
+  int k = 0, local = blockIdx.z;
+  while (k + 1 < dc.n && local >= dc.cls[k].Tr * dc.cls[k].Ts) { local -= dc.cls[k].Tr * dc.cls[k].Ts; ++k; }
   const DgradClass& c = dc.cls[k];
-  int64_t m = t - c.w_off;
-  const int co = (int)(m % cs.Coutp); m /= cs.Coutp;
-  const int ts = (int)(m % c.Ts); m /= c.Ts;
-  const int tr = (int)(m % c.Tr);
-  const int ci = (int)(m / c.Tr);
+  if (local >= c.Tr * c.Ts) return;
+  const int tr = local / c.Ts, ts = local - tr * c.Ts;
   const int r = c.r0 + cs.sh * (c.Tr - 1 - tr), s = c.s0 + cs.sw * (c.Ts - 1 - ts);   // mirrored order
-  int8_t v = 0;
-  if (co < cs.Cout) v = qW[(((int64_t)co * cs.R + r) * cs.S + s) * cs.Cinp + ci];  // ci >= Cin holds 0
-  wT[t] = v;
+  const int co0 = blockIdx.x * 64, ci0 = blockIdx.y * 64;
+  {
+    const int co = co0 + threadIdx.x / 4, ci = ci0 + (threadIdx.x & 3) * 16;
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (co < cs.Cout && ci < cs.Cinp)     // channels ci >= Cin hold zeros in qW
+      v = *reinterpret_cast<const uint4*>(qW + (((int64_t)co * cs.R + r) * cs.S + s) * cs.Cinp + ci);
+    *reinterpret_cast<uint4*>(&tile[threadIdx.x / 4][(threadIdx.x & 3) * 16]) = v;
+  }
+  __syncthreads();
+  const int ci = ci0 + threadIdx.x / 4, cq = (threadIdx.x & 3) * 16;
+  if (ci >= cs.Cinp || co0 + cq >= cs.Coutp) return;
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int j = 0; j < 16; ++j) w[j >> 2] |= (uint32_t)tile[cq + j][threadIdx.x / 4] << (8 * (j & 3));
+  *reinterpret_cast<uint4*>(wT + c.w_off + (((int64_t)ci * c.Tr + tr) * c.Ts + ts) * cs.Coutp + co0 + cq) =
+      make_uint4(w[0], w[1], w[2], w[3]);
 }
+
+__device__ __forceinline__ void add4(int4& a, const int4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 
 template <int GROUPS>
 __global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                            const float* __restrict__ s, ConvShape cs, int pack_cin, int pack_R, int pack_S,
                            void* __restrict__ dW, dai8_dtype dtype) {
-  // A block sums kThreads/GROUPS consecutive accumulators [co][r][s][ci] over the partial images:
-  // GROUPS groups of threads take every GROUPS-th image (coalesced reads, several in flight), shared
-  // memory combines the groups in a fixed order.  Integer sums: exact whatever the order.  GROUPS is
-  // chosen from the number of images, so that few images do not leave most of a block idle.
+  // A block sums kThreads/GROUPS consecutive groups of four accumulators [co][r][s][ci..ci+3] over the
+  // partial images: GROUPS groups of threads take every GROUPS-th image (16-byte coalesced reads,
+  // several in flight), shared memory combines the groups in a fixed order.  Integer sums: exact
+  // whatever the order.  GROUPS is chosen by the host so that small images still fill the device.
   constexpr int PER = kThreads / GROUPS;
-  __shared__ int part[GROUPS][PER];
+  __shared__ int4 part[GROUPS > 1 ? GROUPS - 1 : 1][PER];
   const int lane = threadIdx.x % PER, grp = threadIdx.x / PER;
   const int64_t per_image = (int64_t)cs.Coutp * cs.R * cs.S * cs.Cinp;
-  const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;
-  const int64_t e = (int64_t)blockIdx.x * PER + lane;     // index into one partial image
-  int a = 0;
+  const int64_t valid = (int64_t)cs.Cout * cs.R * cs.S * cs.Cinp;      // a multiple of 16
+  const int64_t e = ((int64_t)blockIdx.x * PER + lane) * 4;           // index into one partial image
+  int4 a = make_int4(0, 0, 0, 0);
   if (e < valid) {
     const int* src = acc + e;
     int k = grp;
     for (; k + 3 * GROUPS < splits; k += 4 * GROUPS) {
-      const int v0 = src[(size_t)k * per_image], v1 = src[(size_t)(k + GROUPS) * per_image];
-      const int v2 = src[(size_t)(k + 2 * GROUPS) * per_image], v3 = src[(size_t)(k + 3 * GROUPS) * per_image];
-      a += v0 + v1 + v2 + v3;
+      const int4 v0 = __ldg(reinterpret_cast<const int4*>(src + (size_t)k * per_image));
+      const int4 v1 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + GROUPS) * per_image));
+      const int4 v2 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + 2 * GROUPS) * per_image));
+      const int4 v3 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + 3 * GROUPS) * per_image));
+      add4(a, v0); add4(a, v1); add4(a, v2); add4(a, v3);
     }
-    for (; k < splits; k += GROUPS) a += src[(size_t)k * per_image];
+    for (; k < splits; k += GROUPS) add4(a, __ldg(reinterpret_cast<const int4*>(src + (size_t)k * per_image)));
   }
   if (GROUPS > 1) {
-    part[grp][lane] = a;
+    if (grp != 0) part[grp - 1][lane] = a;
     __syncthreads();
     if (grp != 0) return;
 #pragma unroll
-    for (int g = 1; g < GROUPS; ++g) a += part[g][lane];
+    for (int g = 1; g < GROUPS; ++g) add4(a, part[g - 1][lane]);
   }
   if (e >= valid) return;
-  int ci = (int)(e % cs.Cinp);
-  if (ci >= cs.Cin) return;                                // padding channel
+  const int ci0 = (int)(e % cs.Cinp);                      // the four share (co, r, s): Cinp is a multiple of 16
   int64_t m = e / cs.Cinp;
-  int ss = (int)(m % cs.S); m /= cs.S;
-  int r = (int)(m % cs.R);
+  const int ss0 = (int)(m % cs.S); m /= cs.S;
+  const int r0 = (int)(m % cs.R);
   const int co = (int)(m / cs.R);
-  int Cin = cs.Cin, R = cs.R, S = cs.S;
-  if (pack_cin > 0) {
-    // the images come from the packed pointwise form: `ci` is k' = (r*S + s)*Cin + ci of the real filter
-    const int k = ci;
-    if (k >= pack_R * pack_S * pack_cin) return;
-    const int tap = k / pack_cin;
-    ci = k - tap * pack_cin; r = tap / pack_S; ss = tap - r * pack_S;
-    Cin = pack_cin; R = pack_R; S = pack_S;
-  }
   const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
-  store_result(dW, dtype, (((size_t)co * Cin + ci) * R + r) * S + ss, a, scale);
+  const int v[4] = {a.x, a.y, a.z, a.w};
+  if (pack_cin == 0 && cs.R * cs.S == 1 && dtype == DAI8_F32 && (cs.Cin & 3) == 0) {
+    // pointwise filters: dW is [co][ci], the four results are one aligned 16-byte store
+    if (ci0 < cs.Cin)
+      *reinterpret_cast<float4*>(static_cast<float*>(dW) + (size_t)co * cs.Cin + ci0) =
+          make_float4(__fmul_rn((float)v[0], scale), __fmul_rn((float)v[1], scale), __fmul_rn((float)v[2], scale),
+                      __fmul_rn((float)v[3], scale));
+    return;
+  }
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    int ci = ci0 + j, r = r0, ss = ss0, Cin = cs.Cin, R = cs.R, S = cs.S;
+    if (ci >= cs.Cin) continue;                            // padding channel
+    if (pack_cin > 0) {
+      // the images come from the packed pointwise form: `ci` is k' = (r*S + s)*Cin + ci of the real filter
+      const int k = ci;
+      if (k >= pack_R * pack_S * pack_cin) continue;
+      const int tap = k / pack_cin;
+      ci = k - tap * pack_cin; r = tap / pack_S; ss = tap - r * pack_S;
+      Cin = pack_cin; R = pack_R; S = pack_S;
+    }
+    store_result(dW, dtype, (((size_t)co * Cin + ci) * R + r) * S + ss, v[j], scale);
+  }
 }
 
 // Few partial images, large filters: one block per output channel.  The sums are taken in the order
@@ -328,10 +395,18 @@ finalize_bwd_filter_rows_kernel(const int* __restrict__ acc, int splits, const f
   const int co = blockIdx.x, T = cs.R * cs.S, n = T * cs.Cinp;
   const size_t per_image = (size_t)cs.Coutp * n;
   const int* src = acc + (size_t)co * n;
-  for (int i = threadIdx.x; i < n; i += kThreads) {
-    int a = 0;
-    for (int k = 0; k < splits; ++k) a += src[(size_t)k * per_image + i];
-    row[i] = a;
+  for (int i = threadIdx.x * 4; i < n; i += kThreads * 4) {     // n is a multiple of 16
+    int4 a = make_int4(0, 0, 0, 0);
+    int k = 0;
+    for (; k + 3 < splits; k += 4) {
+      const int4 v0 = __ldg(reinterpret_cast<const int4*>(src + (size_t)k * per_image + i));
+      const int4 v1 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + 1) * per_image + i));
+      const int4 v2 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + 2) * per_image + i));
+      const int4 v3 = __ldg(reinterpret_cast<const int4*>(src + (size_t)(k + 3) * per_image + i));
+      add4(a, v0); add4(a, v1); add4(a, v2); add4(a, v3);
+    }
+    for (; k < splits; ++k) add4(a, __ldg(reinterpret_cast<const int4*>(src + (size_t)k * per_image + i)));
+    *reinterpret_cast<int4*>(row + i) = a;
   }
   __syncthreads();
   const float scale = dtype == DAI8_I32 ? 0.f : dequant_scale(*sX, s[co]);
@@ -392,16 +467,22 @@ dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int
 
 dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const DgradClasses& dc, int8_t* wT,
                                    cudaStream_t st) {
-  const int64_t total = (int64_t)cs.Cinp * cs.R * cs.S * cs.Coutp;
-  repack_weights_classes_kernel<<<blocks_for(total), kThreads, 0, st>>>(qW, cs, dc, wT);
+  const dim3 grid((unsigned)((cs.Coutp + 63) / 64), (unsigned)((cs.Cinp + 63) / 64), (unsigned)(cs.R * cs.S));
+  repack_weights_classes_kernel<<<grid, kThreads, 0, st>>>(qW, cs, dc, wT);
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
 }
 
 dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st) {
-  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
-  pack_im2col_kernel<<<blocks_for(total), kThreads, 0, st>>>(qX, cs, Kp, A);
+  const int rowpix = (cs.Q - 1) * cs.sw + cs.S;
+  const int rowbytes = round_up(rowpix * cs.Cin, 4);
+  if ((size_t)cs.R * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
+    pack_im2col_rows_kernel<<<(unsigned)(cs.N * cs.P), kThreads, (size_t)cs.R * rowbytes, st>>>(qX, cs, Kp, rowpix, rowbytes, A);
+  } else {
+    const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
+    pack_im2col_kernel<<<blocks_for(total), kThreads, 0, st>>>(qX, cs, Kp, A);
+  }
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
@@ -422,12 +503,20 @@ dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, con
   const size_t row_bytes = (size_t)cs.R * cs.S * cs.Cinp * sizeof(int);
   if (!packed_from && splits <= 16 && row_bytes <= 48 * 1024 && row_bytes >= 4096) {
     finalize_bwd_filter_rows_kernel<<<(unsigned)cs.Cout, kThreads, row_bytes, st>>>(acc, splits, sX, s, cs, dW, dtype);
-  } else if (splits >= 8)
-    finalize_bwd_filter_kernel<8><<<(unsigned)ceil_div64(valid, kThreads / 8), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
-  else if (splits >= 3)
-    finalize_bwd_filter_kernel<2><<<(unsigned)ceil_div64(valid, kThreads / 2), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
-  else
-    finalize_bwd_filter_kernel<1><<<(unsigned)ceil_div64(valid, kThreads), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+  } else {
+    // enough groups to put some 150 thousand threads to work, as far as there are images to share out
+    const int64_t quads = valid / 4;
+    int groups = 1;
+    while (groups < 8 && groups * 2 <= splits && quads * groups < 150000) groups *= 2;
+    if (groups == 8)
+      finalize_bwd_filter_kernel<8><<<(unsigned)ceil_div64(quads, kThreads / 8), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+    else if (groups == 4)
+      finalize_bwd_filter_kernel<4><<<(unsigned)ceil_div64(quads, kThreads / 4), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+    else if (groups == 2)
+      finalize_bwd_filter_kernel<2><<<(unsigned)ceil_div64(quads, kThreads / 2), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+    else
+      finalize_bwd_filter_kernel<1><<<(unsigned)ceil_div64(quads, kThreads), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+  }
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
