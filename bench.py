@@ -456,7 +456,7 @@ def run_layer_report(args):
     peaks = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     bf = torch.bfloat16
-    rows, seen = [], {}
+    rows, seen, no_dx = [], {}, []
     tot = {"fwd": [0.0, 0], "bwd_data": [0.0, 0], "bwd_filter": [0.0, 0], "quantize_grad": [0.0, 0]}
 
     def timed(call, reps=3):
@@ -505,6 +505,9 @@ def run_layer_report(args):
                      "tops": {k: round(ops / t[k] / 1e9, 1) for k in ("fwd", "bwd_data", "bwd_filter")},
                      "gvq_gbs": round(gvq_bytes / t["quantize_grad"] / 1e6, 1)})
         for k in ("fwd", "bwd_data", "bwd_filter"):
+            if k == "bwd_data" and L.Cin == 3:
+                no_dx.append(L.name)      # the gradient of the input image has no consumer in training
+                continue
             tot[k][0] += t[k]; tot[k][1] += ops
         tot["quantize_grad"][0] += t["quantize_grad"]; tot["quantize_grad"][1] += gvq_bytes
     assert api.get_device_status() == api.OK
@@ -520,6 +523,7 @@ def run_layer_report(args):
                "gvq_gbs": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6, 1),
                "gvq_frac_hbm": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6 / peaks["hbm_gbs"], 4),
                "int8_peak_tops": int8_peak, "hbm_peak_gbs": peaks["hbm_gbs"]},
+           "bwd_data_not_counted": no_dx,   # layers fed by the image: timed per layer below, left out of the totals
            "layers": rows}
     print(json.dumps(out))
 
