@@ -537,6 +537,30 @@ absmax_kernel(const T* __restrict__ x, int64_t nvec, uint32_t* __restrict__ out_
   if ((threadIdx.x & 31) == 0 && m > 0.f) atomicMax(out_bits, __float_as_uint(m));
 }
 
+// Eq. 1 with one scale and nearest rounding over a tensor whose codes have the layout of its values
+// (NHWC with C a multiple of 16, or any layout-free use): no index arithmetic at all.  The vectors are
+// visited from the END of the tensor downwards: absmax_kernel, which runs just before, has left the
+// tail of the tensor in L2, so most of this second read never reaches DRAM.
+template <typename T, int VE>
+__global__ void __launch_bounds__(kThreads)
+quantize_flat_nearest_kernel(const T* __restrict__ x, int64_t nvec, const float* __restrict__ scale,
+                             int8_t* __restrict__ q) {
+  const float inv = inv_scale(*scale);
+  const int64_t stride = (int64_t)gridDim.x * kThreads;
+#pragma unroll 4
+  for (int64_t i = nvec - 1 - ((int64_t)blockIdx.x * kThreads + threadIdx.x); i >= 0; i -= stride) {
+    float v[VE];
+    load_vec<T, VE>(x + i * VE, v);
+    uint32_t r[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) r[e] = quant_nearest_bits(v[e], inv);
+    if constexpr (VE == 8)
+      *reinterpret_cast<uint2*>(q + i * VE) = make_uint2(pack_codes4(r[0], r[1], r[2], r[3]), pack_codes4(r[4], r[5], r[6], r[7]));
+    else
+      *reinterpret_cast<uint32_t*>(q + i * VE) = pack_codes4(r[0], r[1], r[2], r[3]);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Fused NHWC path: statistics, density count, clip update and both code tensors in ONE persistent
 // cooperative kernel, one CTA per SM, in two sweeps over dY (plus a rare partial third).
@@ -1536,8 +1560,16 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
   const int total = N * C * HW;
   if (absmax_mode) {
     float m = 0.f;
-#pragma unroll 4
-    for (int i = tid; i < total; i += kSmallThreads) m = fmaxf(m, fabsf(to_f32(x[i])));
+    constexpr int VE = 16 / (int)sizeof(T);          // 16-byte loads, several in flight per thread
+    const int nvec = total / VE;
+#pragma unroll 8
+    for (int i = tid; i < nvec; i += kSmallThreads) {
+      float v[VE];
+      load_vec<T, VE>(x + (size_t)i * VE, v);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) m = fmaxf(m, fabsf(v[e]));
+    }
+    for (int i = nvec * VE + tid; i < total; i += kSmallThreads) m = fmaxf(m, fabsf(to_f32(x[i])));
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
     if ((tid & 31) == 0) s_part[tid >> 5] = m;
     __syncthreads();
@@ -1603,7 +1635,11 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
     note_launch(1);
   }
   const bool stoch = round == DAI8_ROUND_STOCHASTIC;
-  if (layout == DAI8_NHWC) {
+  if (layout == DAI8_NHWC && !stoch && C == Cp) {
+    const int64_t nvec = total / VEfull;      // C is a multiple of 16
+    const int blocks = (int)(ceil_div64(nvec, kThreads * 4) < 2 * kMaxPixelBlocks ? ceil_div64(nvec, kThreads * 4) : 2 * kMaxPixelBlocks);
+    quantize_flat_nearest_kernel<T, VEfull><<<blocks, kThreads, 0, st>>>(x, nvec, scale, q);
+  } else if (layout == DAI8_NHWC) {
     if (C % VEfull == 0) {
       const NhwcGrid g = nhwc_grid(npix, Cp / VEfull);
       if (stoch)
