@@ -203,6 +203,8 @@ repack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int8_t* __res
 // convolutions then run as pointwise convolutions with Kp input channels on the tensor-core kernels.
 __global__ void __launch_bounds__(kThreads)
 pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* __restrict__ A) {
+  grid_dependency_release();
+  grid_dependency_wait();
   const int groups = Kp / 16;                                   // 16-byte groups per pixel row of A'
   const int64_t total = (int64_t)cs.N * cs.P * cs.Q * groups;
   const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
@@ -238,6 +240,8 @@ pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* 
 __global__ void __launch_bounds__(kThreads)
 pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int rowpix, int rowbytes,
                         int8_t* __restrict__ A) {
+  grid_dependency_release();
+  grid_dependency_wait();
   extern __shared__ uint8_t xrows[];                            // [R][rowbytes]
   const int p = blockIdx.x % cs.P, n = blockIdx.x / cs.P;
   for (int i = threadIdx.x; i < cs.R * rowpix; i += kThreads) {
@@ -275,6 +279,8 @@ pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int
 // [Cout][R][S][Cinp] -> [Cout][Kp] in the same k' order.
 __global__ void __launch_bounds__(kThreads)
 pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t* __restrict__ Wp) {
+  grid_dependency_release();
+  grid_dependency_wait();
   const int64_t total = (int64_t)cs.Cout * Kp;
   const int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x;
   if (t >= total) return;
@@ -291,6 +297,8 @@ pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t*
 // along ci, 16-byte writes along co.  blockIdx.z runs over the taps in class order.
 __global__ void __launch_bounds__(kThreads)
 repack_weights_classes_kernel(const int8_t* __restrict__ qW, ConvShape cs, DgradClasses dc, int8_t* __restrict__ wT) {
+  grid_dependency_release();
+  grid_dependency_wait();
   __shared__ __align__(16) uint8_t tile[64][80];              // [co][ci], rows padded against bank conflicts
   int k = 0, local = blockIdx.z;
   while (k + 1 < dc.n && local >= dc.cls[k].Tr * dc.cls[k].Ts) { local -= dc.cls[k].Tr * dc.cls[k].Ts; ++k; }
@@ -323,6 +331,8 @@ __global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                            const float* __restrict__ s, ConvShape cs, int pack_cin, int pack_R, int pack_S,
                            void* __restrict__ dW, dai8_dtype dtype) {
+  grid_dependency_release();
+  grid_dependency_wait();
   // A block sums kThreads/GROUPS consecutive groups of four accumulators [co][r][s][ci..ci+3] over the
   // partial images: GROUPS groups of threads take every GROUPS-th image (16-byte coalesced reads,
   // several in flight), shared memory combines the groups in a fixed order.  Integer sums: exact
@@ -391,6 +401,8 @@ finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float*
 __global__ void __launch_bounds__(kThreads)
 finalize_bwd_filter_rows_kernel(const int* __restrict__ acc, int splits, const float* __restrict__ sX,
                                 const float* __restrict__ s, ConvShape cs, void* __restrict__ dW, dai8_dtype dtype) {
+  grid_dependency_release();
+  grid_dependency_wait();
   extern __shared__ int row[];                         // [T][Cinp]
   const int co = blockIdx.x, T = cs.R * cs.S, n = T * cs.Cinp;
   const size_t per_image = (size_t)cs.Coutp * n;
@@ -468,7 +480,7 @@ dai8_status repack_weights_transposed(const int8_t* qW, const ConvShape& cs, int
 dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const DgradClasses& dc, int8_t* wT,
                                    cudaStream_t st) {
   const dim3 grid((unsigned)((cs.Coutp + 63) / 64), (unsigned)((cs.Cinp + 63) / 64), (unsigned)(cs.R * cs.S));
-  repack_weights_classes_kernel<<<grid, kThreads, 0, st>>>(qW, cs, dc, wT);
+  DAI8_RETURN_IF_CUDA(launch_dependent(repack_weights_classes_kernel, dim3(grid), dim3(kThreads), 0, st, qW, cs, dc, wT));
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
@@ -478,10 +490,10 @@ dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t
   const int rowpix = (cs.Q - 1) * cs.sw + cs.S;
   const int rowbytes = round_up(rowpix * cs.Cin, 4);
   if ((size_t)cs.R * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
-    pack_im2col_rows_kernel<<<(unsigned)(cs.N * cs.P), kThreads, (size_t)cs.R * rowbytes, st>>>(qX, cs, Kp, rowpix, rowbytes, A);
+    DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_rows_kernel, dim3((unsigned)(cs.N * cs.P)), dim3(kThreads), (size_t)cs.R * rowbytes, st, qX, cs, Kp, rowpix, rowbytes, A));
   } else {
     const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
-    pack_im2col_kernel<<<blocks_for(total), kThreads, 0, st>>>(qX, cs, Kp, A);
+    DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_kernel, dim3(blocks_for(total)), dim3(kThreads), 0, st, qX, cs, Kp, A));
   }
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
@@ -489,7 +501,7 @@ dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t
 }
 
 dai8_status pack_small_cin_weights(const int8_t* qW, const ConvShape& cs, int Kp, int8_t* Wp, cudaStream_t st) {
-  pack_weights_kernel<<<blocks_for((int64_t)cs.Cout * Kp), kThreads, 0, st>>>(qW, cs, Kp, Wp);
+  DAI8_RETURN_IF_CUDA(launch_dependent(pack_weights_kernel, dim3(blocks_for((int64_t)cs.Cout * Kp)), dim3(kThreads), 0, st, qW, cs, Kp, Wp));
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
@@ -502,20 +514,20 @@ dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, con
   const int pc = packed_from ? packed_from->Cin : 0, pr = packed_from ? packed_from->R : 0, ps = packed_from ? packed_from->S : 0;
   const size_t row_bytes = (size_t)cs.R * cs.S * cs.Cinp * sizeof(int);
   if (!packed_from && splits <= 16 && row_bytes <= 48 * 1024 && row_bytes >= 4096) {
-    finalize_bwd_filter_rows_kernel<<<(unsigned)cs.Cout, kThreads, row_bytes, st>>>(acc, splits, sX, s, cs, dW, dtype);
+    DAI8_RETURN_IF_CUDA(launch_dependent(finalize_bwd_filter_rows_kernel, dim3((unsigned)cs.Cout), dim3(kThreads), row_bytes, st, acc, splits, sX, s, cs, dW, dtype));
   } else {
     // enough groups to put some 150 thousand threads to work, as far as there are images to share out
     const int64_t quads = valid / 4;
     int groups = 1;
     while (groups < 8 && groups * 2 <= splits && quads * groups < 150000) groups *= 2;
     if (groups == 8)
-      finalize_bwd_filter_kernel<8><<<(unsigned)ceil_div64(quads, kThreads / 8), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+      DAI8_RETURN_IF_CUDA(launch_dependent(finalize_bwd_filter_kernel<8>, dim3((unsigned)ceil_div64(quads, kThreads / 8)), dim3(kThreads), 0, st, acc, splits, sX, s, cs, pc, pr, ps, dW, dtype));
     else if (groups == 4)
-      finalize_bwd_filter_kernel<4><<<(unsigned)ceil_div64(quads, kThreads / 4), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+      DAI8_RETURN_IF_CUDA(launch_dependent(finalize_bwd_filter_kernel<4>, dim3((unsigned)ceil_div64(quads, kThreads / 4)), dim3(kThreads), 0, st, acc, splits, sX, s, cs, pc, pr, ps, dW, dtype));
     else if (groups == 2)
-      finalize_bwd_filter_kernel<2><<<(unsigned)ceil_div64(quads, kThreads / 2), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+      DAI8_RETURN_IF_CUDA(launch_dependent(finalize_bwd_filter_kernel<2>, dim3((unsigned)ceil_div64(quads, kThreads / 2)), dim3(kThreads), 0, st, acc, splits, sX, s, cs, pc, pr, ps, dW, dtype));
     else
-      finalize_bwd_filter_kernel<1><<<(unsigned)ceil_div64(quads, kThreads), kThreads, 0, st>>>(acc, splits, sX, s, cs, pc, pr, ps, dW, dtype);
+      DAI8_RETURN_IF_CUDA(launch_dependent(finalize_bwd_filter_kernel<1>, dim3((unsigned)ceil_div64(quads, kThreads)), dim3(kThreads), 0, st, acc, splits, sX, s, cs, pc, pr, ps, dW, dtype));
   }
   note_launch();
   DAI8_RETURN_IF_CUDA(cudaGetLastError());

@@ -273,6 +273,8 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  grid_dependency_release();
+  grid_dependency_wait();   // everything above overlapped the tail of the previous kernel
 
   if (warp == 0) {
     if (lane == 0) {
@@ -631,8 +633,11 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   prm.out_elem_bytes = out_es;
   const bool identity_place = pb.oH == pb.P && pb.oW == pb.Q && pb.oh_step == 1 && pb.ow_step == 1 && pb.oh_off == 0 && pb.ow_off == 0;
   prm.tma_store = (identity_place && out.layout == DAI8_NHWC && (pb.Nout * out_es) % 16 == 0 && pb.Nout * out_es >= 128) ? 1 : 0;
-  const int stage_out_bytes = prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0;
   prm.b_resident = b_res <= 96 * 1024 ? 1 : 0;
+  // streamed weights make the operand ring the bottleneck (bytes in flight per SM): those layers
+  // give the epilogue's staging blocks to the ring and store straight from registers
+  if (!prm.b_resident) prm.tma_store = 0;
+  const int stage_out_bytes = prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0;
   const int stage_bytes = prm.G * (a_chunk + (prm.b_resident ? 0 : b_chunk));
   int stages = (smem_budget - stage_out_bytes - (prm.b_resident ? b_res : 0)) / stage_bytes;
   if (stages > 8) stages = 8;
@@ -691,9 +696,8 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   int ctas = sm_count();
   if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
   if (ctas > num_tiles) ctas = num_tiles;
-  igemm_kmajor_kernel<<<dim3((unsigned)ctas), kThreadsPersist, smem_bytes, st>>>(mapA, mapB, mapC, prm);
+  DAI8_RETURN_IF_CUDA(launch_dependent(igemm_kmajor_kernel, dim3((unsigned)ctas), dim3(kThreadsPersist), smem_bytes, st, mapA, mapB, mapC, prm));
   note_launch();
-  DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
 }
 
@@ -834,6 +838,8 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_slot;
+  grid_dependency_release();
+  grid_dependency_wait();   // everything above overlapped the tail of the previous kernel
 
   if (warp == 0) {
     if (lane == 0) {
@@ -1035,9 +1041,8 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   });
   if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
   const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
-  wgrad_mnmajor_kernel<<<grid, kThreadsIgemm, smem_bytes, st>>>(mapG, mapX, prm);
+  DAI8_RETURN_IF_CUDA(launch_dependent(wgrad_mnmajor_kernel, grid, dim3(kThreadsIgemm), smem_bytes, st, mapG, mapX, prm));
   note_launch();
-  DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;
 }
 

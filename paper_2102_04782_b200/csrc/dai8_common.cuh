@@ -23,6 +23,32 @@ dai8_status read_clear_device_status(int* host_status, cudaStream_t stream);
 // Device address of that status word on the current device (nullptr on failure).
 unsigned int* device_status_address();
 
+// Programmatic dependent launch.  A kernel launched with launch_dependent() may start while the
+// kernel before it on the stream is still running: its CTAs take the SM resources that become free
+// and run their set-up (barrier initialisation, tensor-memory allocation, descriptor prefetch), then
+// stop in grid_dependency_wait() until the earlier kernel has completed and its writes are visible.
+// Nothing that reads or writes global memory may come before that wait.  grid_dependency_release()
+// lets the NEXT kernel on the stream begin launching; it says nothing about memory.  Both are no-ops
+// in a kernel launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }

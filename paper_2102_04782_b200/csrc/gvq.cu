@@ -545,6 +545,8 @@ template <typename T, int VE>
 __global__ void __launch_bounds__(kThreads)
 quantize_flat_nearest_kernel(const T* __restrict__ x, int64_t nvec, const float* __restrict__ scale,
                              int8_t* __restrict__ q) {
+  grid_dependency_release();
+  grid_dependency_wait();
   const float inv = inv_scale(*scale);
   const int64_t stride = (int64_t)gridDim.x * kThreads;
 #pragma unroll 4
@@ -1554,6 +1556,8 @@ template <typename T, bool NHWC_IN>
 __global__ void __launch_bounds__(kSmallThreads)
 quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int absmax_mode, int stochastic,
                       uint32_t seed, float* __restrict__ scale, int8_t* __restrict__ q) {
+  grid_dependency_release();
+  grid_dependency_wait();
   __shared__ float s_part[kSmallThreads / 32];
   __shared__ float s_scale;
   const int tid = threadIdx.x;
@@ -1614,9 +1618,9 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
     int small_ctas = (int)ceil_div64(npix * Cp, 4 * kSmallThreads);
     if (small_ctas > 32) small_ctas = 32;
     if (layout == DAI8_NHWC)
-      quantize_small_kernel<T, true><<<small_ctas, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+      DAI8_RETURN_IF_CUDA(launch_dependent(quantize_small_kernel<T, true>, dim3((unsigned)small_ctas), dim3(kSmallThreads), 0, st, x, N, C, (int)HW, Cp, am, sr, seed, scale, q));
     else
-      quantize_small_kernel<T, false><<<small_ctas, kSmallThreads, 0, st>>>(x, N, C, (int)HW, Cp, am, sr, seed, scale, q);
+      DAI8_RETURN_IF_CUDA(launch_dependent(quantize_small_kernel<T, false>, dim3((unsigned)small_ctas), dim3(kSmallThreads), 0, st, x, N, C, (int)HW, Cp, am, sr, seed, scale, q));
     note_launch(1);
     DAI8_RETURN_IF_CUDA(cudaGetLastError());
     return DAI8_OK;
@@ -1638,7 +1642,7 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
   if (layout == DAI8_NHWC && !stoch && C == Cp) {
     const int64_t nvec = total / VEfull;      // C is a multiple of 16
     const int blocks = (int)(ceil_div64(nvec, kThreads * 4) < 2 * kMaxPixelBlocks ? ceil_div64(nvec, kThreads * 4) : 2 * kMaxPixelBlocks);
-    quantize_flat_nearest_kernel<T, VEfull><<<blocks, kThreads, 0, st>>>(x, nvec, scale, q);
+    DAI8_RETURN_IF_CUDA(launch_dependent(quantize_flat_nearest_kernel<T, VEfull>, dim3((unsigned)blocks), dim3(kThreads), 0, st, x, nvec, scale, q));
   } else if (layout == DAI8_NHWC) {
     if (C % VEfull == 0) {
       const NhwcGrid g = nhwc_grid(npix, Cp / VEfull);
