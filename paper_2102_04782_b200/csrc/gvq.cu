@@ -734,18 +734,21 @@ __device__ __noinline__ bool grid_barrier(uint32_t* counter, uint32_t target, un
                                           volatile uint32_t* abort_flag, uint32_t* s_ok) {
   consumer_sync();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(counter, 1u);
+    // release: the CTA's writes (ordered before this thread by the barrier above) become visible
+    // to whoever acquires the counter; acquire: the other CTAs' writes are visible after the loop
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(counter) : "memory");
     uint32_t ok = *abort_flag ? 0u : 1u;
     const long long t0 = clock64();
-    while (ok && *reinterpret_cast<volatile uint32_t*>(counter) < target) {
+    for (;;) {
+      uint32_t seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
+      if (!ok || seen >= target) break;
       if (clock64() - t0 > kWaitTimeoutCycles) {
         atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
         *abort_flag = 1u;
         ok = 0u;
       }
     }
-    __threadfence();
     *s_ok = ok;
   }
   consumer_sync();
