@@ -42,6 +42,23 @@ int packed_bwd_filter(const ConvShape& cs, ConvShape* pw) {
 }
 size_t packed_a_bytes(const ConvShape& cs, int Kp) { return up256((size_t)cs.N * cs.P * cs.Q * Kp); }
 
+// The input gradient of a stride-1 layer is the forward convolution of the gradient codes with the
+// mirrored, transposed filter.  With at most 16 output channels that forward problem has "few input
+// channels" and can take the packed pointwise route on the tensor cores.  Returns Kp (0: not applicable).
+int packed_bwd_data(const ConvShape& cs, ConvShape* as_fwd, ConvShape* pw) {
+  if (cs.Coutp != 16 || cs.sh != 1 || cs.sw != 1 || cs.ph > cs.R - 1 || cs.pw > cs.S - 1) return 0;
+  ConvShape f = cs;
+  f.Cin = cs.Cout; f.Cout = cs.Cin; f.Cinp = cs.Coutp; f.Coutp = cs.Cinp;
+  f.H = cs.P; f.W = cs.Q; f.P = cs.H; f.Q = cs.W;
+  f.ph = cs.R - 1 - cs.ph; f.pw = cs.S - 1 - cs.pw;
+  ConvShape tmp;
+  const int Kp = packed_fwd(f, &tmp);
+  if (Kp == 0) return 0;
+  if (as_fwd) *as_fwd = f;
+  if (pw) *pw = tmp;
+  return Kp;
+}
+
 }  // namespace
 }  // namespace dai8
 
@@ -57,7 +74,11 @@ extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geo
       const int Kp = umma_fwd_supported(cs) ? 0 : packed_fwd(cs, nullptr);
       return Kp ? packed_a_bytes(cs, Kp) + up256((size_t)cs.Coutp * Kp) + 256 : 256;
     }
-    case DAI8_OP_BWD_DATA: return (wt_bytes(cs) + 255) / 256 * 256 + 256;
+    case DAI8_OP_BWD_DATA: {
+      ConvShape f;
+      const int Kp = umma_bwd_data_supported(cs) ? 0 : packed_bwd_data(cs, &f, nullptr);
+      return up256(wt_bytes(cs)) + (Kp ? packed_a_bytes(f, Kp) + up256((size_t)f.Coutp * Kp) : 0) + 256;
+    }
     case DAI8_OP_BWD_FILTER: {
       // one int32 image, or one per pixel slice of the tensor-core kernel
       ConvShape pw;
@@ -118,6 +139,17 @@ extern "C" dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, co
   int8_t* wT = static_cast<int8_t*>(ws);
   const int mode = g_backend.load();
   if (mode != 1 && umma_bwd_data_supported(cs)) return umma_bwd_data(gq, qW, wT, gmax, sW, cs, out, st);
+  ConvShape f, pw;
+  if (const int Kp = mode != 1 ? packed_bwd_data(cs, &f, &pw) : 0) {
+    // few output channels: forward form of the input gradient on the packed pointwise route
+    int8_t* A = wT + up256(wt_bytes(cs));
+    int8_t* Wp = A + packed_a_bytes(f, Kp);
+    dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/1, st);   // [Cinp][R][S][Coutp], taps mirrored
+    if (r == DAI8_OK) r = pack_small_cin(gq, f, Kp, A, st);
+    if (r == DAI8_OK) r = pack_small_cin_weights(wT, f, Kp, Wp, st);
+    if (r != DAI8_OK) return r;
+    return umma_fwd(A, Wp, gmax, sW, pw, out, st);
+  }
   if (mode == 2) return DAI8_ERR_UNSUPPORTED;
   dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/0, st);
   if (r != DAI8_OK) return r;

@@ -25,6 +25,8 @@ GEOMS = [
     (1, 16, 16, 5, 7, 3, 5, (1, 2), (1, 2)),
     (2, 130, 70, 6, 6, 3, 3, 1, 1),         # channel counts that are not multiples of 16
     (1, 64, 128, 30, 30, 3, 3, 1, 1),       # several 128-pixel tiles with a ragged tail
+    (2, 32, 16, 20, 20, 1, 1, 1, 0),        # 16 output channels: input gradient in its packed forward form
+    (2, 40, 12, 13, 12, 3, 3, 1, 1),        # the same with a 3x3 filter and ragged channel counts
 ]
 
 
