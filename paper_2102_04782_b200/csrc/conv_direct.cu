@@ -233,6 +233,30 @@ pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* 
   reinterpret_cast<uint4*>(A)[t] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// Exactly 16 input channels: every tap of every pixel is one 16-byte vector of X.
+__global__ void __launch_bounds__(kThreads)
+pack_im2col_c16_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* __restrict__ A) {
+  grid_dependency_release();
+  grid_dependency_wait();
+  const int groups = Kp / 16, T = cs.R * cs.S;
+  const int64_t total = (int64_t)cs.N * cs.P * cs.Q * groups;
+  for (int64_t t = (int64_t)blockIdx.x * kThreads + threadIdx.x; t < total; t += (int64_t)gridDim.x * kThreads) {
+    const int tap = (int)(t % groups);
+    int64_t m = t / groups;
+    const int q = (int)(m % cs.Q); m /= cs.Q;
+    const int p = (int)(m % cs.P);
+    const int n = (int)(m / cs.P);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (tap < T) {
+      const int r = tap / cs.S, s = tap - r * cs.S;
+      const int h = p * cs.sh + r - cs.ph, x = q * cs.sw + s - cs.pw;
+      if (h >= 0 && h < cs.H && x >= 0 && x < cs.W)
+        v = *reinterpret_cast<const uint4*>(qX + (((int64_t)n * cs.H + h) * cs.W + x) * 16);
+    }
+    reinterpret_cast<uint4*>(A)[t] = v;
+  }
+}
+
 // The same matrix, one output row (n, p) per block: the R input rows it needs are first compacted to
 // their real channels in shared memory, where the S*Cin bytes of one filter row of one output pixel
 // are contiguous, so every input vector is fetched once per block and the rows of A' leave as
@@ -489,7 +513,11 @@ dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const 
 dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st) {
   const int rowpix = (cs.Q - 1) * cs.sw + cs.S;
   const int rowbytes = round_up(rowpix * cs.Cin, 4);
-  if ((size_t)cs.R * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
+  if (cs.Cin == 16) {
+    const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
+    const int64_t want = ceil_div64(total, kThreads * 4);
+    DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_c16_kernel, dim3((unsigned)(want < 148 * 16 ? want : 148 * 16)), dim3(kThreads), 0, st, qX, cs, Kp, A));
+  } else if ((size_t)cs.R * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
     DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_rows_kernel, dim3((unsigned)(cs.N * cs.P)), dim3(kThreads), (size_t)cs.R * rowbytes, st, qX, cs, Kp, rowpix, rowbytes, A));
   } else {
     const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);

@@ -384,7 +384,8 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const int quarter = warp & 3;
     const int half = (warp - 2) >> 2;
     const bool nhwc = prm.out.layout == DAI8_NHWC;
-    const bool vec_ok = nhwc && (prm.Nout & 15) == 0;
+    // 16-byte stores need the pixel rows to be 16-byte multiples: 8 bf16 or 4 fp32 / int32 channels
+    const bool vec_ok = nhwc && (prm.Nout % (prm.out_elem_bytes == 2 ? 8 : 4)) == 0;
     const size_t plane = (size_t)prm.oH * prm.oW;
     const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
     int tile_i = 0, n_store = 0;
@@ -476,12 +477,13 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           if (g == 1 && !second) break;
           const int (&v)[16] = va[g];
           const int j0 = n0 + col + g * 16;
-          if (vec_ok && j0 + 16 <= prm.Nout) {
+          if (vec_ok) {
+            const int nv = min(16, prm.Nout - j0);     // valid columns of this group: a multiple of 8 (bf16) or 4
             if (prm.out.dtype == DAI8_F32) {
               float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.out.ptr) + pix_base + j0);
 #pragma unroll
               for (int i = 0; i < 4; ++i)
-                dst[i] = make_float4(__fmul_rn(__int2float_rn(v[4 * i]), scale), __fmul_rn(__int2float_rn(v[4 * i + 1]), scale),
+                if (4 * i < nv) dst[i] = make_float4(__fmul_rn(__int2float_rn(v[4 * i]), scale), __fmul_rn(__int2float_rn(v[4 * i + 1]), scale),
                                      __fmul_rn(__int2float_rn(v[4 * i + 2]), scale), __fmul_rn(__int2float_rn(v[4 * i + 3]), scale));
             } else if (prm.out.dtype == DAI8_BF16) {
               uint32_t w[8];
@@ -490,11 +492,11 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
                 w[i] = pack_bf16x2(__fmul_rn(__int2float_rn(v[2 * i]), scale), __fmul_rn(__int2float_rn(v[2 * i + 1]), scale));
               uint4* dst = reinterpret_cast<uint4*>(static_cast<uint16_t*>(prm.out.ptr) + pix_base + j0);
               dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-              dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+              if (nv > 8) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
             } else {
               int4* dst = reinterpret_cast<int4*>(static_cast<int*>(prm.out.ptr) + pix_base + j0);
 #pragma unroll
-              for (int i = 0; i < 4; ++i) dst[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+              for (int i = 0; i < 4; ++i) if (4 * i < nv) dst[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
             }
           } else {
 #pragma unroll
