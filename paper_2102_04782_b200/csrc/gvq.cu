@@ -756,8 +756,9 @@ __device__ __noinline__ bool grid_barrier(uint32_t* counter, uint32_t target, un
 }
 
 // How the 512 consumer threads of a CTA tile (pixel row, vector column) pairs: with Gp <= 32 vector
-// columns a warp holds rows_per_warp = 32/Gp whole rows, otherwise the CTA holds rpi = 512/Gp rows.
-__host__ __device__ inline int fused_rows_per_iteration(int Gp) { return Gp <= 32 ? (kFT / 32) * (32 / Gp) : kFT / Gp; }
+// columns, Gp a divisor of 32, a warp holds rows_per_warp = 32/Gp whole rows; otherwise the CTA holds
+// rpi = 512/Gp rows that run across warp boundaries (only 512 mod Gp threads idle).
+__host__ __device__ inline int fused_rows_per_iteration(int Gp) { return (Gp <= 32 && 32 % Gp == 0) ? (kFT / 32) * (32 / Gp) : kFT / Gp; }
 
 // Combines, in a fixed order, what the consumer threads have stored per (vector element e, pixel
 // row lane, vector column) at index e*kFT + row*Gp + col over the row lanes, and writes the result for
@@ -928,7 +929,7 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   // ---------------- consumers ----------------------------------------------------------------------
   int col, rl;
   bool active;
-  if (a.rows_per_warp > 0) {       // Gp <= 32: a warp holds rows_per_warp whole rows
+  if (a.rows_per_warp > 0) {       // Gp divides 32: a warp holds rows_per_warp whole rows
     const int r = lane / Gp;
     col = lane - r * Gp;
     rl = warp * a.rows_per_warp + r;
@@ -1406,7 +1407,7 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   a.rpi = rpi;
   a.adv_q = (int)(rpi / a.HW);
   a.adv_rem = (int)(rpi % a.HW);
-  a.rows_per_warp = a.Gp <= 32 ? 32 / a.Gp : 0;
+  a.rows_per_warp = (a.Gp <= 32 && 32 % a.Gp == 0) ? 32 / a.Gp : 0;   // else rows run across warp boundaries
   int mult = kPieceBytes / (rpi * rb);
   if (mult < 1) mult = 1;
   a.rp = rpi * mult;

@@ -92,6 +92,7 @@ def test_config1_grad_quant(layout, bf16):
     (1, 3, 11, 13),     # tiny C, odd extents, misaligned NCHW rows
     (2, 2048, 2, 2),    # several column blocks
     (5, 96, 9, 9),
+    (3, 144, 10, 11),   # 18 bf16 vector columns: rows of the fused kernel run across warp boundaries
     (1, 1, 1, 1),
     (2, 16, 1, 300),
 ])
