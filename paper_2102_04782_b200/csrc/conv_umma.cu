@@ -807,7 +807,6 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
   __shared__ uint64_t full_bar[8], empty_bar[8], acc_bar;
   __shared__ uint32_t tmem_base_slot;
   __shared__ volatile uint32_t abort_flag;
-  __shared__ int tr[4][32][33];
 
   const int chunk_begin = blockIdx.x * prm.chunks_per_split;
   const int k_iters = min(prm.chunks_total, chunk_begin + prm.chunks_per_split) - chunk_begin;
@@ -902,8 +901,10 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
     const bool ok = mbar_wait(&acc_bar, 0, &abort_flag);
     tc_fence_after();
     if (ok) {
-      int (*trw)[33] = tr[warp - 2];
+      // Tensor-memory lane = output channel: every lane holds 32 consecutive input channels of its
+      // own row per pair of loads and writes them as eight 16-byte stores.
       int* part = prm.acc + (size_t)blockIdx.x * prm.acc_stride;   // this pixel slice's partial sums
+      const int co = co0 + quarter * 32 + lane;
       for (int tl = 0; tl < ntap; ++tl) {
         const int tap = tap_begin + tl;
         for (int cg = 0; cg < Nw / 32; ++cg) {
@@ -912,16 +913,14 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
           tmem_ld16(taddr, v0);
           tmem_ld16(taddr + 16, v1);
           tmem_ld_wait();
-          __syncwarp();
+          const int ci = ci0 + cg * 32;
+          if (co < prm.Cout && ci < prm.Cinp) {            // Cinp is a multiple of 16
+            int4* dst = reinterpret_cast<int4*>(part + ((size_t)co * T + tap) * prm.Cinp + ci);
 #pragma unroll
-          for (int i = 0; i < 16; ++i) { trw[lane][i] = v0[i]; trw[lane][16 + i] = v1[i]; }
-          __syncwarp();
-          const int ci = ci0 + cg * 32 + lane;
-          if (ci < prm.Cinp) {
-            for (int rr = 0; rr < 32; ++rr) {
-              const int co = co0 + quarter * 32 + rr;
-              if (co >= prm.Cout) break;
-              part[((size_t)co * T + tap) * prm.Cinp + ci] = trw[rr][lane];
+            for (int i = 0; i < 4; ++i) dst[i] = make_int4(v0[4 * i], v0[4 * i + 1], v0[4 * i + 2], v0[4 * i + 3]);
+            if (ci + 16 < prm.Cinp) {
+#pragma unroll
+              for (int i = 0; i < 4; ++i) dst[4 + i] = make_int4(v1[4 * i], v1[4 * i + 1], v1[4 * i + 2], v1[4 * i + 3]);
             }
           }
         }
