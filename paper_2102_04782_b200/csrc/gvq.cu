@@ -596,7 +596,7 @@ constexpr int kFT = 512;             // consumer threads per CTA (one CTA per SM
 constexpr int kFusedThreads = kFT + 32;  // plus the producer warp
 constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
 constexpr int kMaxSlots = 28;        // shared-memory pieces per CTA
-constexpr int kMaxRing = 4;
+constexpr int kMaxRing = 8;
 constexpr int kPieceBytes = 16384;
 constexpr long long kWaitTimeoutCycles = 2000000000LL;  // about one second
 
@@ -1421,7 +1421,7 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   if (slots > kMaxSlots) slots = kMaxSlots;
   if (slots > pieces) slots = pieces;
   a.slots = (int)slots;
-  a.ring_log2 = slots >= 8 ? 2 : (slots >= 4 ? 1 : 0);   // 4, 2 or 1 cycling pieces
+  a.ring_log2 = slots >= 10 ? 3 : (slots >= 8 ? 2 : (slots >= 4 ? 1 : 0));   // 8, 4, 2 or 1 cycling pieces
   {
     const double M = (double)a.npix;
     const double denom = a.mp.std_unbiased ? M - 1.0 : M;
