@@ -257,42 +257,71 @@ pack_im2col_c16_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8
   }
 }
 
-// The same matrix, one output row (n, p) per block: the R input rows it needs are first compacted to
-// their real channels in shared memory, where the S*Cin bytes of one filter row of one output pixel
-// are contiguous, so every input vector is fetched once per block and the rows of A' leave as
-// full 16-byte stores.
+// The same matrix, kPackRows output rows (n, p .. p+3) per block: the input rows they need are first
+// compacted to their real channels in shared memory, where the S*Cin bytes of one filter row of one
+// output pixel are contiguous, so every input vector is fetched once per block (neighbouring output
+// rows share most of their input rows) and the rows of A' leave as full 16-byte stores.
+constexpr int kPackRows = 4;
 __global__ void __launch_bounds__(kThreads)
 pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int rowpix, int rowbytes,
                         int8_t* __restrict__ A) {
   grid_dependency_release();
   grid_dependency_wait();
-  extern __shared__ uint8_t xrows[];                            // [R][rowbytes]
-  const int p = blockIdx.x % cs.P, n = blockIdx.x / cs.P;
-  for (int i = threadIdx.x; i < cs.R * rowpix; i += kThreads) {
-    const int r = i / rowpix, xi = i - r * rowpix;
-    const int h = p * cs.sh + r - cs.ph, x = xi - cs.pw;
-    uint4 v = make_uint4(0u, 0u, 0u, 0u);
-    if (h >= 0 && h < cs.H && x >= 0 && x < cs.W)
-      v = *reinterpret_cast<const uint4*>(qX + (((int64_t)n * cs.H + h) * cs.W + x) * 16);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    uint8_t* dst = xrows + r * rowbytes + xi * cs.Cin;
+  extern __shared__ uint8_t xrows[];                            // [(np-1)*sh + R][rowbytes]
+  const int pblocks = (cs.P + kPackRows - 1) / kPackRows;
+  const int n = blockIdx.x / pblocks, p0 = (blockIdx.x - n * pblocks) * kPackRows;
+  const int np = min(kPackRows, cs.P - p0);
+  const int nrows = (np - 1) * cs.sh + cs.R;
+  const int total_in = nrows * rowpix;
+#pragma unroll 1
+  for (int i0 = threadIdx.x; i0 < total_in; i0 += 4 * kThreads) {
+    uint32_t first[4];                                          // only channels 0..3 can be real when Cin <= 4
+    uint4 full[4];
+    int r[4], xi[4];
 #pragma unroll
-    for (int c = 0; c < 16; ++c)
-      if (c < cs.Cin) dst[c] = (uint8_t)(w[c >> 2] >> (8 * (c & 3)));
+    for (int u = 0; u < 4; ++u) {                               // four independent loads in flight
+      const int i = i0 + u * kThreads;
+      r[u] = i / rowpix; xi[u] = i - r[u] * rowpix;
+      const int h = p0 * cs.sh + r[u] - cs.ph, x = xi[u] - cs.pw;
+      full[u] = make_uint4(0u, 0u, 0u, 0u);
+      if (i < total_in && h >= 0 && h < cs.H && x >= 0 && x < cs.W) {
+        const int8_t* src = qX + (((int64_t)n * cs.H + h) * cs.W + x) * 16;
+        if (cs.Cin <= 4) full[u].x = *reinterpret_cast<const uint32_t*>(src);
+        else full[u] = *reinterpret_cast<const uint4*>(src);
+      }
+      first[u] = full[u].x;
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      if (i0 + u * kThreads >= total_in) break;
+      uint8_t* dst = xrows + r[u] * rowbytes + xi[u] * cs.Cin;
+      if (cs.Cin <= 4) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c)
+          if (c < cs.Cin) dst[c] = (uint8_t)(first[u] >> (8 * c));
+      } else {
+        const uint32_t w[4] = {full[u].x, full[u].y, full[u].z, full[u].w};
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if (c < cs.Cin) dst[c] = (uint8_t)(w[c >> 2] >> (8 * (c & 3)));
+      }
+    }
   }
   __syncthreads();
   const int groups = Kp / 16, SC = cs.S * cs.Cin, Kreal = cs.R * SC;
-  uint4* out = reinterpret_cast<uint4*>(A) + (int64_t)blockIdx.x * cs.Q * groups;
-  for (int i = threadIdx.x; i < cs.Q * groups; i += kThreads) {
-    const int q = i / groups, kg = i - q * groups;
+  uint4* out = reinterpret_cast<uint4*>(A) + ((int64_t)n * cs.P + p0) * cs.Q * groups;
+  const int per_row = cs.Q * groups;
+  for (int i = threadIdx.x; i < np * per_row; i += kThreads) {
+    const int pl = i / per_row, j = i - pl * per_row;
+    const int q = j / groups, kg = j - q * groups;
     int k = kg * 16;
     int r = k / SC, off = k - r * SC;
-    const uint8_t* src = xrows + q * cs.sw * cs.Cin;
+    const uint8_t* src = xrows + (pl * cs.sh) * rowbytes + q * cs.sw * cs.Cin;
     uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
-    for (int j = 0; j < 16; ++j, ++k) {
+    for (int jj = 0; jj < 16; ++jj, ++k) {
       if (k < Kreal) {
-        w[j >> 2] |= (uint32_t)src[r * rowbytes + off] << (8 * (j & 3));
+        w[jj >> 2] |= (uint32_t)src[r * rowbytes + off] << (8 * (jj & 3));
         if (++off == SC) { off = 0; ++r; }
       }
     }
@@ -517,8 +546,10 @@ dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t
     const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
     const int64_t want = ceil_div64(total, kThreads * 4);
     DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_c16_kernel, dim3((unsigned)(want < 148 * 16 ? want : 148 * 16)), dim3(kThreads), 0, st, qX, cs, Kp, A));
-  } else if ((size_t)cs.R * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
-    DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_rows_kernel, dim3((unsigned)(cs.N * cs.P)), dim3(kThreads), (size_t)cs.R * rowbytes, st, qX, cs, Kp, rowpix, rowbytes, A));
+  } else if ((size_t)((kPackRows - 1) * cs.sh + cs.R) * rowbytes <= 48 * 1024 && (int64_t)cs.N * cs.P < ((int64_t)1 << 31)) {
+    const int pblocks = (cs.P + kPackRows - 1) / kPackRows;
+    const size_t smem = (size_t)((kPackRows - 1) * cs.sh + cs.R) * rowbytes;
+    DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_rows_kernel, dim3((unsigned)(cs.N * pblocks)), dim3(kThreads), smem, st, qX, cs, Kp, rowpix, rowbytes, A));
   } else {
     const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
     DAI8_RETURN_IF_CUDA(launch_dependent(pack_im2col_kernel, dim3(blocks_for(total)), dim3(kThreads), 0, st, qX, cs, Kp, A));
