@@ -268,3 +268,64 @@ def test_unsupported_and_errors():
     with pytest.raises(api.Dai8Error) as e:
         api.conv_bwd_data(q, w, scalar(1), scalar(1), gg, out, api.NHWC, ws_bytes(16))
     assert e.value.code == api.ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("g", [(16, 64, 64, 56, 56, 3, 3, 1, 1), (16, 256, 64, 56, 56, 1, 1, 1, 0),
+                               (16, 128, 128, 28, 28, 3, 3, 2, 1)])
+def test_back_to_back_calls_match_synchronised_calls(g):
+    """The kernels of consecutive calls overlap on the device (a kernel's set-up starts while the
+    kernel before it drains).  A whole layer step -- quantize X and W, forward, gradient quantization,
+    weight and data gradient -- is run once with a device synchronisation after every call, then six
+    times back to back without any, alternating between two input sets that share every intermediate
+    buffer: a kernel that started reading before its producer had finished would pick up values of the
+    other input set.  The last iteration must reproduce the synchronised run bit for bit."""
+    from helpers import ws_bytes as wsb
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    gg = geom(*g)
+    P, Q = gg.P, gg.Q
+    Cip, Cop = api.padded_channels(Cin), api.padded_channels(Cout)
+    bf = torch.bfloat16
+    gen = torch.Generator(device="cuda").manual_seed(5)
+    sets = []
+    for k in range(2):
+        sets.append(((torch.randn((N, H, W, Cin), device="cuda", generator=gen) * (1 + k)).to(bf),
+                     (torch.randn((Cout, Cin, R, S), device="cuda", generator=gen) * 0.1 * (1 + k)).to(bf),
+                     (torch.randn((N, P, Q, Cout), device="cuda", generator=gen) * 1e-3 * (1 + k)).to(bf)))
+    qX = torch.empty((N, H, W, Cip), dtype=torch.int8, device="cuda")
+    qW = torch.empty((Cout, R, S, Cip), dtype=torch.int8, device="cuda")
+    vq = torch.empty((N, P, Q, Cop), dtype=torch.int8, device="cuda")
+    gq = torch.empty_like(vq)
+    sX, sW, gmax = scalar(0), scalar(0), scalar(0)
+    s_c = torch.zeros(Cout, device="cuda")
+    Y = torch.empty((N, P, Q, Cout), dtype=bf, device="cuda")
+    dX = torch.empty((N, H, W, Cin), dtype=bf, device="cuda")
+    dW = torch.empty((Cout, Cin, R, S), dtype=torch.float32, device="cuda")
+    ws_g = wsb(api.quantize_grad_workspace_bytes(Cout))
+    ws_f = wsb(max(16, api.conv_workspace_bytes(api.OP_FWD, gg)))
+    ws_d = wsb(api.conv_workspace_bytes(api.OP_BWD_DATA, gg))
+    ws_w = wsb(api.conv_workspace_bytes(api.OP_BWD_FILTER, gg))
+
+    def step(inputs, sync):
+        x, w, dy = inputs
+        calls = [
+            lambda: api.quantize_tensor(x, api.NHWC, N, Cin, H, W, api.SCALE_ABSMAX, sX, api.ROUND_NEAREST_EVEN, 0, qX),
+            lambda: api.quantize_tensor(w, api.NCHW, Cout, Cin, R, S, api.SCALE_ABSMAX, sW, api.ROUND_NEAREST_EVEN, 0, qW),
+            lambda: api.conv_fwd(qX, qW, sX, sW, gg, Y, api.NHWC, ws_f),
+            lambda: api.quantize_grad(dy, api.NHWC, N, Cout, P, Q, None, s_c, False, gmax, None, None, vq, gq, 9, ws_g),
+            lambda: api.conv_bwd_filter(qX, vq, sX, s_c, gg, dW, ws_w),
+            lambda: api.conv_bwd_data(gq, qW, gmax, sW, gg, dX, api.NHWC, ws_d),
+        ]
+        for c in calls:
+            c()
+            if sync:
+                torch.cuda.synchronize()
+
+    step(sets[0], sync=True)
+    want = [t.clone() for t in (qX, qW, Y, vq, gq, dW, dX, s_c)]
+    for it in range(6):
+        step(sets[(it + 1) % 2], sync=False)       # other set first, ends on input set 0
+    torch.cuda.synchronize()
+    names = ("qX", "qW", "Y", "vq", "gq", "dW", "dX", "s_c")
+    bad = [n for n, a, b in zip(names, want, (qX, qW, Y, vq, gq, dW, dX, s_c)) if not torch.equal(a, b)]
+    assert not bad, bad
+    assert api.get_device_status() == api.OK
