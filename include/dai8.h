@@ -22,6 +22,9 @@
  *   - Scratch memory is passed in (`ws`, `ws_bytes`); ask dai8_*_workspace_bytes for the size.
  *     Its contents are undefined between calls.  Calls that share a workspace must be ordered
  *     on one stream.
+ *   - Work enqueued on one stream takes effect in order, as usual.  Most kernels are launched as
+ *     programmatic dependents of the kernel before them on the stream: their set-up may run while
+ *     that kernel finishes, but they touch global memory only after it has completed.
  *   - Errors are return codes; arguments are checked on the host before anything is enqueued.
  *     A geometry the kernels do not cover returns DAI8_ERR_UNSUPPORTED: there is no CPU path.
  *   - Device-side waits are bounded.  A wait that runs out records DAI8_ERR_TIMEOUT in a device
