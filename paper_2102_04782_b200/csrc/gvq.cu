@@ -577,26 +577,29 @@ quantize_flat_nearest_kernel(const T* __restrict__ x, int64_t nvec, const float*
 //
 // Sweep 1 takes the statistics.  The per-CTA partial moments are combined once: channel c is
 // finished by one warp of CTA c mod gridDim.x (fixed order, hence deterministic), and after a second
-// barrier every CTA reads the finished |g|max and sigma.  Sweep 2 takes the density count (integer
-// atomics) AND writes the codes, with the clip value of the class it predicts for each channel; the
-// class that the count then yields is the one reported and the one the codes must match, so channels
-// with a wrong prediction are re-quantized in a fix-up sweep that only their threads take part in.
+// barrier every CTA reads the finished |g|max and sigma.  Sweep 2 takes the density count AND writes
+// the codes, with the clip value of the class it predicts for each channel.  The per-CTA partial
+// counts are summed the same distributed way after a third barrier; the class that the count yields
+// is the one reported and the one the codes must match, so the warp that classifies a channel flags
+// a wrong prediction, and after a fourth barrier the flagged channels are re-quantized in a fix-up
+// sweep that only their threads take part in.
 //
-// Two things bound this kernel, and neither is HBM.  (1) Instruction issue in phase 3: two
-// stochastic roundings per element, each with its own hash-derived uniform.  So bf16 inputs take
-// |g|max and the density count two elements at a time in packed bf16 arithmetic (both are exact
-// there), codes come out of a magic-number addition instead of a float-to-int conversion, and
-// tensors of fewer than 2^32 elements use 32-bit index arithmetic.  (2) Everything outside the three
-// loops runs exactly once per CTA, straight from a cold instruction cache, at roughly ten cycles per
-// instruction: the code between the loops is therefore kept SMALL rather than fast -- one
-// out-of-line reduction routine with run-time loops serves all four column reductions, binary64
-// division and square root are avoided (reciprocals come from the host), spin loops are out of line.
+// Two things bound this kernel, and neither is HBM.  (1) The integer/logic pipe in sweep 2, which
+// issues at half the rate of the floating-point pipes: every element needs a 32-bit hash, two
+// uniforms and two stochastic roundings.  So bf16 inputs take |g|max and the density count two
+// elements at a time in packed bf16 arithmetic (both are exact there), codes come out of a
+// magic-number addition instead of a float-to-int conversion, rows without large elements skip the
+// clamps and add in pairs, and tensors of fewer than 2^32 elements use 32-bit index arithmetic.
+// (2) Everything outside the loops runs exactly once per CTA, straight from a cold instruction
+// cache, at roughly ten cycles per instruction: the code between the loops is therefore kept SMALL
+// rather than fast -- out-of-line reduction routines with run-time loops, no binary64 division or
+// square root (reciprocals come from the host), spin loops out of line.
 // ------------------------------------------------------------------------------------------------
 constexpr int kFT = 512;             // consumer threads per CTA (one CTA per SM)
 constexpr int kFusedThreads = kFT + 32;  // plus the producer warp
 constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
 constexpr int kMaxSlots = 28;        // shared-memory pieces per CTA
-constexpr int kMaxRing = 8;
+constexpr int kMaxRing = 8;          // of which at most this many cycle when not all pieces fit
 constexpr int kPieceBytes = 16384;
 constexpr long long kWaitTimeoutCycles = 2000000000LL;  // about one second
 
