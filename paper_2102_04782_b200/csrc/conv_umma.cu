@@ -9,10 +9,16 @@
 // K-major swizzled layout the MMA descriptors name.  For the input gradient A is q(G) and B the
 // transposed, tap-mirrored weights, with padding R-1-pad.
 //
-// Roles inside a CTA of 192 threads: warp 0 issues TMA loads, warp 1 owns the tensor memory and
-// issues the MMAs (one elected lane), warps 2-5 read the accumulators back (tcgen05.ld), apply the
+// Roles inside a CTA: warp 0 issues TMA loads, warp 1 owns the tensor memory and issues the MMAs
+// (one elected lane), the remaining warps (eight in the persistent forward / input-gradient kernel,
+// four in the weight-gradient kernel) read the accumulators back (tcgen05.ld), apply the
 // de-quantization scale and store.  Stages are handed over with mbarriers; every wait is bounded
 // and a wait that expires records DAI8_ERR_TIMEOUT in the device status word instead of hanging.
+//
+// Measured tcgen05 rates that shaped the tiling (operands resident in shared memory, nothing else
+// running): one kind::i8 MMA of M = 128, K = 32 takes 128 cycles with N = 256 and never less than 73
+// cycles whatever N, and M = 64 costs what M = 128 costs.  Hence tiles as wide as the output allows
+// (up to 256 columns), and in the weight gradient several filter taps side by side in one MMA.
 #include <cuda.h>
 
 #include <cstring>
@@ -871,8 +877,8 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
     if (lane == 0) {
       // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128.  The
       // boxes of consecutive taps lie side by side in shared memory and in tensor memory, so one
-      // MMA covers as many of them as fit N <= 256: an instruction costs about the same whether it
-      // is 64 or 256 columns wide (the 128-row operand is fetched once per instruction).
+      // MMA covers as many of them as fit N <= 256: an instruction of 64 columns takes 73 cycles,
+      // one of 256 columns 128.
       const int nbox = ntap * prm.nb;              // boxes of bw channels in this CTA's stage
       const int per_mma = 256 / prm.bw;            // boxes per MMA
       bool ok = true;
