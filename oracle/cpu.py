@@ -101,8 +101,10 @@ def rand_bits(seed: int, stream: int, index: int) -> int:
     return int(lib().dai8o_rand_bits(seed & 0xFFFFFFFF, stream, index))
 
 
-def quantize(x, scale, stochastic: bool = False, seed: int = 0, stream: int = 0) -> np.ndarray:
-    """Eq. 1.  scale: scalar (layer-wide) or array [C] (per channel).  Returns NCHW int8 codes."""
+def quantize(x, scale, stochastic: bool = False, seed: int = 0, stream: int = 0, first_image: int = 0) -> np.ndarray:
+    """Eq. 1.  scale: scalar (layer-wide) or array [C] (per channel).  Returns NCHW int8 codes.
+    x may be images first_image .. first_image + N - 1 of a larger tensor: stochastic rounding draws
+    its numbers by the element's index in the whole tensor."""
     x = _f32(x)
     N, C, H, W = x.shape
     scale = np.atleast_1d(_f32(scale))
@@ -110,8 +112,8 @@ def quantize(x, scale, stochastic: bool = False, seed: int = 0, stream: int = 0)
     if per_channel:
         assert scale.shape == (C,)
     q = np.empty(x.shape, np.int8)
-    lib().dai8o_quantize(_p(x), N, C, H, W, _p(scale), int(per_channel), int(stochastic),
-                         ctypes.c_uint32(seed & 0xFFFFFFFF), ctypes.c_uint32(stream), _p(q))
+    lib().dai8o_quantize_at(_p(x), N, C, H, W, ctypes.c_int64(first_image), _p(scale), int(per_channel),
+                            int(stochastic), ctypes.c_uint32(seed & 0xFFFFFFFF), ctypes.c_uint32(stream), _p(q))
     return q
 
 

@@ -187,18 +187,26 @@ static inline int8_t quantize_one(float x, float s, int round_mode, uint32_t see
   return (int8_t)q;
 }
 
-void dai8o_quantize(const float* x, int N, int C, int H, int W, const float* scale,
-                    int per_channel, int round_mode, uint32_t seed, uint32_t stream, int8_t* q) {
+// x holds images first_image .. first_image + N - 1 of a larger NCHW tensor: the generator's counter
+// is the element's index in that whole tensor (first_image = 0: x is the whole tensor).
+void dai8o_quantize_at(const float* x, int N, int C, int H, int W, int64_t first_image, const float* scale,
+                       int per_channel, int round_mode, uint32_t seed, uint32_t stream, int8_t* q) {
   std::fesetround(FE_TONEAREST);
   const int64_t HW = (int64_t)H * W;
+  const uint64_t offset = (uint64_t)first_image * (uint64_t)C * (uint64_t)HW;
 #pragma omp parallel for schedule(static) collapse(2)
   for (int n = 0; n < N; ++n)
     for (int c = 0; c < C; ++c) {
       const float s = per_channel ? scale[c] : scale[0];
       const int64_t base = ((int64_t)n * C + c) * HW;
       for (int64_t i = 0; i < HW; ++i)
-        q[base + i] = quantize_one(x[base + i], s, round_mode, seed, stream, (uint64_t)(base + i));
+        q[base + i] = quantize_one(x[base + i], s, round_mode, seed, stream, offset + (uint64_t)(base + i));
     }
+}
+
+void dai8o_quantize(const float* x, int N, int C, int H, int W, const float* scale,
+                    int per_channel, int round_mode, uint32_t seed, uint32_t stream, int8_t* q) {
+  dai8o_quantize_at(x, N, C, H, W, 0, scale, per_channel, round_mode, seed, stream, q);
 }
 
 // De-quantizer of Eq. 1: x_hat = q * s / 127 (binary32: (float)q * (s / 127)).

@@ -195,3 +195,46 @@ def test_config2_full_size_grad_quant():
     g, _, _ = synth.channel_mixed_grad(64, 64, 56, 56, seed=9)
     g = synth.round_to_bf16(g)
     check_grad_quant(g, True, api.NHWC, iters=2)
+
+
+def test_more_than_2_32_elements():
+    """A gradient with more than 2^32 elements (4097 x 128 x 128 x 64, 8.6 GB in bf16) takes the fused
+    kernel's 64-bit index arithmetic, and the generator's key then depends on the high half of the
+    element index.  All images but the last are zero, so everything the oracle needs -- |g|max, the
+    density count, the codes of the last image, whose element indices lie beyond 2^32 -- follows
+    from the last image alone; every other code must be 0."""
+    N, C, H, W = 4097, 64, 128, 128
+    M = N * H * W
+    last, _, _ = synth.channel_mixed_grad(1, C, H, W, seed=31)
+    last = synth.round_to_bf16(last)
+    dY = torch.zeros((N, H, W, C), dtype=torch.bfloat16, device="cuda")
+    dY[N - 1] = torch.from_numpy(last[0].transpose(1, 2, 0).copy()).cuda().to(torch.bfloat16)
+    vq = torch.full((N, H, W, C), 77, dtype=torch.int8, device="cuda")
+    gq = torch.full((N, H, W, C), 77, dtype=torch.int8, device="cuda")
+    s_state = torch.zeros(C, device="cuda"); gmax = torch.zeros(1, device="cuda")
+    stats = torch.zeros(C, 4, device="cuda"); cls = torch.zeros(C, dtype=torch.uint8, device="cuda")
+    ws = torch.empty(api.quantize_grad_workspace_bytes(C), dtype=torch.uint8, device="cuda")
+    seed = 12
+    api.quantize_grad(dY, api.NHWC, N, C, H, W, None, s_state, False, gmax, stats, cls, vq, gq, seed, ws)
+    torch.cuda.synchronize()
+    assert api.get_device_status() == api.OK
+    assert int(torch.count_nonzero(vq[: N - 1]).item()) == 0 and int(torch.count_nonzero(gq[: N - 1]).item()) == 0
+    st = stats.cpu().numpy()
+    absmax, _, _, gl = O.channel_stats(last)
+    np.testing.assert_array_equal(st[:, 0], absmax)
+    assert float(gmax.item()) == gl
+    # moments over all M pixels from the last image's (binary64): the zeros only enter through M
+    x = last[0].reshape(C, -1).astype(np.float64)
+    mean = x.sum(axis=1) / M
+    sigma = np.sqrt(np.maximum((x * x).sum(axis=1) / M - mean * mean, 0.0))
+    np.testing.assert_allclose(st[:, 2], sigma, rtol=REL, atol=0)
+    cnt = O.density_count(last, st[:, 2])          # zeros never exceed a positive sigma
+    np.testing.assert_array_equal(st[:, 3], (cnt.astype(np.float64) / M).astype(np.float32))
+    s_or, cls_or = O.classify_clip(cnt, absmax, M, s_prev=None)
+    np.testing.assert_array_equal(cls.cpu().numpy(), cls_or)
+    s_gpu = s_state.cpu().numpy()
+    np.testing.assert_allclose(s_gpu, s_or, rtol=REL, atol=0)
+    got_v = vq[N - 1].cpu().numpy().transpose(2, 0, 1)[None]
+    got_g = gq[N - 1].cpu().numpy().transpose(2, 0, 1)[None]
+    np.testing.assert_array_equal(got_v, O.quantize(last, s_gpu, True, seed, 0, first_image=N - 1))
+    np.testing.assert_array_equal(got_g, O.quantize(last, gl, True, seed, 1, first_image=N - 1))

@@ -265,3 +265,20 @@ def test_layout_of_global_vs_vector_scale():
     np.testing.assert_array_equal(qg.ravel(), np.rint(np.arange(-8, 8) * 127 / 8.0).clip(-127, 127))
     qv = O.quantize(x, np.abs(x).max(axis=(0, 2, 3)))
     assert np.all(np.abs(qv).max(axis=(0, 2, 3)) == 127)
+
+
+def test_quantize_slice_of_a_larger_tensor():
+    """first_image only moves the generator's counter: the codes of images 2..3 of a tensor equal the
+    codes of those two images quantized on their own with first_image = 2, and differ without it."""
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((4, 5, 3, 7)).astype(np.float32)
+    s = np.abs(x).max(axis=(0, 2, 3))
+    whole = O.quantize(x, s, True, 11, 0)
+    part = O.quantize(x[2:4], s, True, 11, 0, first_image=2)
+    np.testing.assert_array_equal(whole[2:4], part)
+    assert np.any(O.quantize(x[2:4], s, True, 11, 0) != part)
+    # beyond 2^32 elements the high half of the index enters the key: one element against the scalar generator
+    big = O.quantize(x[:1, :1, :1, :1], s[:1], True, 11, 1, first_image=1 << 33)
+    u = O.rand_uniform(11, 1, (1 << 33) * 5 * 21)
+    v = np.float32(np.float32(x[0, 0, 0, 0]) * np.float32(np.float32(127.0) / s[0]))
+    assert int(big[0, 0, 0, 0]) == min(127, int(np.floor(np.float32(v + np.float32(u)))))
