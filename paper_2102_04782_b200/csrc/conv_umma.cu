@@ -774,6 +774,7 @@ IgemmProblem dgrad_class_problem(const int8_t* gq, const int8_t* wT, const ConvS
 // de-quantizing kernel adds the slices in a fixed order: a hundred-odd CTAs adding into one small
 // image with atomics took longer to drain in L2 than the whole contraction.
 // ---------------------------------------------------------------------------------------------
+constexpr int kWgradSmem = 222 * 1024;   // operand ring of the weight-gradient kernel
 constexpr int kKP = 128;  // pixels per pipeline stage (4 MMAs of K = 32); 256 where the stage is small
 
 struct WgradParams {
@@ -973,7 +974,13 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
   const int T = cs.R * cs.S;
   const int b_tap_bytes = prm.nb * kKP * prm.bw;
   int tg_max = 512 / Nw;
-  const int tg_smem = (100 * 1024 - kKP * 128) / b_tap_bytes;
+  // Many pixels per slice: fat stages (several taps share the gradient tile, two stages in flight)
+  // are fastest, the MMA phase dominates.  Few pixels (28x28 and below at batch 64): the partial
+  // images dominate, and fewer taps per CTA mean fewer pixel slices, i.e. fewer partial images, and
+  // four lighter stages in flight.  Measured on the VGG-16 / ResNet-50 shapes.
+  const int stage_cap = prm.npix >= 100000 ? 100 * 1024 : 56 * 1024;
+  int tg_smem = (stage_cap - kKP * 128) / b_tap_bytes;
+  if (tg_smem < 1) tg_smem = 1;
   if (tg_max > tg_smem) tg_max = tg_smem;
   if (tg_max < 1) return 0;
   const int ngroups = (T + tg_max - 1) / tg_max;
@@ -984,8 +991,8 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
   // pixels per stage (halving the stage to 64 pixels where it is large made things slower).
   prm.kp = kKP;
   int stage_bytes = kKP * 128 + prm.tg * b_tap_bytes;
-  if ((200 * 1024) / (2 * stage_bytes) >= 3 && prm.npix >= 8 * 256) { prm.kp = 256; stage_bytes *= 2; }
-  int stages = (200 * 1024) / stage_bytes;
+  if ((kWgradSmem) / (2 * stage_bytes) >= 3 && prm.npix >= 8 * 256) { prm.kp = 256; stage_bytes *= 2; }
+  int stages = kWgradSmem / stage_bytes;
   if (stages > 8) stages = 8;
   prm.chunks_total = (prm.npix + prm.kp - 1) / prm.kp;
   const int co_tiles = (cs.Cout + kBM - 1) / kBM;
@@ -1044,7 +1051,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(attr_once, [] {
     attr_err = cudaFuncSetAttribute(wgrad_mnmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    227 * 1024 - 20 * 1024);
+                                    kWgradSmem + 1024);
   });
   if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
   const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
