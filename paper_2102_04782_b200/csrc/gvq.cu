@@ -1376,6 +1376,308 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Column-owner variant of the fused path, for gradients with many channels and few pixels (the deep
+// stages of ResNet-50 / MobileNetV2 at 14x14 and 7x7).  There the pixel-partitioned kernel above is
+// bound by its cross-CTA reductions: 148 CTAs each hold a partial for every channel.  Here a CTA owns
+// whole vector columns (8 bf16 / 4 fp32 channels) with ALL their pixels, held in shared memory, so
+// |g|max, mean, sigma, the density count, the class and the clip value are CTA-local and exact
+// before a single code is written: no prediction, no fix-up.  Only the layer-wide |g|max needs the
+// grid: one atomic max per CTA and one grid barrier, which the density count overlaps.
+// ------------------------------------------------------------------------------------------------
+constexpr int kColMaxLocal = 4;      // vector columns per CTA
+
+struct ColArgs {
+  int64_t npix, HW;
+  double inv_M, inv_denom;
+  int C, Cp, G, Gp;
+  int cols_per_cta;
+  uint32_t* gmax_bits;
+  uint32_t* gridbar;
+  const float* sigma_override;
+  McsDev mp;
+  float* s_state;
+  int has_prev;
+  float* gmax_layer;
+  float* stats_out;
+  uint8_t* cls;
+  uint32_t seed;
+  int8_t* q1;
+  int8_t* q2;
+  unsigned int* status;
+};
+
+// Eight bf16 elements (one vector) with 32-bit element indices, none of them large enough for a clamp
+// to act: the clamp-free form of the stochastic quantizer with paired additions (see the sweep of
+// the pixel-partitioned kernel for the argument).
+template <bool DUAL>
+__device__ __forceinline__ void quantize_vec8_unclipped(const uint4& raw, const float (&inv1)[8], float inv2, uint32_t idx,
+                                                        uint32_t HW, uint32_t keyx0, uint32_t (&ra)[8], uint32_t (&rb)[8]) {
+  const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
+  const uint64_t minus1 = f32x2_pack(0xBF800000u, 0xBF800000u), magic = f32x2_pack(0x4B400000u, 0x4B400000u);
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    const uint32_t h0 = sr_hash_folded(idx, keyx0);
+    idx += HW;
+    const uint32_t h1 = sr_hash_folded(idx, keyx0);
+    idx += HW;
+    const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
+    const uint64_t v1 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv1[2 * j])), __float_as_uint(__fmul_rn(g1, inv1[2 * j + 1])));
+    const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0, 0x7Fu, 9), __funnelshift_r(h1, 0x7Fu, 9)), minus1);
+    f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v1, u1), magic), ra[2 * j], ra[2 * j + 1]);
+    if (DUAL) {
+      const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0 * 0x9E3779B1u, 0x7Fu, 9),
+                                                  __funnelshift_r(h1 * 0x9E3779B1u, 0x7Fu, 9)), minus1);
+      const uint64_t v2 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv2)), __float_as_uint(__fmul_rn(g1, inv2)));
+      f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v2, u2), magic), rb[2 * j], rb[2 * j + 1]);
+    }
+  }
+}
+
+template <typename T, int VE, bool DUAL>
+__global__ void __launch_bounds__(kFT, 1)
+gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
+  extern __shared__ __align__(16) uint8_t csmem[];
+  __shared__ double red_d[kFT / 32][2 * VE];     // per warp: sum and sum of squares of every channel
+  __shared__ float red_f[kFT / 32][VE];          // per warp: |g|max
+  __shared__ uint32_t red_u[kFT / 32][VE];       // per warp: density count
+  __shared__ float ch_inv[kColMaxLocal][VE], ch_sig[kColMaxLocal][VE];
+  __shared__ volatile uint32_t s_abort;
+  __shared__ uint32_t s_ok;
+  using Idx = uint64_t;
+  const int tid = threadIdx.x;
+  const int C = a.C, G = a.G;
+  const int npix = (int)a.npix;                       // at most a few ten thousand (host check)
+  uint4* cols = reinterpret_cast<uint4*>(csmem);      // [local column][pixel]
+  if (tid == 0) s_abort = 0u;
+  const float tcoef = __fsub_rn(1.0f, __fmul_rn(a.mp.k, a.mp.A));
+  const double thr = (double)a.mp.lambda * (double)a.npix;
+
+  // ---- load the columns, statistics, density count, class and clip: all local -------------------
+#pragma unroll 1
+  for (int lc = 0; lc < a.cols_per_cta; ++lc) {
+    const int col = blockIdx.x + lc * gridDim.x;
+    if (col >= G) break;                              // padding columns hold no input
+    const int c0 = col * VE;
+    uint4* mine = cols + (size_t)lc * npix;
+    float piv[VE], amax[VE], fs[VE], fss[VE];
+    load_vec<T, VE>(x + c0, piv);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { amax[e] = 0.f; fs[e] = 0.f; fss[e] = 0.f; }
+    double ds[VE], dss[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { ds[e] = 0.0; dss[e] = 0.0; }
+    int run = 0;
+#pragma unroll 4
+    for (int p = tid; p < npix; p += kFT) {
+      const uint4 raw = *reinterpret_cast<const uint4*>(x + (size_t)p * C + c0);
+      mine[p] = raw;
+      float v[VE];
+      unpack_raw(raw, v, (const T*)nullptr);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) {
+        amax[e] = fmaxf(amax[e], fabsf(v[e]));
+        const float d = v[e] - piv[e];
+        fs[e] += d;
+        fss[e] = fmaf(d, d, fss[e]);
+      }
+      if (++run == 32) {
+        run = 0;
+#pragma unroll
+        for (int e = 0; e < VE; ++e) { ds[e] += (double)fs[e]; dss[e] += (double)fss[e]; fs[e] = 0.f; fss[e] = 0.f; }
+      }
+    }
+    // all channels of the vector at once: butterflies inside the warps, then thread e adds the sixteen
+    // warp results of channel e in warp order (fixed order: deterministic)
+#pragma unroll
+    for (int e = 0; e < VE; ++e) {
+      float m = amax[e];
+      double s1 = ds[e] + (double)fs[e], s2 = dss[e] + (double)fss[e];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+        s1 += __shfl_xor_sync(0xFFFFFFFFu, s1, o);
+        s2 += __shfl_xor_sync(0xFFFFFFFFu, s2, o);
+      }
+      if ((tid & 31) == 0) { red_f[tid >> 5][e] = m; red_d[tid >> 5][e] = s1; red_d[tid >> 5][VE + e] = s2; }
+    }
+    __syncthreads();
+    if (tid < VE) {
+      const int e = tid, c = c0 + e;
+      float mx = red_f[0][e];
+      double s1 = red_d[0][e], s2 = red_d[0][VE + e];
+#pragma unroll
+      for (int w = 1; w < kFT / 32; ++w) { mx = fmaxf(mx, red_f[w][e]); s1 += red_d[w][e]; s2 += red_d[w][VE + e]; }
+      const double pivot = (double)to_f32(x[c]);
+      const double md = s1 * a.inv_M;
+      double var = a.mp.center_mean ? (s2 - s1 * md) : (s2 + 2.0 * pivot * s1 + pivot * pivot * (double)a.npix);
+      var = fmax(var, 0.0) * a.inv_denom;
+      const float vf = (float)var;
+      const float sigma = (vf > 1e-30f || var == 0.0) ? sqrtf(vf) : sigma_wide(var);
+      ch_sig[lc][e] = a.sigma_override ? a.sigma_override[c] : sigma;
+      ch_inv[lc][e] = mx;                              // |g|max for now, the scale after the count
+      if (a.stats_out) {
+        a.stats_out[c * 4 + DAI8_STAT_ABSMAX] = mx;
+        a.stats_out[c * 4 + DAI8_STAT_MEAN] = (float)(pivot + md);
+        a.stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma;
+      }
+      if (mx > 0.f) atomicMax(a.gmax_bits, __float_as_uint(mx));
+    }
+    __syncthreads();
+  }
+
+  // density count on the resident columns (overlaps the other CTAs' way to the barrier)
+#pragma unroll 1
+  for (int lc = 0; lc < a.cols_per_cta; ++lc) {
+    const int col = blockIdx.x + lc * gridDim.x;
+    if (col >= G) break;
+    const int c0 = col * VE;
+    const uint4* mine = cols + (size_t)lc * npix;
+    float sg[VE];
+    uint32_t k[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) { sg[e] = ch_sig[lc][e]; k[e] = 0u; }
+#pragma unroll 4
+    for (int p = tid; p < npix; p += kFT) {
+      float v[VE];
+      unpack_raw(mine[p], v, (const T*)nullptr);
+#pragma unroll
+      for (int e = 0; e < VE; ++e) k[e] += (fabsf(v[e]) > sg[e]) ? 1u : 0u;
+    }
+#pragma unroll
+    for (int e = 0; e < VE; ++e) {
+      uint32_t n = k[e];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xFFFFFFFFu, n, o);
+      if ((tid & 31) == 0) red_u[tid >> 5][e] = n;
+    }
+    __syncthreads();
+    if (tid < VE) {
+      const int e = tid, c = c0 + e;
+      uint32_t cnt = 0u;
+#pragma unroll
+      for (int w = 0; w < kFT / 32; ++w) cnt += red_u[w][e];
+      const float gmax = ch_inv[lc][e];
+      const bool bell = (double)cnt > thr;
+      float s = gmax;
+      if (!bell) s = __fadd_rn(__fmul_rn(tcoef, a.has_prev ? a.s_state[c] : gmax), __fmul_rn(a.mp.A, gmax));
+      a.s_state[c] = s;
+      if (a.cls) a.cls[c] = bell ? 1 : 0;
+      if (a.stats_out) a.stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt * a.inv_M);
+      ch_inv[lc][e] = inv_scale(s);
+    }
+    __syncthreads();
+  }
+
+  // ---- the layer-wide scale needs every CTA's maximum --------------------------------------------
+  bool ok = true;
+  {
+    if (tid == 0) {
+      asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.gridbar) : "memory");
+      uint32_t good = 1u;
+      const long long t0 = clock64();
+      for (;;) {
+        uint32_t seen;
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.gridbar) : "memory");
+        if (seen >= gridDim.x) break;
+        if (clock64() - t0 > kWaitTimeoutCycles) {
+          atomicExch(a.status, (unsigned int)DAI8_ERR_TIMEOUT);
+          good = 0u;
+          break;
+        }
+      }
+      s_ok = good;
+    }
+    __syncthreads();
+    ok = s_ok != 0u;
+  }
+  if (!ok) return;
+  const float gmax_l = __uint_as_float(__ldcg(a.gmax_bits));
+  const float inv2 = inv_scale(gmax_l);
+  if (blockIdx.x == 0 && tid == 0) *a.gmax_layer = gmax_l;
+
+  // ---- codes --------------------------------------------------------------------------------------
+  const uint32_t key0 = sr_key(a.seed, 0u);
+  const Idx HWi = (Idx)a.HW;
+#pragma unroll 1
+  for (int lc = 0; lc < a.cols_per_cta; ++lc) {
+    const int col = blockIdx.x + lc * gridDim.x;
+    if (col >= a.Gp) break;
+    const int c0 = col * VE;
+    int8_t* o1 = a.q1 + c0;
+    int8_t* o2 = DUAL ? a.q2 + c0 : nullptr;
+    if (col >= G) {                                   // zero padding of the code rows
+      for (int p = tid; p < npix; p += kFT) {
+        if (VE == 8) {
+          *reinterpret_cast<uint2*>(o1 + (size_t)p * a.Cp) = make_uint2(0u, 0u);
+          if (DUAL) *reinterpret_cast<uint2*>(o2 + (size_t)p * a.Cp) = make_uint2(0u, 0u);
+        } else {
+          *reinterpret_cast<uint32_t*>(o1 + (size_t)p * a.Cp) = 0u;
+          if (DUAL) *reinterpret_cast<uint32_t*>(o2 + (size_t)p * a.Cp) = 0u;
+        }
+      }
+      continue;
+    }
+    const uint4* mine = cols + (size_t)lc * npix;
+    float inv1[VE];
+#pragma unroll
+    for (int e = 0; e < VE; ++e) inv1[e] = ch_inv[lc][e];
+    // bf16, fewer than 2^32 elements: packed bounds below which no clamp can act (126.6/inv, the
+    // smaller of the channel's and the layer's, rounded toward zero to bf16)
+    const bool small_idx = (uint64_t)a.npix * (uint64_t)C < ((uint64_t)1 << 32);
+    uint32_t cthr[4] = {0u, 0u, 0u, 0u};
+    if (VE == 8) {
+      const float lim2 = DUAL ? (inv2 > 0.f ? __fdiv_rn(126.6f, inv2) : 3.0e38f) : 3.0e38f;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const float l0 = fminf(inv1[(2 * j) % VE] > 0.f ? __fdiv_rn(126.6f, inv1[(2 * j) % VE]) : 3.0e38f, lim2);
+        const float l1 = fminf(inv1[(2 * j + 1) % VE] > 0.f ? __fdiv_rn(126.6f, inv1[(2 * j + 1) % VE]) : 3.0e38f, lim2);
+        cthr[j] = (__float_as_uint(l0) >> 16) | (__float_as_uint(l1) & 0xFFFF0000u);
+      }
+    }
+    const uint32_t keyx0 = key0 ^ (key0 >> 16);
+#pragma unroll 2
+    for (int p = tid; p < npix; p += kFT) {
+      const uint4 raw = mine[p];
+      float v[VE];
+      unpack_raw(raw, v, (const T*)nullptr);
+      const uint32_t n = (uint32_t)p / (uint32_t)a.HW;
+      const uint32_t hw = (uint32_t)p - n * (uint32_t)a.HW;
+      Idx idx = ((Idx)n * (Idx)C + (Idx)c0) * HWi + (Idx)hw;      // NCHW index of (n, c0, hw)
+      uint32_t ra[VE], rb[VE];
+      bool done = false;
+      if constexpr (VE == 8) {
+        if (small_idx) {
+          const uint32_t over = bf16x2_gt_one(raw.x & 0x7FFF7FFFu, cthr[0]) | bf16x2_gt_one(raw.y & 0x7FFF7FFFu, cthr[1]) |
+                                bf16x2_gt_one(raw.z & 0x7FFF7FFFu, cthr[2]) | bf16x2_gt_one(raw.w & 0x7FFF7FFFu, cthr[3]);
+          if (over == 0u) {
+            quantize_vec8_unclipped<DUAL>(raw, inv1, inv2, (uint32_t)idx, (uint32_t)a.HW, keyx0, ra, rb);
+            done = true;
+          }
+        }
+      }
+      if (!done) {
+#pragma unroll
+      for (int e = 0; e < VE; ++e) {
+        const uint32_t hi = (uint32_t)(idx >> 32);
+        const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
+        const uint32_t h = avalanche32((uint32_t)idx ^ key);
+        ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
+        if (DUAL) rb[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+        idx += HWi;
+      }
+      }
+      if (VE == 8) {
+        *reinterpret_cast<uint2*>(o1 + (size_t)p * a.Cp) = make_uint2(pack_codes4(ra[0], ra[1], ra[2], ra[3]), pack_codes4(ra[4 % VE], ra[5 % VE], ra[6 % VE], ra[7 % VE]));
+        if (DUAL) *reinterpret_cast<uint2*>(o2 + (size_t)p * a.Cp) = make_uint2(pack_codes4(rb[0], rb[1], rb[2], rb[3]), pack_codes4(rb[4 % VE], rb[5 % VE], rb[6 % VE], rb[7 % VE]));
+      } else {
+        *reinterpret_cast<uint32_t*>(o1 + (size_t)p * a.Cp) = pack_codes4(ra[0], ra[1], ra[2], ra[3]);
+        if (DUAL) *reinterpret_cast<uint32_t*>(o2 + (size_t)p * a.Cp) = pack_codes4(rb[0], rb[1], rb[2], rb[3]);
+      }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Host-side launch helpers
 // ------------------------------------------------------------------------------------------------
 struct FusedConfig {
@@ -1449,6 +1751,45 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   return DAI8_OK;
 }
 
+// Column-owner kernel: applicable when all pixels of a CTA's vector columns fit in shared memory.
+template <typename T, int VE>
+bool columns_plan(int64_t npix, int Gp, int* grid, int* cols_per_cta, size_t* smem) {
+  const FusedConfig& cfg = fused_config();
+  if (!cfg.coop || npix > 65536) return false;
+  int per = (Gp + cfg.sms - 1) / cfg.sms;
+  if (per > kColMaxLocal) return false;
+  const size_t bytes = (size_t)per * (size_t)npix * 16;
+  if (bytes + 8192 > cfg.smem_max) return false;      // static shared memory of the kernel: about 4 KB
+  *grid = (Gp + per - 1) / per;
+  *cols_per_cta = per;
+  *smem = bytes;
+  return true;
+}
+
+template <typename T, int VE>
+dai8_status launch_columns(const T* dY, ColArgs& a, bool dual, int grid, size_t smem, cudaStream_t st) {
+  const double M = (double)a.npix;
+  const double denom = a.mp.std_unbiased ? M - 1.0 : M;
+  a.inv_M = 1.0 / M;
+  a.inv_denom = denom > 0.0 ? 1.0 / denom : 0.0;
+  void* args[] = {(void*)&dY, (void*)&a};
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] {
+    const int lim = (int)fused_config().smem_max - 8192;
+    attr_err = cudaFuncSetAttribute(gvq_columns_kernel<T, VE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+    if (attr_err == cudaSuccess)
+      attr_err = cudaFuncSetAttribute(gvq_columns_kernel<T, VE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  });
+  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  if (dual)
+    DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)gvq_columns_kernel<T, VE, true>, dim3((unsigned)grid), dim3(kFT), args, smem, st));
+  else
+    DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)gvq_columns_kernel<T, VE, false>, dim3((unsigned)grid), dim3(kFT), args, smem, st));
+  note_launch(1);
+  return DAI8_OK;
+}
+
 template <typename T, int VE>
 dai8_status launch_fused_select(const T* dY, FusedArgs& a, bool dual, bool idx32, cudaStream_t st) {
   if (dual) return idx32 ? launch_fused<T, VE, true, true>(dY, a, st) : launch_fused<T, VE, true, false>(dY, a, st);
@@ -1498,6 +1839,28 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
   const float* sigma = sigma_override ? sigma_override : ws.sigma;
+  if (layout == DAI8_NHWC && C % VEfull == 0) {
+    // many channels, few pixels: whole vector columns per CTA (no cross-CTA reductions)
+    int grid = 0, per = 0;
+    size_t smem = 0;
+    const int Gp = Cp / VEfull;
+    const bool fits = columns_plan<T, VEfull>(npix, Gp, &grid, &per, &smem);
+    // Fits to measured times (microseconds, B200): the column kernel costs a fixed part plus its
+    // longest CTA's rows; the pixel-partitioned kernel a larger fixed part (four barriers), its
+    // cross-CTA reductions (per channel) and the elements.
+    const double t_columns = 9.0 + 3.4e-3 * (double)npix * per;
+    const double t_pixels = 18.0 + 0.019 * C + (double)npix * C / 1.2e6;
+    const bool wanted = t_columns < t_pixels;
+    if (fits && wanted) {
+      ColArgs a;
+      a.npix = npix; a.HW = HW; a.inv_M = 0.0; a.inv_denom = 0.0; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Gp;
+      a.cols_per_cta = per; a.gmax_bits = ws.gmax_bits; a.gridbar = ws.gridbar; a.sigma_override = sigma_override;
+      a.mp = mp; a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
+      a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
+      if (!a.status) return DAI8_ERR_CUDA;
+      return launch_columns<T, VEfull>(dY, a, gq != nullptr, grid, smem, st);
+    }
+  }
   if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
     FusedArgs a;
     a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Cp / VEfull;
