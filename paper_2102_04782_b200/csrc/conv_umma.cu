@@ -6,8 +6,11 @@
 // A[pixel(m) + offset(t)][k] * B[j][t][k].  A is an NHWC code tensor read with TMA in im2col mode
 // (128 consecutive output pixels per tile, padding filled with zeros by the copy engine), B the
 // weight codes [rows][taps][channels] read with a tiled TMA box; both land in shared memory in the
-// K-major swizzled layout the MMA descriptors name.  For the input gradient A is q(G) and B the
-// transposed, tap-mirrored weights, with padding R-1-pad.
+// K-major swizzled layout the MMA descriptors name.  For the input gradient A is q(G), the filter
+// taps are mirrored (padding R-1-pad) and the contraction runs over Cout, which is the strided index
+// of the stored weights [Cout][taps][Cinp]: B is then read in place as an MN-major operand (boxes of
+// kc output channels x 32/64/128 input channels), or, where the tile width is not a multiple of 32
+// channels, from a transposed K-major copy.
 //
 // Roles inside a CTA: warp 0 issues TMA loads, warp 1 owns the tensor memory and issues the MMAs
 // (one elected lane), the remaining warps (eight in the persistent forward / input-gradient kernel,
@@ -166,6 +169,18 @@ __device__ __forceinline__ void mma_i8_parts(uint32_t d_tmem, uint32_t a_lo, uin
       ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
       : "memory");
 }
+// The same with separate high words for A and B (B in another layout than A).
+__device__ __forceinline__ void mma_i8_parts2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                              uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "mov.b64 da, {%1, %2};\n\t"
+      "mov.b64 db, {%3, %4};\n\t"
+      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
                "r"(ncols) : "memory");
@@ -227,6 +242,10 @@ struct IgemmParams {
   int stages;
   int m_tiles, n_tiles;  // tiles of 128 pixels x BN channels; tile t = m_tile*n_tiles + n_tile
   int b_resident;        // the CTA's whole weight tile stays in shared memory (loaded once)
+  // B read straight from the forward weight layout [Cout][taps][Cinp] as an MN-major operand (input
+  // gradient: the contraction runs over Cout): b_nb boxes of kc rows x b_bw bytes per chunk, and the
+  // tap of the full filter that class tap (r, s) stands for is b_tap_base - r*b_tap_dr - s*b_tap_ds
+  int b_mn, b_bw, b_nb, b_tap_base, b_tap_dr, b_tap_ds;
   int tma_store;         // NHWC output rows are staged in shared memory and written with tile stores
   int out_elem_bytes;    // 2 (bf16) or 4 (fp32, int32)
   int sh, sw, lower_h, lower_w;  // pixel (p,q) reads input (lower_h + p*sh + r, lower_w + q*sw + s)
@@ -293,7 +312,15 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         for (int c = 0; c < total_chunks; ++c) {
           const int tap = c / prm.chunks_per_tap;
           const int k0 = (c - tap * prm.chunks_per_tap) * prm.kc_bytes;
-          tma_load_tile_3d(&mapB, &b_full, smem + (size_t)c * b_chunk_bytes, k0, tap, n0);
+          if (prm.b_mn) {
+            const int tr = tap / prm.S, ts = tap - tr * prm.S;
+            const int ftap = prm.b_tap_base - tr * prm.b_tap_dr - ts * prm.b_tap_ds;
+            for (int b = 0; b < prm.b_nb; ++b)
+              tma_load_tile_3d(&mapB, &b_full, smem + (size_t)c * b_chunk_bytes + (size_t)b * prm.kc_bytes * prm.b_bw,
+                               n0 + b * prm.b_bw, ftap, k0);
+          } else {
+            tma_load_tile_3d(&mapB, &b_full, smem + (size_t)c * b_chunk_bytes, k0, tap, n0);
+          }
         }
       }
       // A single thread drives the copy engine, so this loop is a latency chain: no integer
@@ -302,7 +329,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       const uint64_t pa = reinterpret_cast<uint64_t>(&mapA), pb = reinterpret_cast<uint64_t>(&mapB);
       const uint32_t ring_a = smem_u32(ring), full_a = smem_u32(&full_bar[0]);
       const int G = prm.G, S = prm.S, cpt = prm.chunks_per_tap, kc = prm.kc_bytes, nst = prm.stages, kit = prm.k_iters;
-      const bool resident = prm.b_resident != 0;
+      const bool resident = prm.b_resident != 0, b_mn = prm.b_mn != 0;
       int stage = 0;
       uint32_t phase = 0;            // parity of the current pass over the ring
       bool first_pass = true;        // nothing to wait for until the ring has wrapped once
@@ -329,7 +356,15 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           uint32_t sb = sa + (uint32_t)(G * a_chunk_bytes);
           for (int j = 0; j < nch; ++j, ++c) {
             tma_load_im2col_4d_a(pa, bar, sa, k0, cw, ch, img, (uint16_t)ss, (uint16_t)r);
-            if (!resident) tma_load_tile_3d_a(pb, bar, sb, k0, r * S + ss, n0);
+            if (!resident) {
+              if (b_mn) {
+                const int ftap = prm.b_tap_base - r * prm.b_tap_dr - ss * prm.b_tap_ds;
+                for (int b = 0; b < prm.b_nb; ++b)
+                  tma_load_tile_3d_a(pb, bar, sb + (uint32_t)(b * kc * prm.b_bw), n0 + b * prm.b_bw, ftap, k0);
+              } else {
+                tma_load_tile_3d_a(pb, bar, sb, k0, r * S + ss, n0);
+              }
+            }
             sa += (uint32_t)a_chunk_bytes; sb += (uint32_t)b_chunk_bytes;
             k0 += kc;
             if (++kchunk == cpt) { kchunk = 0; k0 = 0; if (++ss == S) { ss = 0; ++r; } }
@@ -342,14 +377,22 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      const uint32_t idesc = idesc_i8_kmajor(prm.BN);
+      const bool b_mn = prm.b_mn != 0;
+      const uint32_t idesc = idesc_i8_kmajor(prm.BN) | (b_mn ? (1u << 16) : 0u);
+      // MN-major B: the low descriptor word carries the distance between the boxes (one box =
+      // kc rows of b_bw bytes), a K slice of 32 rows lies 32 * b_bw bytes further
+      const uint32_t b_hi = b_mn ? kmajor_desc_hi(prm.b_bw) : kmajor_desc_hi(prm.kc_bytes);
+      const uint32_t b_lbo = b_mn ? ((uint32_t)(prm.kc_bytes * prm.b_bw) >> 4) << 16 : (1u << 16);
+      const uint32_t b_kstep = b_mn ? (uint32_t)(32 * prm.b_bw) >> 4 : 2u;
       bool ok = !prm.b_resident || mbar_wait(&b_full, 0, &abort_flag);
       int stage = 0, tile_i = 0;
       uint32_t phase = 0;
       const int kk_n = prm.kc_bytes / 32, G = prm.G, nst = prm.stages, kit = prm.k_iters;
       const bool resident = prm.b_resident != 0;
       const uint32_t dhi = kmajor_desc_hi(prm.kc_bytes);
-      const uint32_t ring_lo = kmajor_desc_lo(smem_u32(ring)), bres_lo = kmajor_desc_lo(smem_u32(smem));
+      const uint32_t ring_lo = kmajor_desc_lo(smem_u32(ring));
+      const uint32_t bres_lo = ((smem_u32(smem) & 0x3FFFFu) >> 4) | b_lbo;
+      const uint32_t lbo_fix = b_lbo - (1u << 16);   // turns a K-major low word into B's
       const uint32_t stage_step = (uint32_t)stage_bytes >> 4, a_step = (uint32_t)a_chunk_bytes >> 4,
                      b_step = (uint32_t)b_chunk_bytes >> 4;
       const uint32_t empty_a = smem_u32(&empty_bar[0]);
@@ -368,10 +411,10 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           tc_fence_after();
           const int nch = min(total_chunks - c, G);
           uint32_t a_lo = ring_lo + (uint32_t)stage * stage_step;
-          uint32_t b_lo = resident ? bres : a_lo + (uint32_t)G * a_step;
+          uint32_t b_lo = resident ? bres : a_lo + (uint32_t)G * a_step + lbo_fix;
           for (int j = 0; j < nch; ++j) {
             for (int kk = 0; kk < kk_n; ++kk) {
-              mma_i8_parts(d_tmem, a_lo + 2u * kk, b_lo + 2u * kk, dhi, idesc, accumulate);
+              mma_i8_parts2(d_tmem, a_lo + 2u * kk, dhi, b_lo + b_kstep * kk, b_hi, idesc, accumulate);
               accumulate = 1;
             }
             a_lo += a_step; b_lo += b_step;
@@ -588,6 +631,8 @@ struct IgemmProblem {
   int N, Hi, Wi, Kc, Brows;
   int P, Q, Nout, R, S, sh, sw, lower_h, lower_w;
   int oH, oW, oh_step, oh_off, ow_step, ow_off;   // output placement, see IgemmParams
+  // b_mn: B is the forward weight tensor [Bk][b_taps][Brows bytes] read as an MN-major operand
+  int b_mn = 0, Bk = 0, b_taps = 0, b_tap_base = 0, b_tap_dr = 0, b_tap_ds = 0;
 };
 
 bool igemm_supported(const IgemmProblem& pb) {
@@ -630,6 +675,10 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   const int noutp = round_up(pb.Nout, 16);
   prm.BN = noutp < 256 ? noutp : 256;
   if (noutp > 256 && noutp % 256 != 0 && noutp % 128 == 0) prm.BN = 128;
+  prm.b_mn = pb.b_mn; prm.b_tap_base = pb.b_tap_base; prm.b_tap_dr = pb.b_tap_dr; prm.b_tap_ds = pb.b_tap_ds;
+  prm.b_bw = prm.BN % 128 == 0 ? 128 : (prm.BN % 64 == 0 ? 64 : 32);
+  prm.b_nb = prm.BN / prm.b_bw;
+  if (pb.b_mn && prm.BN % 32 != 0) return DAI8_ERR_UNSUPPORTED;
   prm.tmem_cols = 32;
   while (prm.tmem_cols < 2 * prm.BN) prm.tmem_cols *= 2;
   prm.m_tiles = (prm.Mtot + kBM - 1) / kBM;
@@ -682,7 +731,18 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
-  {
+  if (pb.b_mn) {
+    // weights as stored for the forward pass: [Bk = Cout][taps][Brows = Cinp]; a box is kc output
+    // channels (the contraction) x b_bw input channels (N) of one tap
+    const cuuint64_t dims[3] = {(cuuint64_t)pb.Brows, (cuuint64_t)pb.b_taps, (cuuint64_t)pb.Bk};
+    const cuuint64_t strides[2] = {(cuuint64_t)pb.Brows, (cuuint64_t)pb.b_taps * pb.Brows};
+    const cuuint32_t box[3] = {(cuuint32_t)prm.b_bw, 1, (cuuint32_t)prm.kc_bytes};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
+                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.b_bw),
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
+  } else {
     const cuuint64_t dims[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)(pb.R * pb.S), (cuuint64_t)pb.Brows};
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.R * pb.S * pb.Kc};
     const cuuint32_t box[3] = {(cuuint32_t)prm.kc_bytes, 1, (cuuint32_t)prm.BN};
@@ -1088,11 +1148,30 @@ dai8_status umma_bwd_data(const int8_t* gq, const int8_t* qW, int8_t* wT, const 
     const size_t es = out.dtype == DAI8_BF16 ? 2 : 4;
     DAI8_RETURN_IF_CUDA(cudaMemsetAsync(out.ptr, 0, (size_t)cs.N * cs.H * cs.W * cs.Cin * es, st));
   }
-  dai8_status r = repack_weights_classes(qW, cs, dc, wT, st);
-  if (r != DAI8_OK) return r;
+  // With an output tile width that is a multiple of 32 channels the weights are read where they are,
+  // as an MN-major operand (the contraction index Cout is the strided one in [Cout][taps][Cinp]);
+  // otherwise they are first transposed into the class-ordered K-major buffer.
+  const int noutp = round_up(cs.Cin, 16);
+  int bn = noutp < 256 ? noutp : 256;
+  if (noutp > 256 && noutp % 256 != 0 && noutp % 128 == 0) bn = 128;
+  const bool in_place = bn % 32 == 0;
+  dai8_status r = DAI8_OK;
+  if (!in_place) {
+    r = repack_weights_classes(qW, cs, dc, wT, st);
+    if (r != DAI8_OK) return r;
+  }
   for (int i = 0; i < dc.n; ++i) {
-    if (dc.cls[i].Tr == 0) continue;
-    r = launch_igemm(dgrad_class_problem(gq, wT, cs, dc.cls[i]), gmax, sW, out, st);
+    const DgradClass& c = dc.cls[i];
+    if (c.Tr == 0) continue;
+    IgemmProblem pb = dgrad_class_problem(gq, wT, cs, c);
+    if (in_place) {
+      // class tap (tr, ts) is filter tap (r0 + sh*(Tr-1-tr), s0 + sw*(Ts-1-ts))
+      pb.B = qW; pb.b_mn = 1; pb.Bk = cs.Cout; pb.b_taps = cs.R * cs.S;
+      pb.b_tap_base = (c.r0 + cs.sh * (c.Tr - 1)) * cs.S + c.s0 + cs.sw * (c.Ts - 1);
+      pb.b_tap_dr = cs.sh * cs.S;
+      pb.b_tap_ds = cs.sw;
+    }
+    r = launch_igemm(pb, gmax, sW, out, st);
     if (r != DAI8_OK) return r;
   }
   return DAI8_OK;
