@@ -1024,7 +1024,9 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
   if (cs.Cinp >= 128) {
     prm.bw = 128;
     const int blocks128 = (cs.Cinp + 127) / 128;
-    prm.nb = (blocks128 % 2 == 0) ? 2 : 1;
+    // two boxes (N = 256) share the gradient tile; pointwise filters have so little work per pixel
+    // slice that more, narrower tiles (fewer slices, fewer partial images) are faster
+    prm.nb = (blocks128 % 2 == 0 && cs.R * cs.S > 1) ? 2 : 1;
   } else {
     prm.bw = cs.Cinp > 32 ? 64 : 32;
     prm.nb = 1;
