@@ -214,10 +214,11 @@ pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* 
   const int q = (int)(m % cs.Q); m /= cs.Q;
   const int p = (int)(m % cs.P);
   const int n = (int)(m / cs.P);
-  const int Kreal = cs.R * cs.S * cs.Cin;
+  const int cc = packed_channels(cs);                          // channels >= Cin of X hold zeros
+  const int Kreal = cs.R * cs.S * cc;
   uint32_t w[4] = {0u, 0u, 0u, 0u};
   int k = kg * 16;
-  int tap = k / cs.Cin, ci = k - tap * cs.Cin;
+  int tap = k / cc, ci = k - tap * cc;
   int r = tap / cs.S, s = tap - r * cs.S;
 #pragma unroll
   for (int j = 0; j < 16; ++j, ++k) {
@@ -227,7 +228,7 @@ pack_im2col_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int8_t* 
         const uint32_t v = (uint8_t)qX[(((int64_t)n * cs.H + h) * cs.W + x) * cs.Cinp + ci];
         w[j >> 2] |= v << (8 * (j & 3));
       }
-      if (++ci == cs.Cin) { ci = 0; if (++s == cs.S) { s = 0; ++r; } }
+      if (++ci == cc) { ci = 0; if (++s == cs.S) { s = 0; ++r; } }
     }
   }
   reinterpret_cast<uint4*>(A)[t] = make_uint4(w[0], w[1], w[2], w[3]);
@@ -268,6 +269,7 @@ pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int
   grid_dependency_release();
   grid_dependency_wait();
   extern __shared__ uint8_t xrows[];                            // [(np-1)*sh + R][rowbytes]
+  const int cc = packed_channels(cs);
   const int pblocks = (cs.P + kPackRows - 1) / kPackRows;
   const int n = blockIdx.x / pblocks, p0 = (blockIdx.x - n * pblocks) * kPackRows;
   const int np = min(kPackRows, cs.P - p0);
@@ -294,11 +296,9 @@ pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       if (i0 + u * kThreads >= total_in) break;
-      uint8_t* dst = xrows + r[u] * rowbytes + xi[u] * cs.Cin;
+      uint8_t* dst = xrows + r[u] * rowbytes + xi[u] * cc;
       if (cs.Cin <= 4) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-          if (c < cs.Cin) dst[c] = (uint8_t)(first[u] >> (8 * c));
+        *reinterpret_cast<uint32_t*>(dst) = first[u];         // channels >= Cin of X hold zeros
       } else {
         const uint32_t w[4] = {full[u].x, full[u].y, full[u].z, full[u].w};
 #pragma unroll
@@ -308,15 +308,34 @@ pack_im2col_rows_kernel(const int8_t* __restrict__ qX, ConvShape cs, int Kp, int
     }
   }
   __syncthreads();
-  const int groups = Kp / 16, SC = cs.S * cs.Cin, Kreal = cs.R * SC;
+  const int groups = Kp / 16, SC = cs.S * cc, Kreal = cs.R * SC;
   uint4* out = reinterpret_cast<uint4*>(A) + ((int64_t)n * cs.P + p0) * cs.Q * groups;
   const int per_row = cs.Q * groups;
+  if (cc == 4) {
+    // one 32-bit word per pixel: word j of the row of A' is pixel (r, s) = (j / S, j % S) of the window
+    const int T = cs.R * cs.S;
+    for (int i = threadIdx.x; i < np * per_row; i += kThreads) {
+      const int pl = i / per_row, j = i - pl * per_row;
+      const int q = j / groups, kg = j - q * groups;
+      int tap = kg * 4;
+      int r = tap / cs.S, s = tap - r * cs.S;
+      const uint8_t* src = xrows + (pl * cs.sh) * rowbytes + q * cs.sw * 4;
+      uint32_t w[4];
+#pragma unroll
+      for (int jj = 0; jj < 4; ++jj, ++tap) {
+        w[jj] = tap < T ? *reinterpret_cast<const uint32_t*>(src + r * rowbytes + s * 4) : 0u;
+        if (++s == cs.S) { s = 0; ++r; }
+      }
+      out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    return;
+  }
   for (int i = threadIdx.x; i < np * per_row; i += kThreads) {
     const int pl = i / per_row, j = i - pl * per_row;
     const int q = j / groups, kg = j - q * groups;
     int k = kg * 16;
     int r = k / SC, off = k - r * SC;
-    const uint8_t* src = xrows + (pl * cs.sh) * rowbytes + q * cs.sw * cs.Cin;
+    const uint8_t* src = xrows + (pl * cs.sh) * rowbytes + q * cs.sw * cc;
     uint32_t w[4] = {0u, 0u, 0u, 0u};
 #pragma unroll
     for (int jj = 0; jj < 16; ++jj, ++k) {
@@ -339,9 +358,10 @@ pack_weights_kernel(const int8_t* __restrict__ qW, ConvShape cs, int Kp, int8_t*
   if (t >= total) return;
   const int k = (int)(t % Kp), co = (int)(t / Kp);
   int8_t v = 0;
-  if (k < cs.R * cs.S * cs.Cin) {
-    const int tap = k / cs.Cin, ci = k - tap * cs.Cin;
-    v = qW[((int64_t)co * cs.R * cs.S + tap) * cs.Cinp + ci];
+  const int cc = packed_channels(cs);
+  if (k < cs.R * cs.S * cc) {
+    const int tap = k / cc, ci = k - tap * cc;
+    v = qW[((int64_t)co * cs.R * cs.S + tap) * cs.Cinp + ci];     // channels >= Cin of qW hold zeros
   }
   Wp[t] = v;
 }
@@ -439,9 +459,11 @@ finalize_bwd_filter_kernel(const int* __restrict__ acc, int splits, const float*
     if (pack_cin > 0) {
       // the images come from the packed pointwise form: `ci` is k' = (r*S + s)*Cin + ci of the real filter
       const int k = ci;
-      if (k >= pack_R * pack_S * pack_cin) continue;
-      const int tap = k / pack_cin;
-      ci = k - tap * pack_cin; r = tap / pack_S; ss = tap - r * pack_S;
+      const int cc = pack_cin <= 4 ? 4 : pack_cin;          // packed_channels of the real layer
+      if (k >= pack_R * pack_S * cc) continue;
+      const int tap = k / cc;
+      ci = k - tap * cc; r = tap / pack_S; ss = tap - r * pack_S;
+      if (ci >= pack_cin) continue;                         // word padding
       Cin = pack_cin; R = pack_R; S = pack_S;
     }
     store_result(dW, dtype, (((size_t)co * Cin + ci) * R + r) * S + ss, v[j], scale);
@@ -541,7 +563,7 @@ dai8_status repack_weights_classes(const int8_t* qW, const ConvShape& cs, const 
 
 dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st) {
   const int rowpix = (cs.Q - 1) * cs.sw + cs.S;
-  const int rowbytes = round_up(rowpix * cs.Cin, 4);
+  const int rowbytes = round_up(rowpix * packed_channels(cs), 4);
   if (cs.Cin == 16) {
     const int64_t total = (int64_t)cs.N * cs.P * cs.Q * (Kp / 16);
     const int64_t want = ceil_div64(total, kThreads * 4);

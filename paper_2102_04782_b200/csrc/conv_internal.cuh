@@ -92,11 +92,15 @@ dai8_status finalize_bwd_filter(const int* acc, int splits, const float* sX, con
                                 cudaStream_t st);
 
 // Layers with at most 16 input channels: A'[N*P*Q][Kp] gathers the real channels of all taps
-// (k' = (r*S+s)*Cin + ci, zero padded to Kp = multiple of 32), W'[Cout][Kp] likewise; the layer then
+// (k' = (r*S+s)*cc + ci with cc = packed_channels, zero padded to Kp = multiple of 32), W'[Cout][Kp]
+// likewise; the layer then
 // is a pointwise convolution with Kp input channels.
+// Channels per pixel in the gathered matrix: up to four real channels are kept as one 32-bit word
+// (the gather then moves whole words), more are kept as they are.
+__host__ __device__ inline int packed_channels(const ConvShape& cs) { return cs.Cin <= 4 ? 4 : cs.Cin; }
 inline int packed_small_cin(const ConvShape& cs, ConvShape* pw) {
   if (cs.Cinp != 16) return 0;
-  const int Kp = round_up(cs.R * cs.S * cs.Cin, 32);
+  const int Kp = round_up(cs.R * cs.S * packed_channels(cs), 32);
   if (Kp > 2048) return 0;
   if (pw) {
     *pw = cs;
