@@ -569,7 +569,7 @@ quantize_flat_nearest_kernel(const T* __restrict__ x, int64_t nvec, const float*
 //
 // A CTA owns a contiguous range of pixels, i.e. a contiguous byte range of dY.  One producer warp
 // streams that range into shared memory with bulk asynchronous copies (cp.async.bulk, completion on
-// mbarriers) in pieces of up to 16 KB; sixteen consumer warps work on the pieces.  As many pieces as
+// mbarriers) in pieces of up to 32 KB; sixteen consumer warps work on the pieces.  As many pieces as
 // fit stay resident for all sweeps, the rest cycles through a small ring and is fetched again in the
 // later sweeps (L2 hits for tensors of up to ~100 MB).  The producer runs ahead across sweep
 // boundaries, so the first pieces of the next sweep are already in flight while the CTAs meet at a
@@ -600,7 +600,7 @@ constexpr int kFusedThreads = kFT + 32;  // plus the producer warp
 constexpr int kFusedMaxC = 2048;     // per-channel scalars kept in shared memory
 constexpr int kMaxSlots = 28;        // shared-memory pieces per CTA
 constexpr int kMaxRing = 8;          // of which at most this many cycle when not all pieces fit
-constexpr int kPieceBytes = 16384;
+constexpr int kPieceBytes = 32768;
 constexpr long long kWaitTimeoutCycles = 2000000000LL;  // about one second
 
 // reduction scratch at the start of the dynamic shared memory: per consumer thread and vector
