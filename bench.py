@@ -1,17 +1,20 @@
 #!/usr/bin/env python
 """Benchmark of the dai8 hot path on one B200 (or N independent replicas, one per GPU).
 
-Workload: the ResNet-50 conv2_x bottleneck block (1x1 256->64, 3x3 64->64 pad 1, 1x1 64->256) at
-N=64, 56x56, bf16 NHWC inputs, synthetic tensors (X = ReLU(N(0,1)), He weights, per-channel
-bell-shaped / long-tailed dY).  One step = the whole path for the three layers: forward
-quantization of X and W, int8 forward conv, gradient vectorized quantization of dY (statistics,
-density count, clip update, vq + gq codes), int8 dW and dX convs with de-quantizing epilogues.
+Workload of the JSON line: the thirteen 3x3 convolutions of VGG-16 at N=64, 224x224 input, bf16 NHWC
+tensors -- the compute-bound configuration.  One step = the whole path for every layer: forward
+quantization of X and W and the int8 forward convolution, layer by layer; then, in reverse layer
+order, gradient vectorized quantization of dY (statistics, density count, clip update, vq + gq codes)
+and the int8 dW and dX convolutions with de-quantizing epilogues.  Inputs are synthetic
+(X = ReLU(N(0,1)), He weights, per-channel bell-shaped / long-tailed dY), drawn on the device.
 
 Prints ONE JSON line.  `value` = int8 backward-convolution throughput, 2*MACs(dX+dW) of the step
-divided by the time of the WHOLE step (quantization and the forward conv included), in TOPS, summed
-over ranks.  `detail` holds the per-call breakdown measured with CUDA events in a second pass of the same
-steps, `roofline` the dominant call, `e2e` the same metric with pinned-host inputs and outputs
-copied inside the timed region, `cpu_baseline` the CPU oracle on a bounded sample of the workload.
+divided by the time of the WHOLE step (quantization and the forward pass included), in TOPS, summed
+over ranks.  `roofline` describes the kernel with the largest share of the step, `detail` holds the
+per-call breakdown (a second pass with a CUDA event pair around every call) and the same totals for
+the other configurations (ResNet-50 conv2_x block, all 53 ResNet-50 convolutions, the 34 MobileNetV2
+pointwise convolutions), `e2e` the same metric with pinned-host inputs and outputs copied inside the
+timed region, `cpu_baseline` the CPU oracle on a bounded sample of the workload.
 """
 from __future__ import annotations
 
@@ -31,13 +34,18 @@ import numpy as np
 
 METRIC = "int8 conv-backward TOPS (dX+dW)"
 UNIT = "TOPS"
-WORKLOAD = "resnet50_conv2x_bottleneck_N64_56x56_bf16_nhwc"
-BATCH = 64
 SEED = 2024
 INT8_OVER_BF16 = 2.0   # nominal dense ratio 4.5 / 2.25 PFLOP/s
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant call's kernel, from the ncu
-# capture summarised in profiles/gvq_fused_nhwc_bf16_conv2x.md (bytes; None once the kernel changes)
-NCU_TRAFFIC = {"quantize_grad @ conv2_x.1x1b": 189.12e6 + 58.67e6}
+
+
+def workloads():
+    from paper_2102_04782_b200 import synth
+    return {
+        "vgg16": ("vgg16_13convs_N64_224x224_bf16_nhwc", synth.vgg16_convs, 64),
+        "resnet50": ("resnet50_53convs_N64_224x224_bf16_nhwc", synth.resnet50_convs, 64),
+        "mobilenetv2": ("mobilenetv2_34pointwise_N128_224x224_bf16_nhwc", synth.mobilenetv2_pointwise, 128),
+        "conv2x": ("resnet50_conv2x_bottleneck_N64_56x56_bf16_nhwc", synth.resnet50_conv2x_block, 64),
+    }
 
 
 def measured_peaks():
@@ -53,62 +61,71 @@ def measured_peaks():
 # ------------------------------------------------------------------------------------------------
 # CPU oracle arm (cpu_baseline leg and --impl reference)
 # ------------------------------------------------------------------------------------------------
-def oracle_step(inputs):
-    """The whole path for a list of (layer, x, w, g) with the CPU oracle, as it stands."""
+def oracle_layer_step(L, x, w, g):
+    """The whole path for one layer with the CPU oracle, as it stands."""
     from oracle import cpu as O
-    for L, x, w, g in inputs:
-        sx, sw = float(np.abs(x).max()), float(np.abs(w).max())
-        qx, qw = O.quantize(x, sx), O.quantize(w, sw)
-        O.dequant_acc(O.conv_fwd_acc(qx, qw, L.stride, L.pad)[0], sx, sw)
-        absmax, _, sigma, gl = O.channel_stats(g)
-        cnt = O.density_count(g, sigma)
-        s, _ = O.classify_clip(cnt, absmax, g.size // g.shape[1])
-        vq = O.quantize(g, s, True, SEED, 0)
-        gq = O.quantize(g, gl, True, SEED, 1)
-        O.dequant_acc(O.conv_bwd_filter_acc(qx, vq, (L.R, L.S), L.stride, L.pad)[0], sx, s)
-        O.dequant_acc(O.conv_bwd_data_acc(gq, qw, (L.H, L.W), L.stride, L.pad)[0], gl, sw)
+    sx, sw = float(np.abs(x).max()), float(np.abs(w).max())
+    qx, qw = O.quantize(x, sx), O.quantize(w, sw)
+    O.dequant_acc(O.conv_fwd_acc(qx, qw, L.stride, L.pad)[0], sx, sw)
+    absmax, _, sigma, gl = O.channel_stats(g)
+    cnt = O.density_count(g, sigma)
+    s, _ = O.classify_clip(cnt, absmax, g.size // g.shape[1])
+    vq = O.quantize(g, s, True, SEED, 0)
+    gq = O.quantize(g, gl, True, SEED, 1)
+    O.dequant_acc(O.conv_bwd_filter_acc(qx, vq, (L.R, L.S), L.stride, L.pad)[0], sx, s)
+    O.dequant_acc(O.conv_bwd_data_acc(gq, qw, (L.H, L.W), L.stride, L.pad)[0], gl, sw)
 
 
-def oracle_inputs(batch):
+def oracle_inputs(layers, batch):
     from paper_2102_04782_b200 import synth
-    out = []
-    for i, L in enumerate(synth.resnet50_conv2x_block()):
-        x, w, g, _, _ = synth.layer_inputs(L, batch, SEED + i, bf16=True)
-        out.append((L, x, w, g))
-    return out
+    return [(L,) + synth.layer_inputs(L, batch, SEED + i, bf16=True)[:3] for i, L in enumerate(layers)]
 
 
 def bwd_ops(layers, batch):
     return sum(2 * 2 * L.macs(batch) for L in layers)   # dX + dW, 2 ops per MAC
 
 
-def time_oracle(batch, steps, warmup):
+def oracle_pass(workload, batch):
+    """One pass of the oracle over every layer of the workload at `batch`: (TOPS, seconds, threads)."""
     from oracle import cpu as O
-    from paper_2102_04782_b200 import synth
-    inputs = oracle_inputs(batch)
-    for _ in range(warmup):
-        oracle_step(inputs)
+    _, fn, _ = workloads()[workload]
+    layers = fn()
+    inputs = oracle_inputs(layers, batch)
     t0 = time.perf_counter()
-    for _ in range(steps):
-        oracle_step(inputs)
-    dt = (time.perf_counter() - t0) / steps
-    ops = bwd_ops(synth.resnet50_conv2x_block(), batch)
-    return ops / dt / 1e12, dt, O.num_threads()
+    for L, x, w, g in inputs:
+        oracle_layer_step(L, x, w, g)
+    dt = time.perf_counter() - t0
+    return bwd_ops(layers, batch) / dt / 1e12, dt, O.num_threads()
 
 
 def run_reference(args):
+    """The oracle as the reference arm.  A full step of the workload would take the CPU many minutes,
+    so step i is a bounded sample of it: layer (i mod #layers) of the workload at batch 1."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    batch = 4
-    value, dt, cores = time_oracle(batch, args.steps, args.warmup)
-    sample = f"same three layers at batch {batch} of {BATCH} per step (bounded sample), CPU oracle as it stands"
+    from oracle import cpu as O
+    name, fn, batch = workloads()[args.workload]
+    layers = fn()
+    inputs = oracle_inputs(layers, 1)
+    n = len(layers)
+    for i in range(args.warmup):
+        oracle_layer_step(*inputs[i % n])
+    ops, t0 = 0, time.perf_counter()
+    for i in range(args.steps):
+        L, x, w, g = inputs[i % n]
+        oracle_layer_step(L, x, w, g)
+        ops += bwd_ops([L], 1)
+    dt = time.perf_counter() - t0
+    value = ops / dt / 1e12
+    sample = (f"step i = the whole path for layer (i mod {n}) of the workload at batch 1 of {batch} "
+              "(bounded sample), CPU oracle as it stands")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
-        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "sample": sample},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / max(args.steps, 1) * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -139,14 +156,12 @@ def aggregate_value(ops_per_step_per_rank, ms_per_step, world):
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
 class LayerBuffers:
-    def __init__(self, L, N, seed, torch, api, synth, dev):
+    """Device buffers of one layer; `host` adds pinned host copies of the inputs and results."""
+
+    def __init__(self, L, N, seed, torch, api, synth, dev, host=None):
         self.L, self.N = L, N
-        x, w, g, _, _ = synth.layer_inputs(L, N, seed, bf16=True)
         bf = torch.bfloat16
-        self.h_x = torch.from_numpy(x).permute(0, 2, 3, 1).contiguous().to(bf).pin_memory()
-        self.h_w = torch.from_numpy(w).to(bf).pin_memory()
-        self.h_g = torch.from_numpy(g).permute(0, 2, 3, 1).contiguous().to(bf).pin_memory()
-        self.x, self.w, self.g = self.h_x.to(dev), self.h_w.to(dev), self.h_g.to(dev)
+        self.x, self.w, self.g = synth.device_layer_inputs(L, N, seed, dev)
         self.geom = api.ConvGeom(N, L.Cin, L.Cout, L.H, L.W, L.R, L.S, L.stride, L.stride, L.pad, L.pad)
         Cip, Cop = api.padded_channels(L.Cin), api.padded_channels(L.Cout)
         i8 = dict(dtype=torch.int8, device=dev)
@@ -157,20 +172,18 @@ class LayerBuffers:
         self.gq = torch.empty((N, L.P, L.Q, Cop), **i8)
         self.sX, self.sW, self.gmax = torch.zeros(1, **f32), torch.zeros(1, **f32), torch.zeros(1, **f32)
         self.s_state = torch.zeros(L.Cout, **f32)
+        self.cls = torch.zeros(L.Cout, dtype=torch.uint8, device=dev)
         self.Y = torch.empty((N, L.P, L.Q, L.Cout), dtype=bf, device=dev)
         self.dX = torch.empty((N, L.H, L.W, L.Cin), dtype=bf, device=dev)
         self.dW = torch.empty((L.Cout, L.Cin, L.R, L.S), **f32)
         u8 = dict(dtype=torch.uint8, device=dev)
+        self.ws_q = torch.empty(max(16, api.quantize_tensor_workspace_bytes()), **u8)
         self.ws_g = torch.empty(api.quantize_grad_workspace_bytes(L.Cout), **u8)
-        self.ws_f = torch.empty(api.conv_workspace_bytes(api.OP_FWD, self.geom), **u8)
-        self.ws_d = torch.empty(api.conv_workspace_bytes(api.OP_BWD_DATA, self.geom), **u8)
-        self.ws_w = torch.empty(api.conv_workspace_bytes(api.OP_BWD_FILTER, self.geom), **u8)
-        self.h_Y = torch.empty(self.Y.shape, dtype=bf).pin_memory()
-        self.h_dX = torch.empty(self.dX.shape, dtype=bf).pin_memory()
-        self.h_dW = torch.empty(self.dW.shape, dtype=torch.float32).pin_memory()
+        self.ws_f = torch.empty(max(16, api.conv_workspace_bytes(api.OP_FWD, self.geom)), **u8)
+        self.ws_d = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_DATA, self.geom)), **u8)
+        self.ws_w = torch.empty(max(16, api.conv_workspace_bytes(api.OP_BWD_FILTER, self.geom)), **u8)
         self.has_prev = False
-        self.h2d = sum(t.numel() * t.element_size() for t in (self.h_x, self.h_w, self.h_g))
-        self.d2h = sum(t.numel() * t.element_size() for t in (self.h_Y, self.h_dX, self.h_dW))
+        self.host = host
         npix_in, npix_out = N * L.H * L.W, N * L.P * L.Q
         wbytes = L.Cout * L.R * L.S * Cip
         # algorithmic bytes / ops per call (operands once, outputs once)
@@ -184,17 +197,22 @@ class LayerBuffers:
             "conv_bwd_data": {"bytes": npix_out * Cop + wbytes + npix_in * L.Cin * 2, "ops": 2 * L.macs(N)},
         }
 
-    def calls(self, api, seed):
+    def fwd_calls(self, api):
         L, N = self.L, self.N
         return [
             ("quantize_x", lambda: api.quantize_tensor(self.x, api.NHWC, N, L.Cin, L.H, L.W, api.SCALE_ABSMAX,
-                                                       self.sX, api.ROUND_NEAREST_EVEN, 0, self.qX)),
+                                                       self.sX, api.ROUND_NEAREST_EVEN, 0, self.qX, self.ws_q)),
             ("quantize_w", lambda: api.quantize_tensor(self.w, api.NCHW, L.Cout, L.Cin, L.R, L.S, api.SCALE_ABSMAX,
-                                                       self.sW, api.ROUND_NEAREST_EVEN, 0, self.qW)),
+                                                       self.sW, api.ROUND_NEAREST_EVEN, 0, self.qW, self.ws_q)),
             ("conv_fwd", lambda: api.conv_fwd(self.qX, self.qW, self.sX, self.sW, self.geom, self.Y, api.NHWC,
                                               self.ws_f)),
+        ]
+
+    def bwd_calls(self, api, seed):
+        L, N = self.L, self.N
+        return [
             ("quantize_grad", lambda: api.quantize_grad(self.g, api.NHWC, N, L.Cout, L.P, L.Q, None, self.s_state,
-                                                        self.has_prev, self.gmax, None, None, self.vq, self.gq,
+                                                        self.has_prev, self.gmax, None, self.cls, self.vq, self.gq,
                                                         seed, self.ws_g)),
             ("conv_bwd_filter", lambda: api.conv_bwd_filter(self.qX, self.vq, self.sX, self.s_state, self.geom,
                                                             self.dW, self.ws_w)),
@@ -203,44 +221,254 @@ class LayerBuffers:
         ]
 
 
+class HostBuffers:
+    """Pinned host copies of one layer's inputs (X, W, dY) and room for its results (Y, dX, dW)."""
+
+    def __init__(self, b, torch):
+        self.x, self.w, self.g = (t.cpu().pin_memory() for t in (b.x, b.w, b.g))
+        self.Y = torch.empty(b.Y.shape, dtype=b.Y.dtype).pin_memory()
+        self.dX = torch.empty(b.dX.shape, dtype=b.dX.dtype).pin_memory()
+        self.dW = torch.empty(b.dW.shape, dtype=b.dW.dtype).pin_memory()
+        self.h2d = sum(t.numel() * t.element_size() for t in (self.x, self.w, self.g))
+        self.d2h = sum(t.numel() * t.element_size() for t in (self.Y, self.dX, self.dW))
+
+
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi in a loop, started before the warm-up; stop() keeps the samples whose time stamps
+    fall between mark_start() and mark_end() (all of them if too few do)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, index):
-        self.proc = None
+        self.proc, self.t0, self.t1 = None, None, None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(index), f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                          "--format=csv,noheader,nounits", "-lms", "20"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
+    def mark_start(self):
+        self.t0 = time.time()
+
+    def mark_end(self):
+        self.t1 = time.time()
+
     def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in out.strip().splitlines():
             p = [t.strip() for t in line.split(",")]
-            if len(p) < 7:
+            if len(p) < 8:
                 continue
             try:
-                sm.append(float(p[0])); mx.append(float(p[1]))
+                ts = datetime.datetime.strptime(p[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(p[1]), float(p[2]), float(p[3]),
+                             [n for n, v in zip(names, p[4:8]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, v in zip(names, p[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(name)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        inside = [r for r in rows if self.t0 is not None and self.t0 - 0.02 <= r[0] <= self.t1 + 0.02]
+        window = "timed region"
+        if len(inside) < 3:      # a very short timed region: the loaded samples of the whole run instead
+            busy = [r for r in rows if r[3] > 250.0]
+            inside, window = (busy if len(busy) >= 3 else rows), "whole run (timed region too short to sample)"
+        sm = [r[1] for r in inside]
+        reasons = sorted({n for r in inside for n in r[4]})
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max((r[2] for r in inside), default=None),
+                "power_w_max": max((r[3] for r in inside), default=None),
+                "samples": len(inside), "window": window, "reasons": reasons}
+
+
+KERNEL_OF_CALL = {
+    "quantize_x": "quantize_tensor kernels (layer scale + codes of X)",
+    "quantize_w": "quantize_tensor kernels (layer scale + codes of W)",
+    "conv_fwd": "igemm_kmajor_kernel (forward)",
+    "quantize_grad": "gvq_fused_nhwc_kernel / gvq_columns_kernel",
+    "conv_bwd_filter": "wgrad_mnmajor_kernel + finalize_bwd_filter_kernel",
+    "conv_bwd_data": "igemm_kmajor_kernel (input gradient)",
+}
+
+
+class Runner:
+    """One workload on one GPU: buffers, the step, the timed region, the per-call breakdown."""
+
+    def __init__(self, workload, torch, api, synth, dev, dist, world, with_host=False):
+        self.torch, self.api, self.dev, self.dist, self.world = torch, api, dev, dist, world
+        self.name, fn, self.batch = workloads()[workload]
+        self.layers = fn()
+        self.bufs = [LayerBuffers(L, self.batch, SEED + i, torch, api, synth, dev) for i, L in enumerate(self.layers)]
+        self.step_no = 0
+        self.ops_step = bwd_ops(self.layers, self.batch)
+        self.hosts = [HostBuffers(b, torch) for b in self.bufs] if with_host else None
+
+    def step(self, bufs=None, record=None):
+        torch, api = self.torch, self.api
+        bufs = bufs or self.bufs
+        seed = SEED + self.step_no
+
+        def run(b, calls):
+            for name, fn in calls:
+                if record is not None:
+                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
+                fn()
+                if record is not None:
+                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
+                    record.append((b.L.name, name, e0, e1))
+
+        for b in bufs:                      # forward pass, layer order
+            run(b, b.fwd_calls(api))
+        for b in reversed(bufs):            # backward pass, reverse order
+            run(b, b.bwd_calls(api, seed))
+            b.has_prev = True
+        self.step_no += 1
+
+    def barrier(self):
+        if self.dist is not None:
+            self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def timed(self, steps, warmup, sampler=None):
+        torch, api = self.torch, self.api
+        for _ in range(max(warmup, 3)):
+            self.step()
+        self.barrier()
+        launches0 = api.launch_count()
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        if sampler:
+            sampler.mark_start()
+        t0.record()
+        for _ in range(steps):
+            self.step()
+        t1.record()
+        self.barrier()
+        if sampler:
+            sampler.mark_end()
+        total_ms = max_over_ranks(t0.elapsed_time(t1), self.dist, self.dev)
+        launches = api.launch_count() - launches0
+        assert api.get_device_status() == api.OK
+        return total_ms, launches
+
+    def breakdown(self, steps):
+        """Second pass with a CUDA event pair around every call (the events keep consecutive kernels
+        from overlapping, so this pass is not the one `value` comes from)."""
+        records = []
+        for _ in range(steps):
+            self.step(record=records)
+        self.barrier()
+        agg = {}
+        for lname, cname, a, b_ in records:
+            agg.setdefault((lname, cname), []).append(a.elapsed_time(b_))
+        return {k: sum(v) / len(v) for k, v in agg.items()}
+
+    def e2e(self, steps):
+        """Pinned host inputs -> device, results -> pinned host, every step.  Two complete sets of device
+        buffers alternate, so that the host->device copy of step i+1 and the device->host copy of step
+        i-1 overlap the kernels of step i (three streams, ordered by events).  Every step still copies
+        all of its inputs in and all of its results out."""
+        torch, api = self.torch, self.api
+        from paper_2102_04782_b200 import synth
+        bufs2 = [LayerBuffers(L, self.batch, SEED + i, torch, api, synth, self.dev) for i, L in enumerate(self.layers)]
+        sets = [self.bufs, bufs2]
+        hosts = self.hosts
+        s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
+        ev_in = [torch.cuda.Event(), torch.cuda.Event()]
+        ev_cmp = [torch.cuda.Event(), torch.cuda.Event()]
+        ev_out = [torch.cuda.Event(), torch.cuda.Event()]
+        issued = [0]
+
+        def e2e_step():
+            i = issued[0]; k = i & 1; set_k = sets[k]
+            with torch.cuda.stream(s_in):
+                if i >= 2:
+                    s_in.wait_event(ev_cmp[k])          # the kernels of step i-2 have read these inputs
+                for b, h in zip(set_k, hosts):
+                    b.x.copy_(h.x, non_blocking=True); b.w.copy_(h.w, non_blocking=True)
+                    b.g.copy_(h.g, non_blocking=True)
+                ev_in[k].record(s_in)
+            s_cmp.wait_event(ev_in[k])
+            if i >= 2:
+                s_cmp.wait_event(ev_out[k])             # the results of step i-2 have left the device
+            self.step(bufs=set_k)
+            ev_cmp[k].record(s_cmp)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_cmp[k])
+                for b, h in zip(set_k, hosts):
+                    h.Y.copy_(b.Y, non_blocking=True); h.dX.copy_(b.dX, non_blocking=True)
+                    h.dW.copy_(b.dW, non_blocking=True)
+                ev_out[k].record(s_out)
+            issued[0] += 1
+
+        for _ in range(3):
+            e2e_step()
+        self.barrier()
+        e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+        e0.record(s_cmp)
+        for _ in range(steps):
+            e2e_step()
+        s_cmp.wait_stream(s_out)                        # the last results are on the host
+        s_cmp.wait_stream(s_in)
+        e1.record(s_cmp)
+        self.barrier()
+        ms = max_over_ranks(e0.elapsed_time(e1), self.dist, self.dev) / steps
+        return ms, int(sum(h.h2d for h in hosts)), int(sum(h.d2h for h in hosts))
+
+    def summarize(self, per_call_ms, int8_peak, peaks):
+        """Per-call entries, phase totals and the dominant kernel of the step."""
+        alg = {(b.L.name, k): v for b in self.bufs for k, v in b.alg.items()}
+        shape = {b.L.name: f"{b.L.Cin}->{b.L.Cout} {b.L.R}x{b.L.S}/{b.L.stride} @{b.L.H}" for b in self.bufs}
+        ridge = int8_peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
+        calls, by_call = [], {}
+        for key, ms in per_call_ms.items():
+            a = alg[key]
+            ent = {"layer": key[0], "shape": shape[key[0]], "call": key[1], "ms": round(ms, 5),
+                   "gbs": round(a["bytes"] / ms / 1e6, 1)}
+            if "ops" in a:
+                ent["tops"] = round(a["ops"] / ms / 1e9, 1)
+                ent["frac_int8_peak"] = round(a["ops"] / ms / 1e9 / int8_peak, 4)
+                ent["bound"] = "tensor" if a["ops"] / a["bytes"] > ridge else "hbm"
+            else:
+                ent["frac_hbm"] = round(a["bytes"] / ms / 1e6 / peaks["hbm_gbs"], 4)
+                ent["bound"] = "hbm"
+            calls.append(ent)
+            t = by_call.setdefault(key[1], {"ms": 0.0, "bytes": 0, "ops": 0, "n": 0, "tensor_ms": 0.0, "tensor_ops": 0})
+            t["ms"] += ms; t["bytes"] += a["bytes"]; t["ops"] += a.get("ops", 0); t["n"] += 1
+            if ent["bound"] == "tensor":
+                t["tensor_ms"] += ms; t["tensor_ops"] += a["ops"]
+        total = sum(t["ms"] for t in by_call.values())
+        phases = {}
+        for name, t in by_call.items():
+            p = {"ms": round(t["ms"], 4), "share": round(t["ms"] / total, 4), "launch_groups": t["n"],
+                 "gbs": round(t["bytes"] / t["ms"] / 1e6, 1), "frac_hbm": round(t["bytes"] / t["ms"] / 1e6 / peaks["hbm_gbs"], 4)}
+            if t["ops"]:
+                p["tops"] = round(t["ops"] / t["ms"] / 1e9, 1)
+                p["frac_int8_peak"] = round(t["ops"] / t["ms"] / 1e9 / int8_peak, 4)
+            if t["tensor_ms"] > 0:
+                p["compute_bound_layers_tops"] = round(t["tensor_ops"] / t["tensor_ms"] / 1e9, 1)
+                p["compute_bound_layers_frac_int8_peak"] = round(t["tensor_ops"] / t["tensor_ms"] / 1e9 / int8_peak, 4)
+            phases[name] = p
+        bwd = [by_call.get("conv_bwd_filter"), by_call.get("conv_bwd_data")]
+        bwd_ms = sum(t["ms"] for t in bwd if t)
+        bwd_ops_ = sum(t["ops"] for t in bwd if t)
+        gvq = by_call.get("quantize_grad")
+        out = {"phases": phases,
+               "conv_bwd_tops_calls_only": round(bwd_ops_ / bwd_ms / 1e9, 1),
+               "conv_bwd_frac_int8_peak": round(bwd_ops_ / bwd_ms / 1e9 / int8_peak, 4),
+               "gvq_effective_gbs": round(gvq["bytes"] / gvq["ms"] / 1e6, 1),
+               "gvq_frac_hbm": round(gvq["bytes"] / gvq["ms"] / 1e6 / peaks["hbm_gbs"], 4)}
+        dom_name = max(by_call, key=lambda n: by_call[n]["ms"])
+        return out, calls, dom_name, by_call[dom_name]
 
 
 def run_dai8(args):
@@ -259,182 +487,85 @@ def run_dai8(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     api.lib()
+    peaks = measured_peaks()
 
-    layers = synth.resnet50_conv2x_block()
-    bufs = [LayerBuffers(L, BATCH, SEED + i, torch, api, synth, dev) for i, L in enumerate(layers)]
-    step_no = [0]
-
-    def step(record=None):
-        seed = SEED + step_no[0]
-        for b in bufs:
-            for name, fn in b.calls(api, seed):
-                if record is not None:
-                    e0 = torch.cuda.Event(enable_timing=True); e0.record()
-                fn()
-                if record is not None:
-                    e1 = torch.cuda.Event(enable_timing=True); e1.record()
-                    record.append((b.L.name, name, e0, e1))
-            b.has_prev = True
-        step_no[0] += 1
-
-    def barrier():
-        if dist is not None:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_ranks(ms):
-        return max_over_ranks(ms, dist, dev)
-
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-
-    # ---- timed region: K steps, device-timed, nothing but the path's own launches inside ----------
     sampler = ClockSampler(local) if rank == 0 else None
-    launches0 = api.launch_count()
-    barrier()
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(args.steps):
-        step()
-    t1.record()
-    barrier()
-    total_ms = max_ranks(t0.elapsed_time(t1))
-    launches = api.launch_count() - launches0
+    main = Runner(args.workload, torch, api, synth, dev, dist, world, with_host=True)
+    warmup = max(args.warmup, 3)
+    total_ms, launches = main.timed(args.steps, warmup, sampler)
     clocks = sampler.stop() if sampler else None
-    # per-call breakdown: a second, shorter pass of the same steps with an event pair around every call
-    # (the events cost device time themselves, so this pass is not the one `value` comes from)
-    records = []
-    for _ in range(min(args.steps, 100)):
-        step(records)
-    barrier()
-    assert api.get_device_status() == api.OK
     ms_per_step = total_ms / args.steps
-    ops_step = bwd_ops(layers, BATCH)
-    value = aggregate_value(ops_step, ms_per_step, world)
-
-    # ---- end to end: pinned host inputs -> device, results -> pinned host, every step ------------
-    # Two complete sets of device buffers alternate, so that the host->device copy of step i+1 and
-    # the device->host copy of step i-1 overlap the kernels of step i (three streams, ordered by
-    # events).  Every step still copies all of its inputs in and all of its results out.
-    bufs2 = [LayerBuffers(L, BATCH, SEED + i, torch, api, synth, dev) for i, L in enumerate(layers)]
-    sets = [bufs, bufs2]
-    s_in, s_out, s_cmp = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.current_stream()
-    ev_in = [torch.cuda.Event(), torch.cuda.Event()]
-    ev_cmp = [torch.cuda.Event(), torch.cuda.Event()]
-    ev_out = [torch.cuda.Event(), torch.cuda.Event()]
-    issued = [0]
-
-    def e2e_step():
-        i = issued[0]; k = i & 1; set_k = sets[k]
-        with torch.cuda.stream(s_in):
-            if i >= 2:
-                s_in.wait_event(ev_cmp[k])          # the kernels of step i-2 have read these inputs
-            for b in set_k:
-                b.x.copy_(b.h_x, non_blocking=True); b.w.copy_(b.h_w, non_blocking=True)
-                b.g.copy_(b.h_g, non_blocking=True)
-            ev_in[k].record(s_in)
-        s_cmp.wait_event(ev_in[k])
-        if i >= 2:
-            s_cmp.wait_event(ev_out[k])             # the results of step i-2 have left the device
-        seed = SEED + step_no[0]
-        for b in set_k:
-            for _, fn in b.calls(api, seed):
-                fn()
-            b.has_prev = True
-        step_no[0] += 1
-        ev_cmp[k].record(s_cmp)
-        with torch.cuda.stream(s_out):
-            s_out.wait_event(ev_cmp[k])
-            for b in set_k:
-                b.h_Y.copy_(b.Y, non_blocking=True); b.h_dX.copy_(b.dX, non_blocking=True)
-                b.h_dW.copy_(b.dW, non_blocking=True)
-            ev_out[k].record(s_out)
-        issued[0] += 1
-
-    for _ in range(3):
-        e2e_step()
-    barrier()
-    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
-    e2e_steps = min(args.steps, 40)
-    e0.record(s_cmp)
-    for _ in range(e2e_steps):
-        e2e_step()
-    s_cmp.wait_stream(s_out)                        # the last results are on the host
-    s_cmp.wait_stream(s_in)
-    e1.record(s_cmp)
-    barrier()
-    e2e_ms = max_ranks(e0.elapsed_time(e1)) / e2e_steps
-    e2e_value = aggregate_value(ops_step, e2e_ms, world)
+    value = aggregate_value(main.ops_step, ms_per_step, world)
+    sustained = total_ms > 1000.0
+    int8_peak = INT8_OVER_BF16 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
+    per_call = main.breakdown(min(args.steps, 10))
+    e2e_steps = max(2, min(args.steps, 8))
+    e2e_ms, h2d, d2h = main.e2e(e2e_steps)
+    e2e_value = aggregate_value(main.ops_step, e2e_ms, world)
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    # ---- per-call breakdown and roofline of the dominant call -------------------------------------
-    peaks = measured_peaks()
-    agg = {}
-    for lname, cname, a, b_ in records:
-        agg.setdefault((lname, cname), []).append(a.elapsed_time(b_))
-    alg = {(b.L.name, k): v for b in bufs for k, v in b.alg.items()}
-    detail, dominant = [], None
-    sustained = total_ms > 1000.0
-    int8_peak = INT8_OVER_BF16 * (peaks["bf16_sustained"] if sustained else peaks["bf16_burst"])
-    ridge = int8_peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
-    for key, times in agg.items():
-        ms = sum(times) / len(times)
-        a = alg[key]
-        ent = {"layer": key[0], "call": key[1], "ms": round(ms, 5), "gbs": round(a["bytes"] / ms / 1e6, 1)}
-        if "ops" in a:
-            ent["tops"] = round(a["ops"] / ms / 1e9, 2)
-            ent["bound"] = "tensor" if a["ops"] / a["bytes"] > ridge else "hbm"
-        else:
-            ent["bound"] = "hbm"
-        detail.append(ent)
-        if dominant is None or ms > dominant[0]:
-            dominant = (ms, key, ent)
-    dms, dkey, dent = dominant
-    if dent["bound"] == "tensor":
-        achieved, peak, unit = alg[dkey]["ops"] / dms / 1e9, int8_peak, "TOPS"
+    summary, calls, dom_name, dom = main.summarize(per_call, int8_peak, peaks)
+    tensor_bound = dom["ops"] > 0 and dom["ops"] / dom["bytes"] > int8_peak * 1e12 / (peaks["hbm_gbs"] * 1e9)
+    if tensor_bound:
+        achieved, peak, unit = dom["ops"] / dom["ms"] / 1e9, int8_peak, "TOPS"
     else:
-        achieved, peak, unit = alg[dkey]["bytes"] / dms / 1e6, peaks["hbm_gbs"], "GB/s"
-    roofline = {"bound": dent["bound"], "achieved": round(achieved, 2), "peak": peak, "unit": unit,
-                "frac": round(achieved / peak, 4), "traffic": NCU_TRAFFIC.get(f"{dkey[1]} @ {dkey[0]}"),
-                "algorithmic_bytes": alg[dkey]["bytes"],
-                "kernel": f"{dkey[1]} @ {dkey[0]}", "peak_source": peaks["source"],
-                "peak_kind": ("int8 = 2 x bf16 " + ("sustained" if sustained else "burst")) if unit == "TOPS" else "copy"}
-    def phase_ms(names):
-        return sum(e["ms"] for e in detail if e["call"] in names)
-    conv_bwd_ms = phase_ms(("conv_bwd_filter", "conv_bwd_data"))
-    gvq_ms = phase_ms(("quantize_grad",))
-    gvq_bytes = sum(b.alg["quantize_grad"]["bytes"] for b in bufs)
-    summary = {
-        "conv_bwd_tops_calls_only": round(ops_step / conv_bwd_ms / 1e9, 2),
-        "conv_bwd_frac_int8_peak": round(ops_step / conv_bwd_ms / 1e9 / int8_peak, 4),
-        "gvq_effective_gbs": round(gvq_bytes / gvq_ms / 1e6, 1),
-        "gvq_frac_hbm": round(gvq_bytes / gvq_ms / 1e6 / peaks["hbm_gbs"], 4),
-        "int8_peak_tops": int8_peak, "hbm_peak_gbs": peaks["hbm_gbs"], "calls": detail,
-    }
+        achieved, peak, unit = dom["bytes"] / dom["ms"] / 1e6, peaks["hbm_gbs"], "GB/s"
+    roofline = {"bound": "tensor" if tensor_bound else "hbm", "achieved": round(achieved, 2), "peak": peak,
+                "unit": unit, "frac": round(achieved / peak, 4), "traffic": None,
+                "kernel": KERNEL_OF_CALL[dom_name], "launches_per_step": dom["n"],
+                "share_of_step": summary["phases"][dom_name]["share"],
+                "algorithmic_ops_per_step": dom["ops"], "algorithmic_bytes_per_step": dom["bytes"],
+                "ms_per_step": round(dom["ms"], 4), "peak_source": peaks["source"],
+                "peak_kind": ("int8 = 2 x bf16 " + ("sustained" if sustained else "burst")) if unit == "TOPS" else "copy",
+                "note": "all launches of this kernel in one step, summed: achieved = their algorithmic ops (bytes) / their time"}
+    summary["calls"] = calls
+    summary["int8_peak_tops"] = int8_peak
+    summary["hbm_peak_gbs"] = peaks["hbm_gbs"]
+    summary["targets"] = {"conv_bwd_frac_int8_peak_on_compute_bound_layers": 0.60, "gvq_frac_hbm": 0.70}
+    del main
+    torch.cuda.empty_cache()
+
+    # ---- the other configurations, device-timed the same way (no end-to-end leg) -------------------
+    others = {}
+    if world == 1 and not args.main_only:
+        for wl in ("conv2x", "resnet50", "mobilenetv2", "vgg16"):
+            if wl == args.workload:
+                continue
+            r = Runner(wl, torch, api, synth, dev, None, 1)
+            steps = min(args.steps, 20)
+            t_ms, _ = r.timed(steps, 3)
+            s, c, _, _ = r.summarize(r.breakdown(min(steps, 5)), INT8_OVER_BF16 * peaks["bf16_burst"], peaks)
+            s["workload"] = r.name
+            s["ms_per_step"] = round(t_ms / steps, 4)
+            s["value_tops"] = round(aggregate_value(r.ops_step, t_ms / steps, 1), 2)
+            s["compute_bound_calls"] = [e for e in c if e["bound"] == "tensor"]
+            others[wl] = s
+            del r
+            torch.cuda.empty_cache()
+    summary["other_configs"] = others
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        cb = 8
-        v, dt, cores = time_oracle(cb, 1, 0)
+        v, dt, cores = oracle_pass(args.workload, 1)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"same three layers at batch {cb} of {BATCH}, one pass, {dt:.1f} s"}
+               "sample": f"every layer of the workload at batch 1 of {workloads()[args.workload][2]}, one pass, {dt:.1f} s"}
 
+    name, _, batch = workloads()[args.workload]
     line = {
         "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
+        "warmup": warmup, "ms_per_step": round(ms_per_step, 4), "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
-        "config": {"workload": WORKLOAD, "layers": [l.name for l in layers], "batch": BATCH,
-                   "outputs": "Y,dX bf16 NHWC; dW fp32", "l2": "inputs larger than L2 (about 0.9 GB touched per step)",
+        "config": {"workload": name, "layers": len(workloads()[args.workload][1]()), "batch": batch,
+                   "outputs": "Y,dX bf16 NHWC; dW fp32",
+                   "l2": "inputs larger than L2 (several GB touched per step)",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3), "steps": e2e_steps,
-                "h2d_bytes_per_step": int(sum(b.h2d for b in bufs)),
-                "d2h_bytes_per_step": int(sum(b.d2h for b in bufs))},
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "roofline": roofline, "cpu_baseline": cpu, "detail": summary,
     }
     print(json.dumps(line))
@@ -443,10 +574,10 @@ def run_dai8(args):
 
 
 # ------------------------------------------------------------------------------------------------
-# Per-layer report over one of the network configurations (not the contract line: that is
-# run_dai8 on the conv2_x block).  `python bench.py --layers resnet50|mobilenetv2|vgg16 [--batch N]`
-# prints one JSON object with, per layer, the device time of the gradient quantization and of the
-# three convolutions, and totals as TOPS / GB/s against the measured peaks.
+# Per-layer report over one of the network configurations (not the contract line).
+# `python bench.py --layers resnet50|mobilenetv2|vgg16|conv2x [--batch N]` prints one JSON object
+# with, per layer, the device time of the gradient quantization and of the three convolutions in
+# isolation (L2 flushed, best of 3), and the whole network back to back with the host enqueue time.
 # ------------------------------------------------------------------------------------------------
 def run_layer_report(args):
     import torch
@@ -454,9 +585,7 @@ def run_layer_report(args):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     api.lib()
-    table = {"resnet50": (synth.resnet50_convs, 64), "mobilenetv2": (synth.mobilenetv2_pointwise, 128),
-             "vgg16": (synth.vgg16_convs, 64), "conv2x": (synth.resnet50_conv2x_block, 64)}
-    fn, batch = table[args.layers]
+    _, fn, batch = workloads()[args.layers]
     N = args.batch or batch
     peaks = measured_peaks()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
@@ -501,7 +630,7 @@ def run_layer_report(args):
                 "bwd_filter": timed(lambda: api.conv_bwd_filter(qX, vq, one, s_c, g, dW, ws_w)),
                 "bwd_data": timed(lambda: api.conv_bwd_data(gq, qW, gm, one, g, dX, api.NHWC, ws_d)),
             }
-            npix_o, npix_i = N * L.P * L.Q, N * L.H * L.W
+            npix_o = N * L.P * L.Q
             seen[key] = (t, 2 * L.macs(N), npix_o * (2 * L.Cout + 2 * Cop))
             # the same calls again, kept for the pipelined pass below (buffers stay alive in the closures)
             chain[key] = {
@@ -556,12 +685,12 @@ def run_layer_report(args):
     assert api.get_device_status() == api.OK
     int8_peak = INT8_OVER_BF16 * peaks["bf16_burst"]
     bwd_ms = tot["bwd_data"][0] + tot["bwd_filter"][0]
-    bwd_ops = tot["bwd_data"][1] + tot["bwd_filter"][1]
+    bwd_ops_ = tot["bwd_data"][1] + tot["bwd_filter"][1]
     out = {"layers_config": args.layers, "batch": N, "timing": "best of 3 per call, CUDA events on the device; L2 flushed before each call; the call is enqueued while a delay kernel runs, so host launch latency is not in the time",
            "totals": {
                "fwd_ms": round(tot["fwd"][0], 3), "fwd_tops": round(tot["fwd"][1] / tot["fwd"][0] / 1e9, 1),
-               "bwd_ms": round(bwd_ms, 3), "bwd_tops": round(bwd_ops / bwd_ms / 1e9, 1),
-               "bwd_frac_int8_peak": round(bwd_ops / bwd_ms / 1e9 / int8_peak, 4),
+               "bwd_ms": round(bwd_ms, 3), "bwd_tops": round(bwd_ops_ / bwd_ms / 1e9, 1),
+               "bwd_frac_int8_peak": round(bwd_ops_ / bwd_ms / 1e9 / int8_peak, 4),
                "gvq_ms": round(tot["quantize_grad"][0], 3),
                "gvq_gbs": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6, 1),
                "gvq_frac_hbm": round(tot["quantize_grad"][1] / tot["quantize_grad"][0] / 1e6 / peaks["hbm_gbs"], 4),
@@ -578,9 +707,12 @@ def run_layer_report(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dai8", choices=["dai8", "reference"])
+    ap.add_argument("--workload", default="vgg16", choices=["vgg16", "resnet50", "mobilenetv2", "conv2x"],
+                    help="configuration of the JSON line (default: VGG-16, the compute-bound one)")
+    ap.add_argument("--main-only", action="store_true", help="skip the other configurations in `detail`")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers", default=None, choices=["conv2x", "resnet50", "mobilenetv2", "vgg16"],
                     help="print a per-layer report for a network configuration instead of the benchmark line")

@@ -97,11 +97,20 @@ int dai8_padded_channels(int C);
  *   round      nearest-even (weights, activations) or stochastic (gradients); the stochastic
  *              mode draws u from a counter-based hash of (seed, stream 0, NCHW index)
  *   q          out, int8 [N][H][W][Cp]; padding channels are written with 0
- * Workspace: none.  q(x) = round(clamp(x*(127/s), -127, 127)); s <= 0 gives all-zero codes.
+ *   ws         scratch of dai8_quantize_tensor_workspace_bytes() bytes, or NULL.  With scratch, a
+ *              tensor whose codes have the layout of its values (NHWC, C a multiple of 16) gets its
+ *              scale and its codes from ONE launch that keeps as much of the tensor as fits in
+ *              shared memory between the two sweeps; without it (ws == NULL) the scale and the
+ *              codes take two launches.  The results are identical.  A non-NULL ws that is too
+ *              small returns DAI8_ERR_WORKSPACE.
+ * q(x) = round(clamp(x*(127/s), -127, 127)); s <= 0 gives all-zero codes.
  * -------------------------------------------------------------------------------------------- */
+size_t dai8_quantize_tensor_workspace_bytes(void);
+
 dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout layout, int N, int C,
                                  int H, int W, dai8_scale_mode scale_mode, float* scale,
-                                 dai8_round round, uint32_t seed, int8_t* q, void* stream);
+                                 dai8_round round, uint32_t seed, int8_t* q, void* ws,
+                                 size_t ws_bytes, void* stream);
 
 /* ----------------------------------------------------------------------------------------------
  * dai8_quantize_grad -- Algorithm 1, the quantization half: Gradient Vectorized Quantization with the

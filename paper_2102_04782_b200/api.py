@@ -22,6 +22,7 @@ OP_FWD, OP_BWD_DATA, OP_BWD_FILTER = 0, 1, 2
 
 EXPORTS = [
     "dai8_status_string", "dai8_mcs_defaults", "dai8_padded_channels", "dai8_quantize_tensor",
+    "dai8_quantize_tensor_workspace_bytes",
     "dai8_quantize_grad_workspace_bytes", "dai8_quantize_grad", "dai8_quantize_grad_noalloc",
     "dai8_conv_workspace_bytes",
     "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
@@ -74,8 +75,10 @@ def lib() -> ctypes.CDLL:
         l.dai8_conv_workspace_bytes.argtypes = [c_int, ctypes.POINTER(ConvGeom)]
         l.dai8_launch_count.restype = c_uint64
         l.dai8_set_conv_backend.restype = None
+        l.dai8_quantize_tensor_workspace_bytes.restype = c_size_t
+        l.dai8_quantize_tensor_workspace_bytes.argtypes = []
         l.dai8_quantize_tensor.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_int,
-                                           c_void_p, c_int, c_uint32, c_void_p, c_void_p]
+                                           c_void_p, c_int, c_uint32, c_void_p, c_void_p, c_size_t, c_void_p]
         l.dai8_quantize_grad.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int,
                                          ctypes.POINTER(McsParams), c_void_p, c_int, c_void_p,
                                          c_void_p, c_void_p, c_void_p, c_void_p, c_uint32, c_void_p,
@@ -153,11 +156,18 @@ def get_device_status() -> int:
     return v.value
 
 
+def quantize_tensor_workspace_bytes() -> int:
+    return int(lib().dai8_quantize_tensor_workspace_bytes())
+
+
 def quantize_tensor(x: torch.Tensor, layout: int, N: int, C: int, H: int, W: int, scale_mode: int,
-                    scale: torch.Tensor, rounding: int, seed: int, q: torch.Tensor) -> None:
-    """dai8_quantize_tensor: x (fp32/bf16, `layout`) -> q int8 [N][H][W][Cp]; scale: 1 float."""
+                    scale: torch.Tensor, rounding: int, seed: int, q: torch.Tensor,
+                    ws: Optional[torch.Tensor] = None) -> None:
+    """dai8_quantize_tensor: x (fp32/bf16, `layout`) -> q int8 [N][H][W][Cp]; scale: 1 float;
+    ws: scratch of quantize_tensor_workspace_bytes() bytes or None."""
+    p, n = _ws_args(ws)
     _check(lib().dai8_quantize_tensor(_ptr(x), _dtype_code(x), layout, N, C, H, W, scale_mode,
-                                      _ptr(scale), rounding, seed & 0xFFFFFFFF, _ptr(q), _stream()),
+                                      _ptr(scale), rounding, seed & 0xFFFFFFFF, _ptr(q), p, n, _stream()),
            "dai8_quantize_tensor")
 
 

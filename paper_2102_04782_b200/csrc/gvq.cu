@@ -1678,6 +1678,174 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// dai8_quantize_tensor in ONE launch for tensors whose codes have the layout of their values (NHWC
+// with C a multiple of 16), layer scale = max|x|, nearest rounding: the forward quantization of the
+// activations (Eq. 1, Fig. 2).  The scale needs the whole tensor before the first code can be
+// written, so the tensor is swept twice; this kernel makes the second sweep as cheap as the chip
+// allows.  A persistent cooperative launch, one CTA per SM, each owning a contiguous range of the
+// tensor.  A producer warp streams the range through a ring of 16 KB shared-memory pieces with bulk
+// asynchronous copies; sweep 1 takes max|x| (packed bf16 arithmetic, exact).  After one atomic max
+// per CTA and one grid barrier, sweep 2 writes the codes walking the range BACKWARDS: first the
+// pieces that are still in shared memory from sweep 1 (no memory traffic at all), then the rest in
+// reverse order, so that what it fetches is what sweep 1 touched last and L2 still holds.
+//
+// With scale = max|x| no clamp of Eq. 1 can change a code: |x * fl(127/s)| <= 127 (1 + 2^-23)^2,
+// which rounds to 127 like the clamped value does.  Codes come out of the magic-number addition
+// (quant_nearest_bits without the clamps).
+// ------------------------------------------------------------------------------------------------
+constexpr int kQtPieceBytes = 16384;
+constexpr int kQtPieceVecs = kQtPieceBytes / 16;
+constexpr int kQtMaxSlots = 13;
+
+struct QtArgs {
+  const uint8_t* x;      // the tensor as bytes
+  int8_t* q;
+  float* scale;          // out: max|x|
+  uint32_t* ctrl;        // [0] grid-barrier counter, [1] bit pattern of the running maximum; zeroed before the launch
+  int64_t nvec;          // 16-byte vectors in the tensor
+  int64_t vec_per_cta;
+  int slots;             // shared-memory pieces per CTA
+  unsigned int* status;
+};
+
+template <typename T>
+__global__ void __launch_bounds__(kFusedThreads, 1)
+quantize_flat_fused_kernel(const QtArgs a) {
+  constexpr int VE = 16 / (int)sizeof(T);
+  extern __shared__ __align__(128) uint8_t qsmem[];
+  __shared__ uint64_t full_bar[kQtMaxSlots], empty_bar[kQtMaxSlots];
+  __shared__ volatile uint32_t s_abort;
+  __shared__ uint32_t s_ok;
+  __shared__ float s_wmax[kFT / 32];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int64_t v0 = (int64_t)blockIdx.x * a.vec_per_cta;
+  const int64_t v1 = min(a.nvec, v0 + a.vec_per_cta);
+  const int nv = v1 > v0 ? (int)(v1 - v0) : 0;          // vectors of this CTA
+  const int K = (nv + kQtPieceVecs - 1) / kQtPieceVecs;  // pieces of this CTA
+  const int S = a.slots;
+  // Piece u of sweep 1 goes to slot u mod S; afterwards the last min(K, S) pieces are resident.  Step v
+  // of sweep 2 handles piece K-1-v in the slot of step v - S (the same slot for v < S: resident).
+  auto slot2 = [&](int v) { int r = (K - 1 - (v % S)) % S; return r < 0 ? r + S : r; };
+  auto fills1 = [&](int slot) { return slot < K ? (K - slot + S - 1) / S : 0; };   // sweep-1 fills of a slot
+
+  if (tid == 0) {
+    s_abort = 0u;
+#pragma unroll 1
+    for (int s = 0; s < kQtMaxSlots; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kFT / 32); }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (warp == kFT / 32) {
+    // ---- producer: every fill of a slot but its first waits for the consumers' hand-back of the fill before
+    if (lane == 0 && K > 0) {
+      const uint8_t* src = a.x + (size_t)v0 * 16;
+      const int total = K + (K > S ? K - S : 0);
+#pragma unroll 1
+      for (int t = 0; t < total; ++t) {
+        int piece, slot, fill;
+        if (t < K) { piece = t; slot = t % S; fill = t / S; }
+        else { const int v = t - K + S; piece = K - 1 - v; slot = slot2(v); fill = fills1(slot) - 1 + v / S; }
+        if (fill > 0 && !mbar_wait(&empty_bar[slot], (uint32_t)(fill - 1) & 1u, &s_abort, a.status)) break;
+        const uint32_t bytes = (uint32_t)min(kQtPieceVecs, nv - piece * kQtPieceVecs) * 16u;
+        mbar_expect_tx(&full_bar[slot], bytes);
+        bulk_load(qsmem + (size_t)slot * kQtPieceBytes, src + (size_t)piece * kQtPieceBytes, bytes, &full_bar[slot]);
+      }
+    }
+    return;
+  }
+
+  // ---- sweep 1: max|x| -------------------------------------------------------------------------------
+  bool ok = true;
+  float m = 0.f;
+  uint32_t m2[4] = {0u, 0u, 0u, 0u};
+#pragma unroll 1
+  for (int u = 0; u < K && ok; ++u) {
+    const int slot = u % S;
+    ok = mbar_wait(&full_bar[slot], (uint32_t)(u / S) & 1u, &s_abort, a.status);
+    if (!ok) break;
+    const uint4* pv = reinterpret_cast<const uint4*>(qsmem + (size_t)slot * kQtPieceBytes);
+    const int cnt = min(kQtPieceVecs, nv - u * kQtPieceVecs);
+#pragma unroll 2
+    for (int i = tid; i < cnt; i += kFT) {
+      const uint4 r = pv[i];
+      if constexpr (VE == 8) {
+        m2[0] = bf16x2_max(m2[0], r.x & 0x7FFF7FFFu); m2[1] = bf16x2_max(m2[1], r.y & 0x7FFF7FFFu);
+        m2[2] = bf16x2_max(m2[2], r.z & 0x7FFF7FFFu); m2[3] = bf16x2_max(m2[3], r.w & 0x7FFF7FFFu);
+      } else {
+        m = fmaxf(fmaxf(m, fabsf(__uint_as_float(r.x))), fmaxf(fabsf(__uint_as_float(r.y)),
+            fmaxf(fabsf(__uint_as_float(r.z)), fabsf(__uint_as_float(r.w)))));
+      }
+    }
+    if (u + S < K) {            // the slot is filled again in this sweep: hand it back
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&empty_bar[slot]);
+    }
+  }
+  if constexpr (VE == 8) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      m = fmaxf(m, fmaxf(__uint_as_float(m2[j] << 16), __uint_as_float(m2[j] & 0xFFFF0000u)));
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if (lane == 0) s_wmax[warp] = m;
+  consumer_sync();
+  if (tid == 0) {
+#pragma unroll 1
+    for (int w = 1; w < kFT / 32; ++w) m = fmaxf(m, s_wmax[w]);
+    if (m > 0.f) atomicMax(a.ctrl + 1, __float_as_uint(m));   // non-negative floats order like their bit patterns
+  }
+  ok = grid_barrier(a.ctrl, gridDim.x, a.status, &s_abort, &s_ok) && ok;
+
+  // ---- sweep 2: codes, backwards -----------------------------------------------------------------------
+  if (ok) {
+    const float s = __uint_as_float(__ldcg(a.ctrl + 1));
+    if (blockIdx.x == 0 && tid == 0) *a.scale = s;
+    const float inv = inv_scale(s);
+    int8_t* qbase = a.q + (size_t)v0 * VE;
+#pragma unroll 1
+    for (int v = 0; v < K && ok; ++v) {
+      const int piece = K - 1 - v, slot = slot2(v);
+      ok = mbar_wait(&full_bar[slot], (uint32_t)(fills1(slot) - 1 + v / S) & 1u, &s_abort, a.status);
+      if (!ok) break;
+      const uint4* pv = reinterpret_cast<const uint4*>(qsmem + (size_t)slot * kQtPieceBytes);
+      const int cnt = min(kQtPieceVecs, nv - piece * kQtPieceVecs);
+      int8_t* qp = qbase + (size_t)piece * kQtPieceVecs * VE;
+#pragma unroll 2
+      for (int i = tid; i < cnt; i += kFT) {
+        const uint4 r = pv[i];
+        if constexpr (VE == 8) {
+          const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+          uint32_t c[8];
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            c[2 * j] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(w[j] << 16), inv), kRoundMagic));
+            c[2 * j + 1] = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(w[j] & 0xFFFF0000u), inv), kRoundMagic));
+          }
+          *reinterpret_cast<uint2*>(qp + (size_t)i * 8) = make_uint2(pack_codes4(c[0], c[1], c[2], c[3]), pack_codes4(c[4], c[5], c[6], c[7]));
+        } else {
+          const uint32_t c0 = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r.x), inv), kRoundMagic));
+          const uint32_t c1 = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r.y), inv), kRoundMagic));
+          const uint32_t c2 = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r.z), inv), kRoundMagic));
+          const uint32_t c3 = __float_as_uint(__fadd_rn(__fmul_rn(__uint_as_float(r.w), inv), kRoundMagic));
+          *reinterpret_cast<uint32_t*>(qp + (size_t)i * 4) = pack_codes4(c0, c1, c2, c3);
+        }
+      }
+      if (v + S < K) {          // another piece is fetched into this slot
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[slot]);
+      }
+    }
+  }
+  if (s_abort) {
+    // a wait ran out: give copies that may still be in flight time to land before the CTA ends
+#pragma unroll 1
+    for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
 // Host-side launch helpers
 // ------------------------------------------------------------------------------------------------
 struct FusedConfig {
@@ -1974,15 +2142,52 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
   }
 }
 
+constexpr size_t kQuantizeTensorWsBytes = 256;
+
+// One cooperative launch: layer scale and codes of a tensor whose codes have the layout of its values.
+template <typename T>
+dai8_status launch_quantize_flat_fused(const T* x, int64_t nvec, float* scale, int8_t* q, void* ws, cudaStream_t st) {
+  const FusedConfig& cfg = fused_config();
+  QtArgs a;
+  a.x = reinterpret_cast<const uint8_t*>(x); a.q = q; a.scale = scale; a.ctrl = static_cast<uint32_t*>(ws);
+  a.nvec = nvec;
+  int64_t ctas = ceil_div64(nvec, kQtPieceVecs);
+  if (ctas > cfg.sms) ctas = cfg.sms;
+  a.vec_per_cta = ceil_div64(nvec, ctas);
+  ctas = ceil_div64(nvec, a.vec_per_cta);                 // no CTA without work
+  int64_t slots = ceil_div64(a.vec_per_cta, kQtPieceVecs);
+  if (slots > kQtMaxSlots) slots = kQtMaxSlots;
+  a.slots = (int)slots;
+  a.status = device_status_address();
+  if (!a.status) return DAI8_ERR_CUDA;
+  auto kern = quantize_flat_fused_kernel<T>;
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [&] {
+    attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kQtMaxSlots * kQtPieceBytes);
+  });
+  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, 16, st));
+  void* args[] = {(void*)&a};
+  DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFusedThreads), args,
+                                                  (size_t)slots * kQtPieceBytes, st));
+  note_launch(1);
+  return DAI8_OK;
+}
+
 template <typename T>
 dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, int H, int W,
                                   dai8_scale_mode mode, float* scale, dai8_round round,
-                                  uint32_t seed, int8_t* q, cudaStream_t st) {
+                                  uint32_t seed, int8_t* q, void* ws, cudaStream_t st) {
   const int64_t HW = (int64_t)H * W;
   const int64_t npix = (int64_t)N * HW;
   const int64_t total = npix * C;
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
+  if (ws && mode == DAI8_SCALE_ABSMAX && round == DAI8_ROUND_NEAREST_EVEN && layout == DAI8_NHWC && C == Cp &&
+      npix * Cp > kSmallTensorElems && fused_config().coop && ceil_div64(total / VEfull, fused_config().sms) < ((int64_t)1 << 30) &&
+      fused_config().smem_max >= (size_t)kQtMaxSlots * kQtPieceBytes + 2048)
+    return launch_quantize_flat_fused<T>(x, total / VEfull, scale, q, ws, st);
   if (npix * Cp <= kSmallTensorElems) {
     const int am = mode == DAI8_SCALE_ABSMAX ? 1 : 0, sr = round == DAI8_ROUND_STOCHASTIC ? 1 : 0;
     int small_ctas = (int)ceil_div64(npix * Cp, 4 * kSmallThreads);
@@ -2078,11 +2283,15 @@ extern "C" dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8
                                      has_prev, gmax_layer, stats, cls, vq, gq, seed, sigma_override, w, st);
 }
 
+extern "C" size_t dai8_quantize_tensor_workspace_bytes(void) { return kQuantizeTensorWsBytes; }
+
 extern "C" dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout layout, int N,
                                             int C, int H, int W, dai8_scale_mode scale_mode,
                                             float* scale, dai8_round round, uint32_t seed, int8_t* q,
-                                            void* stream) {
+                                            void* ws, size_t ws_bytes, void* stream) {
   if (!x || !scale || !q) return DAI8_ERR_INVALID_ARG;
+  if (ws && !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (ws && ws_bytes < kQuantizeTensorWsBytes) return DAI8_ERR_WORKSPACE;
   if (bad_dims(N, C, H, W)) return DAI8_ERR_INVALID_ARG;
   if (dtype != DAI8_F32 && dtype != DAI8_BF16) return DAI8_ERR_INVALID_ARG;
   if (layout != DAI8_NCHW && layout != DAI8_NHWC) return DAI8_ERR_INVALID_ARG;
@@ -2094,9 +2303,9 @@ extern "C" dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (dtype == DAI8_F32)
     return quantize_tensor_typed<float>(static_cast<const float*>(x), layout, N, C, H, W, scale_mode,
-                                        scale, round, seed, q, st);
+                                        scale, round, seed, q, ws, st);
   return quantize_tensor_typed<bf16_t>(static_cast<const bf16_t*>(x), layout, N, C, H, W, scale_mode,
-                                       scale, round, seed, q, st);
+                                       scale, round, seed, q, ws, st);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -169,3 +169,30 @@ def layer_inputs(layer: ConvLayer, N: int, seed: int, bf16: bool) -> Tuple[np.nd
     if bf16:
         x, w, g = round_to_bf16(x), round_to_bf16(w), round_to_bf16(g)
     return x, w, g, is_bell, sigma
+
+
+def device_layer_inputs(layer: ConvLayer, N: int, seed: int, device):
+    """The same recipes drawn by torch on `device` (for workloads too large to generate on the host
+    in reasonable time): (X NHWC bf16, W (Cout,Cin,R,S) bf16, dY NHWC bf16).  The per-channel shape
+    and sigma_c of dY come from the same seeded draw as channel_mixed_grad; the samples themselves
+    are torch's, so these tensors feed timing runs, not comparisons with host-generated ones."""
+    import torch
+    gen = torch.Generator(device=device).manual_seed(int(seed) & 0x7FFFFFFF)
+    bf = torch.bfloat16
+    x = torch.randn((N, layer.H, layer.W, layer.Cin), device=device, generator=gen, dtype=torch.float32)
+    x = torch.relu_(x).to(bf)
+    w = torch.randn((layer.Cout, layer.Cin, layer.R, layer.S), device=device, generator=gen, dtype=torch.float32)
+    w = (w * float(np.sqrt(2.0 / (layer.Cin * layer.R * layer.S)))).to(bf)
+    meta = _rng(seed, 3)
+    is_bell = torch.from_numpy(meta.random(layer.Cout) < 0.5).to(device)
+    sigma = torch.from_numpy((10.0 ** meta.uniform(-6.0, -3.0, size=layer.Cout)).astype(np.float32)).to(device)
+    g = torch.empty((N, layer.P, layer.Q, layer.Cout), device=device, dtype=bf)
+    for n0 in range(0, N, 8):      # in slabs of 8 images to bound the fp32 temporaries
+        n1 = min(N, n0 + 8)
+        shape = (n1 - n0, layer.P, layer.Q, layer.Cout)
+        normal = torch.randn(shape, device=device, generator=gen, dtype=torch.float32)
+        # Laplace(0, b) by inversion: -b sign(u) ln(1 - 2|u|), u uniform in (-1/2, 1/2); b = sigma / sqrt(2)
+        u = torch.rand(shape, device=device, generator=gen, dtype=torch.float32) - 0.5
+        lap = -torch.sign(u) * torch.log1p(-2.0 * u.abs().clamp_(max=0.49999997)) * (1.0 / np.sqrt(2.0))
+        g[n0:n1] = (torch.where(is_bell, normal, lap) * sigma).to(bf)
+    return x, w, g

@@ -54,14 +54,17 @@ def test_invalid_arguments_are_rejected_on_the_host(lib):
     null = None
     fake = ctypes.c_void_p(0x1000)      # never dereferenced: validation fails first
     odd = ctypes.c_void_p(0x1004)
-    st = lib.dai8_quantize_tensor(null, api.F32, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None)
+    st = lib.dai8_quantize_tensor(null, api.F32, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None, 0, None)
     assert st == api.ERR_INVALID_ARG
-    st = lib.dai8_quantize_tensor(fake, api.F32, api.NHWC, 0, 1, 1, 1, 0, fake, 0, 0, fake, None)
+    st = lib.dai8_quantize_tensor(fake, api.F32, api.NHWC, 0, 1, 1, 1, 0, fake, 0, 0, fake, None, 0, None)
     assert st == api.ERR_INVALID_ARG
-    st = lib.dai8_quantize_tensor(odd, api.F32, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None)
+    st = lib.dai8_quantize_tensor(odd, api.F32, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None, 0, None)
     assert st == api.ERR_INVALID_ARG
-    st = lib.dai8_quantize_tensor(fake, 7, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None)
+    st = lib.dai8_quantize_tensor(fake, 7, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, None, 0, None)
     assert st == api.ERR_INVALID_ARG
+    st = lib.dai8_quantize_tensor(fake, api.F32, api.NHWC, 1, 1, 1, 1, 0, fake, 0, 0, fake, fake, 8, None)
+    assert st == api.ERR_WORKSPACE
+    assert api.quantize_tensor_workspace_bytes() >= 16
     st = lib.dai8_quantize_grad(fake, api.F32, api.NHWC, 2, 64, 4, 4, None, fake, 0, fake, None, None,
                                 fake, None, 0, None, fake, 16, None)
     assert st == api.ERR_WORKSPACE

@@ -13,7 +13,7 @@ import torch
 from oracle import cpu as O
 from paper_2102_04782_b200 import api, synth
 
-from helpers import GradQuant, codes_to_nchw, dev_input, padding_is_zero, scalar
+from helpers import GradQuant, codes_to_nchw, dev_input, padding_is_zero, scalar, ws_bytes
 
 pytestmark = pytest.mark.gpu
 
@@ -177,6 +177,75 @@ def test_quantize_tensor(shape, layout, bf16):
     np.testing.assert_array_equal(codes_to_nchw(q, C), O.quantize(x, 0.5, stochastic=True, seed=11))
 
 
+# Tensors above 131072 codes leave the single-launch kernel for small tensors and take the
+# large-tensor kernels (layer-scale reduction, then the code kernels), which is what the benchmark
+# times.  One case per code path: NHWC with C = Cp (flat walk, nearest), NHWC with padded code channels
+# (C a vector multiple or not), NCHW activations, NCHW weights (transposed to [Cout][R][S][Cinp]), and
+# a length that is not a multiple of the grid stride.
+LARGE_TENSORS = [
+    # (N, C, H, W), layout
+    ((4, 64, 40, 40), api.NHWC),        # C = Cp: flat path
+    ((3, 48, 33, 35), api.NHWC),        # C = Cp, vector count not a multiple of the block size
+    ((4, 24, 48, 48), api.NHWC),        # C != Cp, C a multiple of the fp32 and bf16 vector
+    ((4, 20, 41, 43), api.NHWC),        # bf16: C not a vector multiple -> element-wise columns
+    ((8, 3, 100, 100), api.NHWC),       # stem-like
+    ((4, 40, 37, 41), api.NCHW),        # NCHW activation, ragged position tiles
+    ((512, 512, 3, 3), api.NCHW),       # VGG weights: rows of 9 elements
+    ((2, 130, 31, 33), api.NCHW),       # channel tiles with a ragged tail
+]
+
+
+@pytest.mark.parametrize("with_ws", [False, True])
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("shape,layout", LARGE_TENSORS)
+def test_quantize_tensor_large(shape, layout, bf16, with_ws):
+    """with_ws: the caller passes scratch memory, which lets flat tensors take the one-launch kernel
+    (scale and codes in one cooperative launch); without it the scale and the codes are two launches."""
+    N, C, H, W = shape
+    ws = ws_bytes(api.quantize_tensor_workspace_bytes()) if with_ws else None
+    Cp = api.padded_channels(C)
+    assert N * H * W * Cp > 131072
+    x = synth.activations(N, C, H, W, seed=71) - np.float32(0.3)
+    if bf16:
+        x = synth.round_to_bf16(x)
+    d = dev_input(x, bf16, layout)
+    for mode, given, rounding in ((api.SCALE_ABSMAX, 0.0, api.ROUND_NEAREST_EVEN),
+                                  (api.SCALE_GIVEN, 0.5, api.ROUND_NEAREST_EVEN),
+                                  (api.SCALE_GIVEN, 0.75, api.ROUND_STOCHASTIC),
+                                  (api.SCALE_ABSMAX, 0.0, api.ROUND_STOCHASTIC)):
+        q = torch.full((N, H, W, Cp), 55, dtype=torch.int8, device="cuda")
+        s = scalar(given)
+        api.quantize_tensor(d, layout, N, C, H, W, mode, s, rounding, 13, q, ws)
+        torch.cuda.synchronize()
+        sv = float(s.item())
+        if mode == api.SCALE_ABSMAX:
+            assert sv == float(np.abs(x).max())
+        else:
+            assert sv == given
+        want = O.quantize(x, sv, stochastic=rounding == api.ROUND_STOCHASTIC, seed=13)
+        np.testing.assert_array_equal(codes_to_nchw(q, C), want)
+        assert padding_is_zero(q, C)
+
+
+def test_quantize_tensor_benchmark_activation():
+    """X of the ResNet-50 conv2_x 1x1 256->64 layer at full size, (64, 256, 56, 56) bf16 NHWC: the
+    layer-scale reduction and the flat code kernel in the launch configuration the benchmark times."""
+    N, C, H, W = 64, 256, 56, 56
+    x = synth.round_to_bf16(synth.activations(N, C, H, W, seed=72) - np.float32(0.1))
+    d = dev_input(x, True, api.NHWC)
+    want = None
+    for ws in (None, ws_bytes(api.quantize_tensor_workspace_bytes())):
+        q = torch.full((N, H, W, C), 55, dtype=torch.int8, device="cuda")
+        s = scalar(0.0)
+        api.quantize_tensor(d, api.NHWC, N, C, H, W, api.SCALE_ABSMAX, s, api.ROUND_NEAREST_EVEN, 0, q, ws)
+        torch.cuda.synchronize()
+        assert api.get_device_status() == api.OK
+        assert float(s.item()) == float(np.abs(x).max())
+        if want is None:
+            want = O.quantize(x, float(s.item()))
+        np.testing.assert_array_equal(codes_to_nchw(q, C), want)
+
+
 def test_weight_layout_from_quantize_tensor():
     """Weights passed as an NCHW tensor (N=Cout, C=Cin, H=R, W=S) come out as [Cout][R][S][Cinp]."""
     w = synth.weights(8, 5, 3, 3, seed=8)
@@ -193,6 +262,15 @@ def test_config2_full_size_grad_quant():
     """ResNet-50 conv2_x 3x3 layer: dY (64,64,56,56) bf16 NHWC, the launch configuration the
     benchmark times; full-tensor comparison (the oracle's O(elements) parts run in seconds)."""
     g, _, _ = synth.channel_mixed_grad(64, 64, 56, 56, seed=9)
+    g = synth.round_to_bf16(g)
+    check_grad_quant(g, True, api.NHWC, iters=2)
+
+
+def test_benchmark_gradient_full_size():
+    """dY of the ResNet-50 conv2_x 1x1 64->256 layer, (64, 256, 56, 56) bf16 NHWC, 102.8 MB: more than a
+    CTA keeps resident in shared memory, so part of every CTA's range cycles through the piece ring and
+    is fetched again in the second sweep.  Whole tensor, every stage, two iterations."""
+    g, _, _ = synth.channel_mixed_grad(64, 256, 56, 56, seed=10)
     g = synth.round_to_bf16(g)
     check_grad_quant(g, True, api.NHWC, iters=2)
 
