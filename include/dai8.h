@@ -208,8 +208,9 @@ dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, const float
 
 /* Kernel family selection for the convolutions (process-wide, host side): 0 = automatic
  * (tensor-core kernels where the geometry allows, direct kernels otherwise), 1 = direct kernels
- * only, 2 = tensor-core kernels only (DAI8_ERR_UNSUPPORTED where they do not apply).  Used by
- * the tests to compare the two families bit for bit. */
+ * only, 2 = tensor-core kernels only (DAI8_ERR_UNSUPPORTED where they do not apply), 3 = like 2 but
+ * multi-tap filters use the copy engine's im2col loads even where the patch form applies.  Used
+ * by the tests to compare the kernel families bit for bit. */
 void dai8_set_conv_backend(int mode);
 
 /* Number of kernels the library has launched from this process so far (host counter). */

@@ -64,7 +64,11 @@ int packed_bwd_data(const ConvShape& cs, ConvShape* as_fwd, ConvShape* pw) {
 
 using namespace dai8;
 
-extern "C" void dai8_set_conv_backend(int mode) { g_backend.store(mode < 0 || mode > 2 ? 0 : mode); }
+extern "C" void dai8_set_conv_backend(int mode) {
+  if (mode < 0 || mode > 3) mode = 0;
+  set_halo_disabled(mode == 3);
+  g_backend.store(mode == 3 ? 2 : mode);
+}
 
 extern "C" size_t dai8_conv_workspace_bytes(dai8_conv_op op, const dai8_conv_geom* geom) {
   if (check_geom(geom) != DAI8_OK) return 0;

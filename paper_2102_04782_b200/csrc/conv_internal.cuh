@@ -112,6 +112,21 @@ inline int packed_small_cin(const ConvShape& cs, ConvShape* pw) {
 dai8_status pack_small_cin(const int8_t* qX, const ConvShape& cs, int Kp, int8_t* A, cudaStream_t st);
 dai8_status pack_small_cin_weights(const int8_t* qW, const ConvShape& cs, int Kp, int8_t* Wp, cudaStream_t st);
 
+// ---- tensor-core kernel for multi-tap filters at stride 1 (conv_halo.cu) --------------------------
+// D[n][y][x][j] = sum over taps (r, s) and channels k of A[n][y + r + lower_h][x + s + lower_w][k] * B[j][r*S+s][k]
+struct HaloProblem {
+  const int8_t* A;   // [N][H][W][Kc] codes
+  const int8_t* B;   // K-major [Brows][R*S][Kc], or (b_mn) the forward weights [Bk][b_taps][Brows] read in place
+  int N, H, W, Kc, Brows;
+  int P, Q, Nout, R, S, lower_h, lower_w;
+  int b_mn = 0, Bk = 0, b_taps = 0, b_tap_base = 0, b_tap_dr = 0, b_tap_ds = 0;
+};
+bool halo_supported(const HaloProblem& pb, dai8_dtype out_dtype, dai8_layout out_layout);
+dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb, const ConvOut& out, cudaStream_t st);
+// 0: the patch form (conv_halo.cu) wherever it applies; 1: the im2col form only (set by the tests through
+// dai8_set_conv_backend to compare the two forms)
+void set_halo_disabled(int disabled);
+
 // ---- tensor-core (tcgen05) kernels: see conv_umma.cu for the geometries covered ------------------
 bool umma_fwd_supported(const ConvShape& cs);
 bool umma_bwd_data_supported(const ConvShape& cs);

@@ -27,7 +27,7 @@
 #include <cstring>
 #include <mutex>
 
-#include "conv_internal.cuh"
+#include "umma_ptx.cuh"
 
 namespace dai8 {
 
@@ -50,184 +50,12 @@ unsigned int* device_status_address() {
 
 namespace {
 
-constexpr int kBM = 128;                      // output pixels per tile (MMA M)
+using namespace umma;
+
 constexpr int kThreadsIgemm = 192;      // weight-gradient kernel: TMA warp, MMA warp, 4 epilogue warps
 constexpr int kEpiWarps = 8;             // persistent kernel: two epilogue warps per tensor-memory lane quarter
 constexpr int kThreadsPersist = 64 + 32 * kEpiWarps;
 constexpr int kOutBlockBytes = 32 * 128; // epilogue staging block: 32 pixel rows x 128 bytes of channels
-constexpr long long kTimeoutCycles = 2000000000LL;  // about one second
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  return ok != 0;
-}
-// Bounded wait.  Returns false if the CTA is aborting (this wait or another one expired).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const long long t0 = clock64();
-  for (;;) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (*abort_flag) return false;
-    if (clock64() - t0 > kTimeoutCycles) {
-      *abort_flag = 1u;
-      atomicExch(&g_device_status, (unsigned int)DAI8_ERR_TIMEOUT);
-      return false;
-    }
-  }
-}
-
-__device__ __forceinline__ void tma_load_im2col_4d(const CUtensorMap* map, uint64_t* bar, void* dst, int c,
-                                                   int w, int h, int n, uint16_t off_w, uint16_t off_h) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c), "r"(w), "r"(h),
-        "r"(n), "h"(off_w), "h"(off_h)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_tile_3d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0,
-                                                 int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
-}
-// Shared -> global tile store (2D), tracked by the issuing thread's bulk async-group.
-__device__ __forceinline__ void tma_store_tile_2d(const CUtensorMap* map, const void* src, int c0, int c1) {
-  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(smem_u32(src)), "r"(c0), "r"(c1) : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
-  asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
-}
-
-// Variants for the single-thread issue loops: shared-memory addresses are passed as 32-bit values
-// computed once, so that no generic-to-shared conversion or 64-bit arithmetic sits between two
-// issues (these loops are latency chains of one thread).
-__device__ __forceinline__ void mbar_expect_tx_a(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void tma_load_im2col_4d_a(uint64_t map, uint32_t bar, uint32_t dst, int c, int w, int h,
-                                                     int n, uint16_t off_w, uint16_t off_h) {
-  asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-      : "memory");
-}
-__device__ __forceinline__ void tma_load_tile_3d_a(uint64_t map, uint32_t bar, uint32_t dst, int c0, int c1, int c2) {
-  asm volatile(
-      "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
-      " [%0], [%1, {%3, %4, %5}], [%2];"
-      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-      : "memory");
-}
-__device__ __forceinline__ void tc_commit_a(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// The 64-bit matrix descriptor of a K-major tile is a constant high word and a low word that holds
-// the 16-byte-granular address: stepping through chunks and K slices is a 32-bit addition.
-__device__ __forceinline__ uint32_t kmajor_desc_hi(int kc_bytes) {
-  const uint32_t layout = kc_bytes == 128 ? 2u : (kc_bytes == 64 ? 4u : 6u);
-  const uint32_t sbo = (uint32_t)(8 * kc_bytes) >> 4;
-  return sbo | (1u << 14) | (layout << 29);
-}
-__device__ __forceinline__ uint32_t kmajor_desc_lo(uint32_t saddr) { return ((saddr & 0x3FFFFu) >> 4) | (1u << 16); }
-__device__ __forceinline__ void mma_i8_parts(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc,
-                                             uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %5, 0;\n\t"
-      "mov.b64 da, {%1, %3};\n\t"
-      "mov.b64 db, {%2, %3};\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-// The same with separate high words for A and B (B in another layout than A).
-__device__ __forceinline__ void mma_i8_parts2(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                              uint32_t idesc, uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-      "setp.ne.b32 p, %6, 0;\n\t"
-      "mov.b64 da, {%1, %2};\n\t"
-      "mov.b64 db, {%3, %4};\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %5, p;\n\t}"
-      ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(dst_smem)),
-               "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
-               : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem], int8 x int8 -> int32, one instruction covers K = 32.
-__device__ __forceinline__ void mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                       uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-      : "memory");
-}
-// 32 lanes x 16 consecutive 32-bit columns: thread i of the warp gets lane (base lane + i).
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, int (&v)[16]) {
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-      : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor for a K-major operand tile [rows][kc_bytes] written by TMA with
-// the matching swizzle (rows of 32/64/128 bytes; groups of 8 rows are `8*kc_bytes` apart).
-__device__ __forceinline__ uint64_t kmajor_desc(uint32_t saddr, int kc_bytes) {
-  const uint64_t layout = kc_bytes == 128 ? 2ull : (kc_bytes == 64 ? 4ull : 6ull);
-  const uint64_t sbo = (uint64_t)(8 * kc_bytes) >> 4;
-  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | (1ull << 16) | (sbo << 32) | (1ull << 46) | (layout << 61);
-}
-// Instruction descriptor: int32 accumulator, signed 8-bit A and B, both K-major, M = 128, N = bn.
-__device__ __forceinline__ uint32_t idesc_i8_kmajor(int bn) {
-  return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(kBM >> 4) << 24);
-}
 
 struct IgemmParams {
   int Mtot, P, Q;        // output pixels and output extent (pixel m = (n*P + p)*Q + q)
@@ -348,7 +176,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
         int c = 0, k0 = 0, kchunk = 0, r = 0, ss = 0;    // chunk, its channel offset, tap row and column
         for (int it = 0; it < kit; ++it) {
-          if (!first_pass && !mbar_wait(&empty_bar[stage], phase ^ 1u, &abort_flag)) { ok = false; break; }
+          if (!first_pass && !mbar_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, &g_device_status)) { ok = false; break; }
           const int nch = min(total_chunks - c, G);
           const uint32_t bar = full_a + 8u * (uint32_t)stage;
           mbar_expect_tx_a(bar, (uint32_t)(nch * chunk_pair_bytes));
@@ -384,7 +212,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       const uint32_t b_hi = b_mn ? kmajor_desc_hi(prm.b_bw) : kmajor_desc_hi(prm.kc_bytes);
       const uint32_t b_lbo = b_mn ? ((uint32_t)(prm.kc_bytes * prm.b_bw) >> 4) << 16 : (1u << 16);
       const uint32_t b_kstep = b_mn ? (uint32_t)(32 * prm.b_bw) >> 4 : 2u;
-      bool ok = !prm.b_resident || mbar_wait(&b_full, 0, &abort_flag);
+      bool ok = !prm.b_resident || mbar_wait(&b_full, 0, &abort_flag, &g_device_status);
       int stage = 0, tile_i = 0;
       uint32_t phase = 0;
       const int kk_n = prm.kc_bytes / 32, G = prm.G, nst = prm.stages, kit = prm.k_iters;
@@ -398,7 +226,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       const uint32_t empty_a = smem_u32(&empty_bar[0]);
       for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_i) {
         const int buf = tile_i & 1;
-        if (tile_i >= 2) ok = mbar_wait(&acc_empty[buf], ((tile_i >> 1) - 1) & 1, &abort_flag);
+        if (tile_i >= 2) ok = mbar_wait(&acc_empty[buf], ((tile_i >> 1) - 1) & 1, &abort_flag, &g_device_status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * prm.BN);
@@ -406,7 +234,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         int c = 0;
         uint32_t bres = bres_lo;                 // descriptor low word of the next resident weight chunk
         for (int it = 0; it < kit; ++it) {
-          ok = mbar_wait(&full_bar[stage], phase, &abort_flag);
+          ok = mbar_wait(&full_bar[stage], phase, &abort_flag, &g_device_status);
           if (!ok) break;
           tc_fence_after();
           const int nch = min(total_chunks - c, G);
@@ -440,7 +268,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     int tile_i = 0, n_store = 0;
     for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++tile_i) {
       const int buf = tile_i & 1;
-      if (!mbar_wait(&acc_full[buf], (tile_i >> 1) & 1, &abort_flag)) break;
+      if (!mbar_wait(&acc_full[buf], (tile_i >> 1) & 1, &abort_flag, &g_device_status)) break;
       tc_fence_after();
       const int m_tile = t / prm.n_tiles;
       const int n0 = (t - m_tile * prm.n_tiles) * prm.BN;
@@ -584,38 +412,6 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
 // ---------------------------------------------------------------------------------------------
 // Host side: tensor maps and launch
 // ---------------------------------------------------------------------------------------------
-using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-using EncodeIm2colFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                    const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t,
-                                    const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                    CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn g_encode_tiled = nullptr;
-EncodeIm2colFn g_encode_im2col = nullptr;
-std::once_flag g_driver_once;
-
-bool load_driver_entry_points() {
-  std::call_once(g_driver_once, [] {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
-    fn = nullptr;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess)
-      g_encode_im2col = reinterpret_cast<EncodeIm2colFn>(fn);
-  });
-  return g_encode_tiled && g_encode_im2col;
-}
-
-CUtensorMapSwizzle swizzle_for(int kc_bytes) {
-  return kc_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
-                         : (kc_bytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
-}
-
 // Contraction bytes per chunk for a code tensor with `cp` channels (multiple of 16, >= 32).
 int chunk_bytes_for(int cp) {
   if (cp % 128 == 0) return 128;
@@ -647,22 +443,9 @@ bool igemm_supported(const IgemmProblem& pb) {
   return true;
 }
 
-int sm_count() {
-  static int cached = 0;
-  if (cached == 0) {
-    int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
-      cached = sms;
-    else
-      return 148;
-  }
-  return cached;
-}
-
 dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* sb, const ConvOut& out,
                          cudaStream_t st) {
-  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
+  if (!driver_api().ok()) return DAI8_ERR_CUDA;
   IgemmParams prm;
   prm.Mtot = pb.N * pb.P * pb.Q;
   prm.P = pb.P; prm.Q = pb.Q; prm.Nout = pb.Nout; prm.R = pb.R; prm.S = pb.S;
@@ -713,7 +496,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const cuuint64_t strides[1] = {(cuuint64_t)pb.Nout * out_es};
     const cuuint32_t box[2] = {128, 32};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode_tiled(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, out.ptr, dims, strides, box, estr,
+    CUresult r = driver_api().tiled(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, out.ptr, dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
@@ -725,7 +508,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const int lower[2] = {pb.lower_w, pb.lower_h};
     const int upper[2] = {pb.lower_w + (pb.Q - 1) * pb.sw - (pb.Wi - 1), pb.lower_h + (pb.P - 1) * pb.sh - (pb.Hi - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)pb.sw, (cuuint32_t)pb.sh, 1};
-    CUresult r = g_encode_im2col(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides,
+    CUresult r = driver_api().im2col(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides,
                                  lower, upper, (cuuint32_t)prm.kc_bytes, (cuuint32_t)kBM, estr,
                                  CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -738,7 +521,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Brows, (cuuint64_t)pb.b_taps * pb.Brows};
     const cuuint32_t box[3] = {(cuuint32_t)prm.b_bw, 1, (cuuint32_t)prm.kc_bytes};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode_tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
+    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.b_bw),
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
@@ -747,18 +530,14 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.R * pb.S * pb.Kc};
     const cuuint32_t box[3] = {(cuuint32_t)prm.kc_bytes, 1, (cuuint32_t)prm.BN};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode_tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
+    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   const size_t smem_bytes = (size_t)(prm.b_resident ? b_res : 0) + stage_out_bytes + (size_t)stages * stage_bytes + 1024;
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(igemm_kmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 2048);
-  });
-  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, igemm_kmajor_kernel, 227 * 1024 - 2048) != cudaSuccess) return DAI8_ERR_CUDA;
   // one persistent CTA per SM; with resident weights a CTA keeps its output-channel tile
   const int num_tiles = prm.m_tiles * prm.n_tiles;
   int ctas = sm_count();
@@ -767,6 +546,26 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   DAI8_RETURN_IF_CUDA(launch_dependent(igemm_kmajor_kernel, dim3((unsigned)ctas), dim3(kThreadsPersist), smem_bytes, st, mapA, mapB, mapC, prm));
   note_launch();
   return DAI8_OK;
+}
+
+std::atomic<int> g_halo_disabled{0};
+
+// The patch form of a stride-1, identity-placed problem, if conv_halo.cu takes it.
+bool as_halo(const IgemmProblem& pb, HaloProblem& h) {
+  if (g_halo_disabled.load(std::memory_order_relaxed)) return false;
+  if (pb.sh != 1 || pb.sw != 1 || pb.R * pb.S <= 1) return false;
+  if (pb.oH != pb.P || pb.oW != pb.Q || pb.oh_step != 1 || pb.ow_step != 1 || pb.oh_off != 0 || pb.ow_off != 0) return false;
+  h.A = pb.A; h.B = pb.B; h.N = pb.N; h.H = pb.Hi; h.W = pb.Wi; h.Kc = pb.Kc; h.Brows = pb.Brows;
+  h.P = pb.P; h.Q = pb.Q; h.Nout = pb.Nout; h.R = pb.R; h.S = pb.S; h.lower_h = pb.lower_h; h.lower_w = pb.lower_w;
+  h.b_mn = pb.b_mn; h.Bk = pb.Bk; h.b_taps = pb.b_taps; h.b_tap_base = pb.b_tap_base; h.b_tap_dr = pb.b_tap_dr; h.b_tap_ds = pb.b_tap_ds;
+  return true;
+}
+
+// Patch form where it applies, im2col form otherwise.
+dai8_status launch_conv(const IgemmProblem& pb, const float* sa, const float* sb, const ConvOut& out, cudaStream_t st) {
+  HaloProblem h;
+  if (as_halo(pb, h) && halo_supported(h, out.dtype, out.layout)) return launch_halo(h, sa, sb, out, st);
+  return launch_igemm(pb, sa, sb, out, st);
 }
 
 IgemmProblem fwd_problem(const int8_t* qX, const int8_t* qW, const ConvShape& cs) {
@@ -915,7 +714,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
       tma_prefetch_desc(&mapX);
       for (int it = 0; it < k_iters; ++it) {
         const int s = it % prm.stages;
-        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag)) break;
+        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag, &g_device_status)) break;
         const int pix0 = (chunk_begin + it) * prm.kp;
         const int q0 = pix0 % prm.Q;
         const int t = pix0 / prm.Q;
@@ -945,7 +744,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
       bool ok = true;
       for (int it = 0; it < k_iters && ok; ++it) {
         const int s = it % prm.stages;
-        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag);
+        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag, &g_device_status);
         if (!ok) break;
         tc_fence_after();
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
@@ -965,7 +764,7 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
     }
   } else {
     const int quarter = warp & 3;
-    const bool ok = mbar_wait(&acc_bar, 0, &abort_flag);
+    const bool ok = mbar_wait(&acc_bar, 0, &abort_flag, &g_device_status);
     tc_fence_after();
     if (ok) {
       // Tensor-memory lane = output channel: every lane holds 32 consecutive input channels of its
@@ -1075,7 +874,7 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
 
 dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs, int* acc, int* splits_out,
                          cudaStream_t st) {
-  if (!load_driver_entry_points()) return DAI8_ERR_CUDA;
+  if (!driver_api().ok()) return DAI8_ERR_CUDA;
   WgradParams prm;
   int ngroups = 0, co_tiles = 0;
   const int ksplit = plan_wgrad(cs, prm, &ngroups, &co_tiles);
@@ -1091,7 +890,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
     const cuuint64_t strides[1] = {(cuuint64_t)cs.Coutp};
     const cuuint32_t box[2] = {128, (cuuint32_t)prm.kp};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = g_encode_tiled(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box,
+    CUresult r = driver_api().tiled(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box,
                                 estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
@@ -1102,20 +901,15 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
     const int lower[2] = {-cs.pw, -cs.ph};
     const int upper[2] = {-cs.pw + (cs.Q - 1) * cs.sw - (cs.W - 1), -cs.ph + (cs.P - 1) * cs.sh - (cs.H - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)cs.sw, (cuuint32_t)cs.sh, 1};
-    CUresult r = g_encode_im2col(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(qX), dims, strides, lower,
+    CUresult r = driver_api().im2col(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(qX), dims, strides, lower,
                                  upper, (cuuint32_t)prm.bw, (cuuint32_t)prm.kp, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                  swizzle_for(prm.bw), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
-  static std::once_flag attr_once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(attr_once, [] {
-    attr_err = cudaFuncSetAttribute(wgrad_mnmajor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kWgradSmem + 1024);
-  });
-  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, wgrad_mnmajor_kernel, kWgradSmem + 1024) != cudaSuccess) return DAI8_ERR_CUDA;
   const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
   DAI8_RETURN_IF_CUDA(launch_dependent(wgrad_mnmajor_kernel, grid, dim3(kThreadsIgemm), smem_bytes, st, mapG, mapX, prm));
   note_launch();
@@ -1123,6 +917,8 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
 }
 
 }  // namespace
+
+void set_halo_disabled(int disabled) { g_halo_disabled.store(disabled ? 1 : 0, std::memory_order_relaxed); }
 
 bool umma_fwd_supported(const ConvShape& cs) { return igemm_supported(fwd_problem(nullptr, nullptr, cs)); }
 
@@ -1139,7 +935,7 @@ bool umma_bwd_filter_supported(const ConvShape& cs) { return umma_bwd_filter_spl
 
 dai8_status umma_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW, const ConvShape& cs,
                      const ConvOut& out, cudaStream_t st) {
-  return launch_igemm(fwd_problem(qX, qW, cs), sX, sW, out, st);
+  return launch_conv(fwd_problem(qX, qW, cs), sX, sW, out, st);
 }
 
 dai8_status umma_bwd_data(const int8_t* gq, const int8_t* qW, int8_t* wT, const float* gmax, const float* sW,
@@ -1173,7 +969,7 @@ dai8_status umma_bwd_data(const int8_t* gq, const int8_t* qW, int8_t* wT, const 
       pb.b_tap_dr = cs.sh * cs.S;
       pb.b_tap_ds = cs.sw;
     }
-    r = launch_igemm(pb, gmax, sW, out, st);
+    r = launch_conv(pb, gmax, sW, out, st);
     if (r != DAI8_OK) return r;
   }
   return DAI8_OK;

@@ -62,6 +62,34 @@ inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
 // DAI8_OK if the current device is compute capability 10.x, else DAI8_ERR_ARCH / DAI8_ERR_CUDA.
 dai8_status check_device_arch();
 
+// Multiprocessors of the current device (looked up once per device).
+inline int sm_count() {
+  static std::atomic<int> cached[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+  int sms = cached[dev].load(std::memory_order_relaxed);
+  if (sms == 0) {
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+    cached[dev].store(sms, std::memory_order_relaxed);
+  }
+  return sms;
+}
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per device for one kernel: `slot` is a
+// per-kernel array of 64 flags.
+template <typename K>
+inline cudaError_t set_max_smem_once(std::atomic<int>* slot, K kernel, int bytes) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+  if (slot[dev].load(std::memory_order_acquire) == 1) return cudaSuccess;
+  e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  if (e == cudaSuccess) slot[dev].store(1, std::memory_order_release);
+  return e;
+}
+
+
 __device__ __forceinline__ float to_f32(float v) { return v; }
 __device__ __forceinline__ float to_f32(bf16_t v) { return __uint_as_float((uint32_t)v.bits << 16); }
 

@@ -1854,20 +1854,23 @@ struct FusedConfig {
   bool coop = false;
 };
 
+// Properties of the current device, looked up once per device.
 const FusedConfig& fused_config() {
-  static FusedConfig cfg;
-  static std::once_flag once;
-  std::call_once(once, [] {
-    int dev = 0, coop = 0, sms = 0, smem = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return;
+  static FusedConfig cfgs[64];
+  static std::once_flag once[64];
+  static const FusedConfig none;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return none;
+  std::call_once(once[dev], [dev] {
+    int coop = 0, sms = 0, smem = 0;
     cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    cfg.sms = sms;
-    cfg.smem_max = (size_t)smem;
-    cfg.coop = coop != 0 && sms > 0;
+    cfgs[dev].sms = sms;
+    cfgs[dev].smem_max = (size_t)smem;
+    cfgs[dev].coop = coop != 0 && sms > 0;
   });
-  return cfg;
+  return cfgs[dev];
 }
 
 template <typename T, int VE, bool DUAL, bool IDX32>
@@ -1907,12 +1910,8 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   }
   const size_t smem = fixed + (size_t)slots * piece_bytes;
   auto kern = gvq_fused_nhwc_kernel<T, VE, DUAL, IDX32>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] {
-    attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(cfg.smem_max - 1024));
-  });
-  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, kern, (int)(cfg.smem_max - 1024)) != cudaSuccess) return DAI8_ERR_CUDA;
   void* args[] = {(void*)&dY, (void*)&a};
   DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFusedThreads), args, smem, st));
   note_launch(1);
@@ -1941,15 +1940,11 @@ dai8_status launch_columns(const T* dY, ColArgs& a, bool dual, int grid, size_t 
   a.inv_M = 1.0 / M;
   a.inv_denom = denom > 0.0 ? 1.0 / denom : 0.0;
   void* args[] = {(void*)&dY, (void*)&a};
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] {
-    const int lim = (int)fused_config().smem_max - 8192;
-    attr_err = cudaFuncSetAttribute(gvq_columns_kernel<T, VE, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-    if (attr_err == cudaSuccess)
-      attr_err = cudaFuncSetAttribute(gvq_columns_kernel<T, VE, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
-  });
-  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  static std::atomic<int> attr_done[2][64];
+  const int lim = (int)fused_config().smem_max - 8192;
+  if (set_max_smem_once(attr_done[0], gvq_columns_kernel<T, VE, true>, lim) != cudaSuccess ||
+      set_max_smem_once(attr_done[1], gvq_columns_kernel<T, VE, false>, lim) != cudaSuccess)
+    return DAI8_ERR_CUDA;
   if (dual)
     DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)gvq_columns_kernel<T, VE, true>, dim3((unsigned)grid), dim3(kFT), args, smem, st));
   else
@@ -2161,12 +2156,8 @@ dai8_status launch_quantize_flat_fused(const T* x, int64_t nvec, float* scale, i
   a.status = device_status_address();
   if (!a.status) return DAI8_ERR_CUDA;
   auto kern = quantize_flat_fused_kernel<T>;
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [&] {
-    attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kQtMaxSlots * kQtPieceBytes);
-  });
-  if (attr_err != cudaSuccess) return DAI8_ERR_CUDA;
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, kern, kQtMaxSlots * kQtPieceBytes) != cudaSuccess) return DAI8_ERR_CUDA;
   DAI8_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, 16, st));
   void* args[] = {(void*)&a};
   DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kFusedThreads), args,

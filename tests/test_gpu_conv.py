@@ -102,13 +102,29 @@ TC_GEOMS = [
     (1, 32, 32, 70, 70, 5, 5, 1, 2),
     (2, 384, 130, 16, 16, 1, 1, 1, 0),
     (4, 128, 128, 20, 20, 1, 1, 2, 0),
+    # multi-tap filters at stride 1 whose output splits into 16 x 8 patches with little waste: the patch
+    # form of the forward / input-gradient kernel (one box per tap column instead of one load per tap)
+    (2, 64, 64, 32, 40, 3, 3, 1, 1),        # whole tiles, 64-byte rows, resident weights
+    (2, 64, 64, 31, 46, 3, 3, 1, 1),        # ragged tiles: clipped stores, zero-filled loads
+    (2, 128, 256, 48, 32, 3, 3, 1, 1),      # 128-byte rows, streamed weights, 256-wide accumulators
+    (2, 256, 128, 32, 32, 3, 3, 1, 1),      # two channel chunks per tap
+    (2, 96, 80, 32, 32, 3, 3, 1, 1),        # ragged channel chunk, 80 output channels
+    (1, 32, 48, 64, 72, 5, 5, 1, 2),        # 5x5 filter, 32-byte rows
+    (2, 64, 512, 32, 32, 3, 3, 1, 1),       # two accumulator tiles across the output channels
+    (3, 64, 64, 47, 32, 3, 3, 1, 0),        # no padding: output 45 x 30
+    (1, 32, 512, 64, 64, 3, 3, 1, 1),       # resident weights with two accumulator tiles per pixel tile
+    (4, 64, 64, 28, 28, 3, 3, 1, 1),        # 28 wide: patches of 4 rows x 32 columns
+    (8, 64, 128, 24, 16, 3, 3, 1, 1),       # 16 wide: patches of 8 rows x 16 columns
+    (2, 64, 48, 30, 60, 3, 3, 1, 1),        # 4 x 32 patches, ragged in both directions, 48 output channels
 ]
 
 
+@pytest.mark.parametrize("backend", [2, 3])
 @pytest.mark.parametrize("g", TC_GEOMS)
-def test_tensor_core_kernels_bit_exact(g):
+def test_tensor_core_kernels_bit_exact(g, backend):
     """Backend 2 = tensor-core kernels only: a geometry they do not take raises instead of being
-    silently served by the direct kernels."""
+    silently served by the direct kernels.  Backend 3 = the same with the im2col form of the forward /
+    input-gradient kernel even where the patch form applies."""
     N, Cin, Cout, H, W, R, S, st, pad = g
     rng = np.random.default_rng(33)
     P, Q = O.out_hw(H, W, R, S, st, pad)
@@ -116,7 +132,7 @@ def test_tensor_core_kernels_bit_exact(g):
     s_c = np.ones(Cout, np.float32)
     stride1 = st == 1
     gg = geom(*g)
-    api.set_conv_backend(2)
+    api.set_conv_backend(backend)
     try:
         for layout in (api.NHWC, api.NCHW):
             Y = torch.empty((N, P, Q, Cout) if layout == api.NHWC else (N, Cout, P, Q), dtype=torch.int32, device="cuda")
@@ -150,7 +166,7 @@ def test_tensor_core_backend_refuses_small_shapes():
         api.set_conv_backend(0)
 
 
-@pytest.mark.parametrize("g", [GEOMS[0], GEOMS[3], GEOMS[6], TC_GEOMS[2], TC_GEOMS[6]])
+@pytest.mark.parametrize("g", [GEOMS[0], GEOMS[3], GEOMS[6], TC_GEOMS[2], TC_GEOMS[6], TC_GEOMS[11], TC_GEOMS[12]])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_dequantized_outputs(g, dtype):
     N, Cin, Cout, H, W, R, S, st, pad = g
