@@ -85,6 +85,25 @@ struct IgemmParams {
   const float* sb;
 };
 
+// The MMAs of one pipeline stage: up to 4/KK chunks of KK instructions (K = 32 each), issued by one
+// lane from straight-line code.  What a tcgen05.mma costs the issuing thread depends on the code
+// around it far more than on the instruction itself (about 180 cycles each from a loop nest, 50 to 100
+// from an unrolled block inside a single elected-lane region), hence the template over the chunk width.
+template <int KK>
+__device__ __forceinline__ void issue_stage(uint32_t d_tmem, uint32_t a_lo, uint32_t a_step, uint32_t a_hi, uint32_t b_lo,
+                                            uint32_t b_step, uint32_t b_kstep, uint32_t b_hi, uint32_t idesc, int nch,
+                                            uint32_t accumulate) {
+#pragma unroll
+  for (int j = 0; j < 4 / KK; ++j) {
+    if (j < nch) {
+#pragma unroll
+      for (int kk = 0; kk < KK; ++kk)
+        mma_i8_parts2(d_tmem, a_lo + (uint32_t)j * a_step + 2u * kk, a_hi, b_lo + (uint32_t)j * b_step + b_kstep * kk, b_hi, idesc,
+                      (j | kk) ? 1u : accumulate);
+    }
+  }
+}
+
 // Persistent: a CTA walks over output tiles t = blockIdx.x, blockIdx.x + gridDim.x, ...  The operand
 // ring keeps filling across tile boundaries and the accumulator is double-buffered in tensor
 // memory, so the epilogue of one tile overlaps the loads and MMAs of the next.  When the weight
@@ -204,55 +223,53 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      const bool b_mn = prm.b_mn != 0;
-      const uint32_t idesc = idesc_i8_kmajor(prm.BN) | (b_mn ? (1u << 16) : 0u);
-      // MN-major B: the low descriptor word carries the distance between the boxes (one box =
-      // kc rows of b_bw bytes), a K slice of 32 rows lies 32 * b_bw bytes further
-      const uint32_t b_hi = b_mn ? kmajor_desc_hi(prm.b_bw) : kmajor_desc_hi(prm.kc_bytes);
-      const uint32_t b_lbo = b_mn ? ((uint32_t)(prm.kc_bytes * prm.b_bw) >> 4) << 16 : (1u << 16);
-      const uint32_t b_kstep = b_mn ? (uint32_t)(32 * prm.b_bw) >> 4 : 2u;
-      bool ok = !prm.b_resident || mbar_wait(&b_full, 0, &abort_flag, &g_device_status);
-      int stage = 0, tile_i = 0;
-      uint32_t phase = 0;
-      const int kk_n = prm.kc_bytes / 32, G = prm.G, nst = prm.stages, kit = prm.k_iters;
-      const bool resident = prm.b_resident != 0;
-      const uint32_t dhi = kmajor_desc_hi(prm.kc_bytes);
-      const uint32_t ring_lo = kmajor_desc_lo(smem_u32(ring));
-      const uint32_t bres_lo = ((smem_u32(smem) & 0x3FFFFu) >> 4) | b_lbo;
-      const uint32_t lbo_fix = b_lbo - (1u << 16);   // turns a K-major low word into B's
-      const uint32_t stage_step = (uint32_t)stage_bytes >> 4, a_step = (uint32_t)a_chunk_bytes >> 4,
-                     b_step = (uint32_t)b_chunk_bytes >> 4;
-      const uint32_t empty_a = smem_u32(&empty_bar[0]);
-      for (int t = blockIdx.x; t < num_tiles && ok; t += gridDim.x, ++tile_i) {
-        const int buf = tile_i & 1;
-        if (tile_i >= 2) ok = mbar_wait(&acc_empty[buf], ((tile_i >> 1) - 1) & 1, &abort_flag, &g_device_status);
-        if (!ok) break;
+    // MMA issue.  The whole warp runs the loops (trip counts depend only on the launch parameters; a
+    // wait that gives up sets the abort flag, after which every later wait returns at once), and one
+    // elected lane issues a stage's instructions from straight-line code: see issue_stage().
+    const bool leader = elect_one();
+    const bool b_mn = prm.b_mn != 0;
+    const uint32_t idesc = idesc_i8_kmajor(prm.BN) | (b_mn ? (1u << 16) : 0u);
+    // MN-major B: the low descriptor word carries the distance between the boxes (one box =
+    // kc rows of b_bw bytes), a K slice of 32 rows lies 32 * b_bw bytes further
+    const uint32_t b_hi = b_mn ? kmajor_desc_hi(prm.b_bw) : kmajor_desc_hi(prm.kc_bytes);
+    const uint32_t b_lbo = b_mn ? ((uint32_t)(prm.kc_bytes * prm.b_bw) >> 4) << 16 : (1u << 16);
+    const uint32_t b_kstep = b_mn ? (uint32_t)(32 * prm.b_bw) >> 4 : 2u;
+    if (prm.b_resident) mbar_wait(&b_full, 0, &abort_flag, &g_device_status);
+    int stage = 0, tile_i = 0;
+    uint32_t phase = 0;
+    const int kk_n = prm.kc_bytes / 32, G = prm.G, nst = prm.stages, kit = prm.k_iters;
+    const bool resident = prm.b_resident != 0;
+    const uint32_t dhi = kmajor_desc_hi(prm.kc_bytes);
+    const uint32_t ring_lo = kmajor_desc_lo(smem_u32(ring));
+    const uint32_t bres_lo = ((smem_u32(smem) & 0x3FFFFu) >> 4) | b_lbo;
+    const uint32_t lbo_fix = b_lbo - (1u << 16);   // turns a K-major low word into B's
+    const uint32_t stage_step = (uint32_t)stage_bytes >> 4, a_step = (uint32_t)a_chunk_bytes >> 4,
+                   b_step = (uint32_t)b_chunk_bytes >> 4;
+    const uint32_t empty_a = smem_u32(&empty_bar[0]);
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++tile_i) {
+      const int buf = tile_i & 1;
+      if (tile_i >= 2) mbar_wait(&acc_empty[buf], ((tile_i >> 1) - 1) & 1, &abort_flag, &g_device_status);
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + (uint32_t)(buf * prm.BN);
+      int c = 0;
+      uint32_t bres = bres_lo;                 // descriptor low word of the next resident weight chunk
+      for (int it = 0; it < kit; ++it) {
+        mbar_wait(&full_bar[stage], phase, &abort_flag, &g_device_status);
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * prm.BN);
-        uint32_t accumulate = 0;
-        int c = 0;
-        uint32_t bres = bres_lo;                 // descriptor low word of the next resident weight chunk
-        for (int it = 0; it < kit; ++it) {
-          ok = mbar_wait(&full_bar[stage], phase, &abort_flag, &g_device_status);
-          if (!ok) break;
-          tc_fence_after();
-          const int nch = min(total_chunks - c, G);
-          uint32_t a_lo = ring_lo + (uint32_t)stage * stage_step;
-          uint32_t b_lo = resident ? bres : a_lo + (uint32_t)G * a_step + lbo_fix;
-          for (int j = 0; j < nch; ++j) {
-            for (int kk = 0; kk < kk_n; ++kk) {
-              mma_i8_parts2(d_tmem, a_lo + 2u * kk, dhi, b_lo + b_kstep * kk, b_hi, idesc, accumulate);
-              accumulate = 1;
-            }
-            a_lo += a_step; b_lo += b_step;
-          }
-          c += nch;
-          bres += (uint32_t)nch * b_step;
+        const int nch = min(total_chunks - c, G);
+        const uint32_t a_lo = ring_lo + (uint32_t)stage * stage_step;
+        const uint32_t b_lo = resident ? bres : a_lo + (uint32_t)G * a_step + lbo_fix;
+        if (leader) {
+          const uint32_t first = it > 0 ? 1u : 0u;
+          if (kk_n == 4) issue_stage<4>(d_tmem, a_lo, a_step, dhi, b_lo, b_step, b_kstep, b_hi, idesc, nch, first);
+          else if (kk_n == 2) issue_stage<2>(d_tmem, a_lo, a_step, dhi, b_lo, b_step, b_kstep, b_hi, idesc, nch, first);
+          else issue_stage<1>(d_tmem, a_lo, a_step, dhi, b_lo, b_step, b_kstep, b_hi, idesc, nch, first);
           tc_commit_a(empty_a + 8u * (uint32_t)stage);   // frees the stage once these MMAs have read it
-          if (++stage == nst) { stage = 0; phase ^= 1u; }
+          if (it == kit - 1) tc_commit(&acc_full[buf]);  // accumulator of this tile complete
         }
-        if (ok) tc_commit(&acc_full[buf]);  // accumulator of this tile complete
+        c += nch;
+        bres += (uint32_t)nch * b_step;
+        if (++stage == nst) { stage = 0; phase ^= 1u; }
       }
     }
   } else {
@@ -658,6 +675,13 @@ __device__ __forceinline__ uint64_t mnmajor_desc(uint32_t saddr, int width_bytes
          (layout << 61);
 }
 
+__device__ __forceinline__ void tma_load_tile_2d_a(uint64_t map, uint32_t bar, uint32_t dst, int c0, int c1) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+      " [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
+      : "memory");
+}
 __device__ __forceinline__ void tma_load_tile_2d(const CUtensorMap* map, uint64_t* bar, void* dst, int c0, int c1) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
@@ -709,58 +733,94 @@ wgrad_mnmajor_kernel(const __grid_constant__ CUtensorMap mapG, const __grid_cons
   grid_dependency_wait();   // everything above overlapped the tail of the previous kernel
 
   if (warp == 0) {
-    if (lane == 0) {
+    // Copy-engine issue: the whole warp runs the loop, one elected lane issues a stage's loads from an
+    // unrolled block (a bulk-tensor copy takes its many operands from uniform registers, which the
+    // compiler fills cheaply only in warp-uniform code: issued from a loop under `lane == 0` a single
+    // load cost the issuing thread about 300 cycles, and the loads, not the MMAs, bound the kernel).
+    const bool leader = elect_one();
+    if (leader) {
       tma_prefetch_desc(&mapG);
       tma_prefetch_desc(&mapX);
-      for (int it = 0; it < k_iters; ++it) {
-        const int s = it % prm.stages;
-        if (it >= prm.stages && !mbar_wait(&empty_bar[s], ((it / prm.stages) - 1) & 1, &abort_flag, &g_device_status)) break;
-        const int pix0 = (chunk_begin + it) * prm.kp;
-        const int q0 = pix0 % prm.Q;
-        const int t = pix0 / prm.Q;
-        const int p0 = t % prm.P, img = t / prm.P;
-        const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
-        mbar_expect_tx(&full_bar[s], (uint32_t)(a_bytes + ntap * prm.nb * b_box_bytes));
-        uint8_t* sa = smem + (size_t)s * stage_bytes;
-        uint8_t* sb = sa + a_bytes;
-        tma_load_tile_2d(&mapG, &full_bar[s], sa, co0, pix0);
-        for (int tl = 0; tl < ntap; ++tl) {
-          const int tap = tap_begin + tl;
-          const int r = tap / prm.S, ss = tap - r * prm.S;
-          for (int b = 0; b < prm.nb; ++b)
-            tma_load_im2col_4d(&mapX, &full_bar[s], sb + (tl * prm.nb + b) * b_box_bytes, ci0 + b * prm.bw, cw, ch,
-                               img, (uint16_t)ss, (uint16_t)r);
+    }
+    const uint64_t pg = reinterpret_cast<uint64_t>(&mapG), px = reinterpret_cast<uint64_t>(&mapX);
+    const uint32_t ring_a = smem_u32(smem), full_a = smem_u32(&full_bar[0]);
+    const uint32_t tx_bytes = (uint32_t)(a_bytes + ntap * prm.nb * b_box_bytes);
+    int tap_r[8], tap_s[8];          // filter row and column of this CTA's taps (tg <= 8)
+#pragma unroll
+    for (int tl = 0; tl < 8; ++tl) {
+      const int tap = tap_begin + tl;
+      tap_r[tl] = tap / prm.S;
+      tap_s[tl] = tap - tap_r[tl] * prm.S;
+    }
+    int s = 0;
+    uint32_t phase = 0;
+    bool first_pass = true, ok = true;
+    for (int it = 0; it < k_iters; ++it) {
+      if (!first_pass) ok = mbar_wait(&empty_bar[s], phase ^ 1u, &abort_flag, &g_device_status) && ok;
+      const int pix0 = (chunk_begin + it) * prm.kp;
+      const int q0 = pix0 % prm.Q;
+      const int t = pix0 / prm.Q;
+      const int p0 = t % prm.P, img = t / prm.P;
+      const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
+      if (leader && ok) {
+        const uint32_t bar = full_a + 8u * (uint32_t)s;
+        const uint32_t sa = ring_a + (uint32_t)(s * stage_bytes);
+        const uint32_t sb = sa + (uint32_t)a_bytes;
+        mbar_expect_tx_a(bar, tx_bytes);
+        tma_load_tile_2d_a(pg, bar, sa, co0, pix0);
+#pragma unroll
+        for (int tl = 0; tl < 8; ++tl) {
+          if (tl < ntap) {
+            tma_load_im2col_4d_a(px, bar, sb + (uint32_t)(tl * prm.nb * b_box_bytes), ci0, cw, ch, img, (uint16_t)tap_s[tl],
+                                 (uint16_t)tap_r[tl]);
+            if (prm.nb > 1)
+              tma_load_im2col_4d_a(px, bar, sb + (uint32_t)((tl * prm.nb + 1) * b_box_bytes), ci0 + prm.bw, cw, ch, img,
+                                   (uint16_t)tap_s[tl], (uint16_t)tap_r[tl]);
+          }
         }
       }
+      if (++s == prm.stages) { s = 0; phase ^= 1u; first_pass = false; }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128.  The
-      // boxes of consecutive taps lie side by side in shared memory and in tensor memory, so one
-      // MMA covers as many of them as fit N <= 256: an instruction of 64 columns takes 73 cycles,
-      // one of 256 columns 128.
-      const int nbox = ntap * prm.nb;              // boxes of bw channels in this CTA's stage
-      const int per_mma = 256 / prm.bw;            // boxes per MMA
-      bool ok = true;
-      for (int it = 0; it < k_iters && ok; ++it) {
-        const int s = it % prm.stages;
-        ok = mbar_wait(&full_bar[s], (it / prm.stages) & 1, &abort_flag, &g_device_status);
-        if (!ok) break;
-        tc_fence_after();
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t sb = sa + a_bytes;
+    // A and B MN-major (bits 15, 16), int32 accumulate, signed 8-bit operands, M = 128.  The
+    // boxes of consecutive taps lie side by side in shared memory and in tensor memory, so one
+    // MMA covers as many of them as fit N <= 256.  The whole warp runs the loop; one elected lane
+    // issues a stage's instructions from an unrolled block (see issue_stage()).
+    const bool leader = elect_one();
+    const int nbox = ntap * prm.nb;              // boxes of bw channels in this CTA's stage
+    const int per_mma = 256 / prm.bw;            // boxes per MMA
+    const uint32_t idesc_full = idesc_i8_kmajor(per_mma * prm.bw) | (1u << 15) | (1u << 16);
+    const int tail = nbox % per_mma;             // boxes of the last, narrower MMA group (0: none)
+    const uint32_t idesc_tail = idesc_i8_kmajor((tail ? tail : per_mma) * prm.bw) | (1u << 15) | (1u << 16);
+    const int groups = (nbox + per_mma - 1) / per_mma;
+    const uint64_t a_kstep = (uint64_t)((32 * 128) >> 4), b_kstep = (uint64_t)((32 * prm.bw) >> 4);
+    int s = 0;
+    uint32_t phase = 0;
+    for (int it = 0; it < k_iters; ++it) {
+      mbar_wait(&full_bar[s], phase, &abort_flag, &g_device_status);
+      tc_fence_after();
+      const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+      const uint32_t sb = sa + a_bytes;
+      if (leader) {
         const uint64_t ad = mnmajor_desc(sa, 128, (uint32_t)a_bytes);
-        for (int b0 = 0; b0 < nbox; b0 += per_mma) {
-          const int cnt = min(per_mma, nbox - b0);
-          const uint32_t idesc = idesc_i8_kmajor(cnt * prm.bw) | (1u << 15) | (1u << 16);
-          const uint64_t bd = mnmajor_desc(sb + b0 * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
-          for (int kk = 0; kk < prm.kp / 32; ++kk)
-            mma_i8(tmem_base + (uint32_t)(b0 * prm.bw), ad + (uint64_t)((kk * 32 * 128) >> 4),
-                   bd + (uint64_t)((kk * 32 * prm.bw) >> 4), idesc, (it > 0 || kk > 0) ? 1u : 0u);
+        const uint32_t first = it > 0 ? 1u : 0u;
+#pragma unroll 1
+        for (int g = 0; g < groups; ++g) {
+          const uint32_t idesc = (g == groups - 1) ? idesc_tail : idesc_full;
+          const uint64_t bd = mnmajor_desc(sb + g * per_mma * b_box_bytes, prm.bw, (uint32_t)b_box_bytes);
+          const uint32_t d = tmem_base + (uint32_t)(g * per_mma * prm.bw);
+          if (prm.kp == 256) {
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) mma_i8(d, ad + a_kstep * kk, bd + b_kstep * kk, idesc, kk ? 1u : first);
+          } else {
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk) mma_i8(d, ad + a_kstep * kk, bd + b_kstep * kk, idesc, kk ? 1u : first);
+          }
         }
         tc_commit(&empty_bar[s]);
+        if (it == k_iters - 1) tc_commit(&acc_bar);
       }
-      if (ok) tc_commit(&acc_bar);
+      if (++s == prm.stages) { s = 0; phase ^= 1u; }
     }
   } else {
     const int quarter = warp & 3;
@@ -835,6 +895,7 @@ int plan_wgrad(const ConvShape& cs, WgradParams& prm, int* ngroups_out, int* co_
   const int T = cs.R * cs.S;
   const int b_tap_bytes = prm.nb * kKP * prm.bw;
   int tg_max = 512 / Nw;
+  if (tg_max > 8) tg_max = 8;          // the producer's unrolled issue block handles up to eight taps
   // Many pixels per slice: fat stages (several taps share the gradient tile, two stages in flight)
   // are fastest, the MMA phase dominates.  Few pixels (28x28 and below at batch 64): the partial
   // images dominate, and fewer taps per CTA mean fewer pixel slices, i.e. fewer partial images, and
