@@ -542,7 +542,10 @@ bool plan_halo(const HaloProblem& pb, dai8_dtype out_dtype, dai8_layout out_layo
     prm.a_stages = (budget - b_all - (store_ok ? prm.stage_bufs * staging1 : 0)) / a_stage;
   } else {
     // streamed weights: two activation stages, the rest of shared memory to the weight ring, stores
-    // straight from registers (the staging blocks would cost a weight piece or two)
+    // straight from registers (the staging blocks would cost a weight piece or two).  These layers are
+    // bound by the weight traffic from L2, which grows with every wasted position: measured, the
+    // wide patches of small images (28 x 28: 4 x 32) lose to the im2col form, 16 x 8 patches win.
+    if (prm.TX != 8) return false;
     prm.a_stages = 2;
     prm.b_stages = (budget - 2 * a_stage) / b_piece;
     if (prm.b_stages < 2) return false;

@@ -149,7 +149,12 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   grid_dependency_wait();   // everything above overlapped the tail of the previous kernel
 
   if (warp == 0) {
-    if (lane == 0) {
+    // Copy-engine issue.  The whole warp runs the loops (ring stage, tile position and filter tap are
+    // running counters: no divisions per load); one elected lane issues a stage's loads from an
+    // unrolled block, where the compiler can keep the many operands of a bulk-tensor copy in
+    // uniform registers.
+    const bool leader = elect_one();
+    if (leader) {
       tma_prefetch_desc(&mapA);
       tma_prefetch_desc(&mapB);
       if (prm.tma_store) tma_prefetch_desc(&mapC);
@@ -170,57 +175,67 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           }
         }
       }
-      // A single thread drives the copy engine, so this loop is a latency chain: no integer
-      // divisions (ring stage, tile position and filter tap are running counters) and only 32-bit
-      // shared-memory addresses computed up front.
-      const uint64_t pa = reinterpret_cast<uint64_t>(&mapA), pb = reinterpret_cast<uint64_t>(&mapB);
-      const uint32_t ring_a = smem_u32(ring), full_a = smem_u32(&full_bar[0]);
-      const int G = prm.G, S = prm.S, cpt = prm.chunks_per_tap, kc = prm.kc_bytes, nst = prm.stages, kit = prm.k_iters;
-      const bool resident = prm.b_resident != 0, b_mn = prm.b_mn != 0;
-      int stage = 0;
-      uint32_t phase = 0;            // parity of the current pass over the ring
-      bool first_pass = true;        // nothing to wait for until the ring has wrapped once
-      bool ok = true;
-      int t = blockIdx.x;
-      int m_tile = t / prm.n_tiles, n_tile = t - m_tile * prm.n_tiles;
-      const int dm = gridDim.x / prm.n_tiles, dn = gridDim.x - dm * prm.n_tiles;   // tile step of this CTA
-      for (; t < num_tiles && ok; t += gridDim.x) {
-        const int n0 = n_tile * prm.BN;
-        // the last tile is shifted back so that every tile covers 128 existing pixels
-        int m0 = m_tile * kBM;
-        if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
-        const int tq = m0 / prm.Q;               // one division pair per tile (not per load)
-        const int q0 = m0 - tq * prm.Q;
-        const int img = tq / prm.P, p0 = tq - img * prm.P;
-        const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
-        int c = 0, k0 = 0, kchunk = 0, r = 0, ss = 0;    // chunk, its channel offset, tap row and column
-        for (int it = 0; it < kit; ++it) {
-          if (!first_pass && !mbar_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, &g_device_status)) { ok = false; break; }
-          const int nch = min(total_chunks - c, G);
-          const uint32_t bar = full_a + 8u * (uint32_t)stage;
-          mbar_expect_tx_a(bar, (uint32_t)(nch * chunk_pair_bytes));
-          uint32_t sa = ring_a + (uint32_t)(stage * stage_bytes);
-          uint32_t sb = sa + (uint32_t)(G * a_chunk_bytes);
-          for (int j = 0; j < nch; ++j, ++c) {
-            tma_load_im2col_4d_a(pa, bar, sa, k0, cw, ch, img, (uint16_t)ss, (uint16_t)r);
-            if (!resident) {
-              if (b_mn) {
-                const int ftap = prm.b_tap_base - r * prm.b_tap_dr - ss * prm.b_tap_ds;
-                for (int b = 0; b < prm.b_nb; ++b)
-                  tma_load_tile_3d_a(pb, bar, sb + (uint32_t)(b * kc * prm.b_bw), n0 + b * prm.b_bw, ftap, k0);
-              } else {
-                tma_load_tile_3d_a(pb, bar, sb, k0, r * S + ss, n0);
-              }
-            }
-            sa += (uint32_t)a_chunk_bytes; sb += (uint32_t)b_chunk_bytes;
+    }
+    const uint64_t pa = reinterpret_cast<uint64_t>(&mapA), pb = reinterpret_cast<uint64_t>(&mapB);
+    const uint32_t ring_a = smem_u32(ring), full_a = smem_u32(&full_bar[0]);
+    const int G = prm.G, S = prm.S, cpt = prm.chunks_per_tap, kc = prm.kc_bytes, nst = prm.stages, kit = prm.k_iters;
+    const bool resident = prm.b_resident != 0, b_mn = prm.b_mn != 0;
+    int stage = 0;
+    uint32_t phase = 0;            // parity of the current pass over the ring
+    bool first_pass = true;        // nothing to wait for until the ring has wrapped once
+    bool ok = true;
+    int m_tile = blockIdx.x / prm.n_tiles, n_tile = blockIdx.x - m_tile * prm.n_tiles;
+    const int dm = gridDim.x / prm.n_tiles, dn = gridDim.x - dm * prm.n_tiles;   // tile step of this CTA
+    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x) {
+      const int n0 = n_tile * prm.BN;
+      // the last tile is shifted back so that every tile covers 128 existing pixels
+      int m0 = m_tile * kBM;
+      if (m0 + kBM > prm.Mtot) m0 = prm.Mtot - kBM;
+      const int tq = m0 / prm.Q;               // one division pair per tile (not per load)
+      const int q0 = m0 - tq * prm.Q;
+      const int img = tq / prm.P, p0 = tq - img * prm.P;
+      const int cw = prm.lower_w + q0 * prm.sw, ch = prm.lower_h + p0 * prm.sh;
+      int c = 0, k0 = 0, kchunk = 0, r = 0, ss = 0;    // chunk, its channel offset, tap row and column
+      for (int it = 0; it < kit; ++it) {
+        if (!first_pass) ok = mbar_wait(&empty_bar[stage], phase ^ 1u, &abort_flag, &g_device_status) && ok;
+        const int nch = min(total_chunks - c, G);
+        // channel offset and tap of the (up to four) chunks of this stage
+        int ck0[4], cr[4], cs[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          ck0[j] = k0; cr[j] = r; cs[j] = ss;
+          if (j < nch) {
             k0 += kc;
             if (++kchunk == cpt) { kchunk = 0; k0 = 0; if (++ss == S) { ss = 0; ++r; } }
           }
-          if (++stage == nst) { stage = 0; phase ^= 1u; first_pass = false; }
         }
-        m_tile += dm; n_tile += dn;
-        if (n_tile >= prm.n_tiles) { n_tile -= prm.n_tiles; ++m_tile; }
+        if (leader && ok) {
+          const uint32_t bar = full_a + 8u * (uint32_t)stage;
+          mbar_expect_tx_a(bar, (uint32_t)(nch * chunk_pair_bytes));
+          const uint32_t sa = ring_a + (uint32_t)(stage * stage_bytes);
+          const uint32_t sb = sa + (uint32_t)(G * a_chunk_bytes);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            if (j < nch) {
+              tma_load_im2col_4d_a(pa, bar, sa + (uint32_t)(j * a_chunk_bytes), ck0[j], cw, ch, img, (uint16_t)cs[j], (uint16_t)cr[j]);
+              if (!resident) {
+                const uint32_t dst = sb + (uint32_t)(j * b_chunk_bytes);
+                if (b_mn) {
+                  const int ftap = prm.b_tap_base - cr[j] * prm.b_tap_dr - cs[j] * prm.b_tap_ds;
+                  for (int b = 0; b < prm.b_nb; ++b)
+                    tma_load_tile_3d_a(pb, bar, dst + (uint32_t)(b * kc * prm.b_bw), n0 + b * prm.b_bw, ftap, ck0[j]);
+                } else {
+                  tma_load_tile_3d_a(pb, bar, dst, ck0[j], cr[j] * S + cs[j], n0);
+                }
+              }
+            }
+          }
+        }
+        c += nch;
+        if (++stage == nst) { stage = 0; phase ^= 1u; first_pass = false; }
       }
+      m_tile += dm; n_tile += dn;
+      if (n_tile >= prm.n_tiles) { n_tile -= prm.n_tiles; ++m_tile; }
     }
   } else if (warp == 1) {
     // MMA issue.  The whole warp runs the loops (trip counts depend only on the launch parameters; a

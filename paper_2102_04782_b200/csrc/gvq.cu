@@ -522,6 +522,46 @@ quantize_nchw_kernel(const T* __restrict__ x, int C, int Cp, int64_t HW,
   }
 }
 
+// NCHW input with few positions per (n, c) row -- weights, (Cout, Cin, R, S) with H*W = R*S -- to
+// [N][H*W][Cp] codes: the tile transpose above would leave most of its 128-position tiles empty.
+// A block takes whole images n: their C*HW values are contiguous, are read coalesced, quantized
+// into a [HW][Cp] image in shared memory and written out as 16-byte vectors.
+template <typename T, bool STOCH>
+__global__ void __launch_bounds__(kThreads)
+quantize_nchw_rows_kernel(const T* __restrict__ x, int N, int C, int Cp, int HW, const float* __restrict__ scale,
+                          uint32_t seed, int8_t* __restrict__ q) {
+  extern __shared__ __align__(16) int8_t rows_sm[];      // [HW][Cp]
+  grid_dependency_release();
+  grid_dependency_wait();
+  const int tid = threadIdx.x;
+  const int per_n = C * HW, codes = HW * Cp;
+  const float inv = inv_scale(*scale);
+  const uint32_t key0 = sr_key(seed, 0u);
+  for (int i = tid; i < codes / 4; i += kThreads) reinterpret_cast<uint32_t*>(rows_sm)[i] = 0u;   // padding channels stay 0
+  __syncthreads();
+  for (int n = blockIdx.x; n < N; n += gridDim.x) {
+    const T* src = x + (size_t)n * per_n;
+    for (int i = tid; i < per_n; i += kThreads) {
+      const int c = i / HW, hw = i - c * HW;
+      const float v = to_f32(src[i]);
+      int code;
+      if (STOCH) {
+        const uint64_t idx = (uint64_t)n * per_n + (uint64_t)i;       // the NCHW index
+        const uint32_t hi = (uint32_t)(idx >> 32);
+        const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
+        code = quant_stochastic(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key)));
+      } else {
+        code = quant_nearest(v, inv);
+      }
+      rows_sm[hw * Cp + c] = (int8_t)code;
+    }
+    __syncthreads();
+    uint4* dst = reinterpret_cast<uint4*>(q + (size_t)n * codes);
+    for (int i = tid; i < codes / 16; i += kThreads) dst[i] = reinterpret_cast<const uint4*>(rows_sm)[i];
+    __syncthreads();
+  }
+}
+
 // max|x| over a whole tensor (layout-free), into the bit pattern at out_bits (zeroed before).
 template <typename T, int VE>
 __global__ void __launch_bounds__(kThreads)
@@ -1683,8 +1723,9 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
 // activations (Eq. 1, Fig. 2).  The scale needs the whole tensor before the first code can be
 // written, so the tensor is swept twice; this kernel makes the second sweep as cheap as the chip
 // allows.  A persistent cooperative launch, one CTA per SM, each owning a contiguous range of the
-// tensor.  A producer warp streams the range through a ring of 16 KB shared-memory pieces with bulk
-// asynchronous copies; sweep 1 takes max|x| (packed bf16 arithmetic, exact).  After one atomic max
+// tensor.  A producer warp streams the range through a ring of 13 KB shared-memory pieces with bulk
+// asynchronous copies, one ring slot per consumer warp; sweep 1 takes max|x| (packed bf16
+// arithmetic, exact).  After one atomic max
 // per CTA and one grid barrier, sweep 2 writes the codes walking the range BACKWARDS: first the
 // pieces that are still in shared memory from sweep 1 (no memory traffic at all), then the rest in
 // reverse order, so that what it fetches is what sweep 1 touched last and L2 still holds.
@@ -1693,9 +1734,9 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
 // which rounds to 127 like the clamped value does.  Codes come out of the magic-number addition
 // (quant_nearest_bits without the clamps).
 // ------------------------------------------------------------------------------------------------
-constexpr int kQtPieceBytes = 16384;
+constexpr int kQtMaxSlots = 16;                // one shared-memory piece per consumer warp
+constexpr int kQtPieceBytes = 13312;           // 16 pieces fill the shared memory of an SM
 constexpr int kQtPieceVecs = kQtPieceBytes / 16;
-constexpr int kQtMaxSlots = 13;
 
 struct QtArgs {
   const uint8_t* x;      // the tensor as bytes
@@ -1712,11 +1753,12 @@ template <typename T>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 quantize_flat_fused_kernel(const QtArgs a) {
   constexpr int VE = 16 / (int)sizeof(T);
+  constexpr int NW = kFT / 32;                 // consumer warps
   extern __shared__ __align__(128) uint8_t qsmem[];
   __shared__ uint64_t full_bar[kQtMaxSlots], empty_bar[kQtMaxSlots];
   __shared__ volatile uint32_t s_abort;
   __shared__ uint32_t s_ok;
-  __shared__ float s_wmax[kFT / 32];
+  __shared__ float s_wmax[NW];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int64_t v0 = (int64_t)blockIdx.x * a.vec_per_cta;
   const int64_t v1 = min(a.nvec, v0 + a.vec_per_cta);
@@ -1725,19 +1767,22 @@ quantize_flat_fused_kernel(const QtArgs a) {
   const int S = a.slots;
   // Piece u of sweep 1 goes to slot u mod S; afterwards the last min(K, S) pieces are resident.  Step v
   // of sweep 2 handles piece K-1-v in the slot of step v - S (the same slot for v < S: resident).
+  // Slot w belongs to consumer warp w, which takes every fill of it in turn: a warp meets the producer
+  // once per 13 KB, and it can never run a whole fill ahead of its slot's barrier (a parity wait
+  // cannot tell the phase before last from the one awaited).
   auto slot2 = [&](int v) { int r = (K - 1 - (v % S)) % S; return r < 0 ? r + S : r; };
   auto fills1 = [&](int slot) { return slot < K ? (K - slot + S - 1) / S : 0; };   // sweep-1 fills of a slot
 
   if (tid == 0) {
     s_abort = 0u;
 #pragma unroll 1
-    for (int s = 0; s < kQtMaxSlots; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], kFT / 32); }
+    for (int s = 0; s < kQtMaxSlots; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
 
-  if (warp == kFT / 32) {
-    // ---- producer: every fill of a slot but its first waits for the consumers' hand-back of the fill before
+  if (warp == NW) {
+    // ---- producer: every fill of a slot but its first waits for the consumer's hand-back of the fill before
     if (lane == 0 && K > 0) {
       const uint8_t* src = a.x + (size_t)v0 * 16;
       const int total = K + (K > S ? K - S : 0);
@@ -1760,14 +1805,14 @@ quantize_flat_fused_kernel(const QtArgs a) {
   float m = 0.f;
   uint32_t m2[4] = {0u, 0u, 0u, 0u};
 #pragma unroll 1
-  for (int u = 0; u < K && ok; ++u) {
-    const int slot = u % S;
+  for (int u = warp; u < K && ok && warp < S; u += S) {
+    const int slot = warp;
     ok = mbar_wait(&full_bar[slot], (uint32_t)(u / S) & 1u, &s_abort, a.status);
     if (!ok) break;
     const uint4* pv = reinterpret_cast<const uint4*>(qsmem + (size_t)slot * kQtPieceBytes);
     const int cnt = min(kQtPieceVecs, nv - u * kQtPieceVecs);
-#pragma unroll 2
-    for (int i = tid; i < cnt; i += kFT) {
+#pragma unroll 4
+    for (int i = lane; i < cnt; i += 32) {
       const uint4 r = pv[i];
       if constexpr (VE == 8) {
         m2[0] = bf16x2_max(m2[0], r.x & 0x7FFF7FFFu); m2[1] = bf16x2_max(m2[1], r.y & 0x7FFF7FFFu);
@@ -1793,7 +1838,7 @@ quantize_flat_fused_kernel(const QtArgs a) {
   consumer_sync();
   if (tid == 0) {
 #pragma unroll 1
-    for (int w = 1; w < kFT / 32; ++w) m = fmaxf(m, s_wmax[w]);
+    for (int w = 1; w < NW; ++w) m = fmaxf(m, s_wmax[w]);
     if (m > 0.f) atomicMax(a.ctrl + 1, __float_as_uint(m));   // non-negative floats order like their bit patterns
   }
   ok = grid_barrier(a.ctrl, gridDim.x, a.status, &s_abort, &s_ok) && ok;
@@ -1804,16 +1849,18 @@ quantize_flat_fused_kernel(const QtArgs a) {
     if (blockIdx.x == 0 && tid == 0) *a.scale = s;
     const float inv = inv_scale(s);
     int8_t* qbase = a.q + (size_t)v0 * VE;
+    int v_first = (K - 1 - warp) % S;        // the first step of sweep 2 that uses this warp's slot
+    if (v_first < 0) v_first += S;
 #pragma unroll 1
-    for (int v = 0; v < K && ok; ++v) {
-      const int piece = K - 1 - v, slot = slot2(v);
+    for (int v = v_first; v < K && ok && warp < S; v += S) {
+      const int piece = K - 1 - v, slot = warp;
       ok = mbar_wait(&full_bar[slot], (uint32_t)(fills1(slot) - 1 + v / S) & 1u, &s_abort, a.status);
       if (!ok) break;
       const uint4* pv = reinterpret_cast<const uint4*>(qsmem + (size_t)slot * kQtPieceBytes);
       const int cnt = min(kQtPieceVecs, nv - piece * kQtPieceVecs);
       int8_t* qp = qbase + (size_t)piece * kQtPieceVecs * VE;
 #pragma unroll 2
-      for (int i = tid; i < cnt; i += kFT) {
+      for (int i = lane; i < cnt; i += 32) {
         const uint4 r = pv[i];
         if constexpr (VE == 8) {
           const uint32_t w[4] = {r.x, r.y, r.z, r.w};
@@ -2223,6 +2270,15 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
       else
         quantize_nhwc_kernel<T, 1, false, false, false><<<g.grid, kThreads, 0, st>>>(x, npix, HW, C, Cp, g.G, scale, nullptr, seed, q, nullptr);
     }
+  } else if (HW <= 32 && HW * Cp <= 40 * 1024) {
+    // weights: few positions per row
+    int blocks = N < 4 * fused_config().sms ? N : 4 * fused_config().sms;
+    if (blocks < 1) blocks = 1;
+    const size_t smem = (size_t)HW * Cp;
+    if (stoch)
+      DAI8_RETURN_IF_CUDA(launch_dependent(quantize_nchw_rows_kernel<T, true>, dim3((unsigned)blocks), dim3(kThreads), smem, st, x, N, C, Cp, (int)HW, (const float*)scale, seed, q));
+    else
+      DAI8_RETURN_IF_CUDA(launch_dependent(quantize_nchw_rows_kernel<T, false>, dim3((unsigned)blocks), dim3(kThreads), smem, st, x, N, C, Cp, (int)HW, (const float*)scale, seed, q));
   } else {
     const dim3 qgrid((unsigned)ceil_div64(HW, kTileHW), (unsigned)((Cp + kTileC - 1) / kTileC), (unsigned)N);
     if (stoch)

@@ -191,6 +191,8 @@ LARGE_TENSORS = [
     ((8, 3, 100, 100), api.NHWC),       # stem-like
     ((4, 40, 37, 41), api.NCHW),        # NCHW activation, ragged position tiles
     ((512, 512, 3, 3), api.NCHW),       # VGG weights: rows of 9 elements
+    ((256, 130, 3, 3), api.NCHW),       # weights with padded code channels
+    ((1024, 256, 1, 1), api.NCHW),      # pointwise weights
     ((2, 130, 31, 33), api.NCHW),       # channel tiles with a ragged tail
 ]
 
