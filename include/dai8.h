@@ -98,11 +98,11 @@ int dai8_padded_channels(int C);
  *              mode draws u from a counter-based hash of (seed, stream 0, NCHW index)
  *   q          out, int8 [N][H][W][Cp]; padding channels are written with 0
  *   ws         scratch of dai8_quantize_tensor_workspace_bytes() bytes, or NULL.  With scratch, a
- *              tensor whose codes have the layout of its values (NHWC, C a multiple of 16) gets its
- *              scale and its codes from ONE launch that keeps as much of the tensor as fits in
- *              shared memory between the two sweeps; without it (ws == NULL) the scale and the
- *              codes take two launches.  The results are identical.  A non-NULL ws that is too
- *              small returns DAI8_ERR_WORKSPACE.
+ *              tensor whose codes have the layout of its values (NHWC, C a multiple of 16) and
+ *              which fits into the shared memory of the whole GPU (about 30 MB) gets its scale and
+ *              its codes from ONE launch that reads it from DRAM once; larger tensors, other
+ *              layouts and ws == NULL take two launches (scale, then codes).  The results are
+ *              identical.  A non-NULL ws that is too small returns DAI8_ERR_WORKSPACE.
  * q(x) = round(clamp(x*(127/s), -127, 127)); s <= 0 gives all-zero codes.
  * -------------------------------------------------------------------------------------------- */
 size_t dai8_quantize_tensor_workspace_bytes(void);

@@ -2223,7 +2223,10 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
   if (ws && mode == DAI8_SCALE_ABSMAX && round == DAI8_ROUND_NEAREST_EVEN && layout == DAI8_NHWC && C == Cp &&
-      npix * Cp > kSmallTensorElems && fused_config().coop && ceil_div64(total / VEfull, fused_config().sms) < ((int64_t)1 << 30) &&
+      npix * Cp > kSmallTensorElems && fused_config().coop &&
+      // measured: the one-launch kernel wins only while the whole tensor stays in shared memory between
+      // its sweeps (one read from DRAM instead of two); beyond that the two plain kernels stream faster
+      total / VEfull <= (int64_t)fused_config().sms * kQtMaxSlots * kQtPieceVecs &&
       fused_config().smem_max >= (size_t)kQtMaxSlots * kQtPieceBytes + 2048)
     return launch_quantize_flat_fused<T>(x, total / VEfull, scale, q, ws, st);
   if (npix * Cp <= kSmallTensorElems) {
