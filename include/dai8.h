@@ -68,13 +68,24 @@ typedef struct {
   int N, Cin, Cout, H, W, R, S, stride_h, stride_w, pad_h, pad_w;
 } dai8_conv_geom;
 
+/* Which quantization strategy dai8_quantize_grad applies to the per-channel codes `vq` (the rows of
+ * the ablation study, Sec. 4.1; the layer-wide codes `gq` always use |g|max of the layer):
+ *   FULL       the method: per-channel statistics, discriminator (Eq. 15), clip rule (Eq. 11 / 14)
+ *   GQ         global quantization, the ablation baseline: one scale |g|max of the layer for every channel
+ *   GVQ_MAX    "Ours_GVQ": per-channel |g|max, no discriminator, no clipping
+ *   LAYER_MCS  "Ours_MCS": Eq. 15 and Eq. 14 on the statistics of the whole layer, one clip value for
+ *              every channel (s_state[c] all equal; s_state[0] is the state that is read back) */
+typedef enum { DAI8_GRAD_FULL = 0, DAI8_GRAD_GQ = 1, DAI8_GRAD_GVQ_MAX = 2, DAI8_GRAD_LAYER_MCS = 3 } dai8_grad_mode;
+
 /* Hyper-parameters of the Magnitude-aware Clipping Strategy.  Paper values: lambda = 0.3
  * (Eq. 15), k = 1, A = 0.8 (Sec. 4.1).  sigma is the population standard deviation about the
- * channel mean unless std_unbiased (divide by M-1) or center_mean = 0 (root mean square). */
+ * channel mean unless std_unbiased (divide by M-1) or center_mean = 0 (root mean square).
+ * mode: a dai8_grad_mode, DAI8_GRAD_FULL by default. */
 typedef struct {
   float lambda, k, A;
   int std_unbiased;
   int center_mean;
+  int mode;
 } dai8_mcs_params;
 
 /* Rows of the `stats` output of dai8_quantize_grad: stats[c*4 + i]. */
@@ -121,7 +132,8 @@ dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai8_layout la
  *   s_state    device [C]: in  s_{c,t-1} (read only if has_prev != 0; otherwise s_{c,t-1} is
  *              taken as |g|max,c), out s_{c,t} -- the per-channel clip values used for `vq`
  *   gmax_layer device [1], out: |g|max of the layer, the scale of `gq`
- *   stats      device [C][4] or NULL, out: |g|max,c, mean, sigma, P = #{|g|>sigma}/M
+ *   stats      device [C][4] or NULL, out: |g|max,c, mean, sigma, P = #{|g|>sigma}/M (per channel; in
+ *              mode LAYER_MCS mean, sigma and P of every row are those of the whole layer)
  *   cls        device [C] or NULL, out: 1 = bell-shaped (P > lambda), 0 = Inverted-T.  When has_prev
  *              != 0 its previous contents are read as a hint (the classes of the last iteration):
  *              the fused kernel writes the codes while it counts, with the clip value of the hinted
@@ -219,6 +231,16 @@ uint64_t dai8_launch_count(void);
 /* Reads and clears the device status word (DAI8_OK or DAI8_ERR_TIMEOUT).  Synchronises `stream`.
  * host_status: host pointer. */
 dai8_status dai8_get_device_status(int* host_status, void* stream);
+
+/* Self-test of the give-up path of the bounded device-side waits.  Runs the library's own wait
+ * helpers (the mbarrier wait and the grid barrier of the gradient quantizer, the mbarrier wait of the
+ * convolution kernels) on barriers that nobody completes, with nothing in flight and a limit of
+ * `limit_cycles` SM cycles (1 .. 1e8) instead of the usual second.  Every wait must return by
+ * itself: report[0..2] (host, 3 ints) get 1 for each wait that gave up, and the device status word
+ * then holds DAI8_ERR_TIMEOUT until dai8_get_device_status reads and clears it.  The kernels end
+ * normally, so the context stays usable.  ws: 32 bytes of device scratch.  Synchronises `stream`. */
+dai8_status dai8_debug_expire_waits(uint64_t limit_cycles, int* report /* host */, void* ws,
+                                    size_t ws_bytes, void* stream);
 
 #ifdef __cplusplus
 }

@@ -93,6 +93,35 @@ def classify_clip(cnt, absmax, M: int, s_prev=None, lam: float = 0.3, k: float =
     return state, cls
 
 
+def grad_scales(g, mode: str = "full", s_prev=None, lam: float = 0.3, k: float = 1.0, A: float = 0.8):
+    """Clip values s[C] and classes cls[C] of the per-channel codes under one of the quantization
+    strategies of the ablation study (Sec. 4.1), composed from the steps above:
+      "full"       Algorithm 1: per-channel sigma, density, discriminator (Eq. 15), clip rule (Eq. 11 / 14)
+      "gq"         global quantization: |g|max of the layer for every channel, no clipping
+      "gvq_max"    per-channel |g|max, no discriminator, no clipping
+      "layer_mcs"  Eq. 15 and Eq. 14 on the statistics of the whole layer (the layer as ONE channel of
+                   N*C*H*W elements), one clip value for every channel; s_prev: its previous value
+    Returns (s[C] fp32, cls[C] uint8, |g|max of the layer)."""
+    g = _f32(g)
+    N, C, H, W = g.shape
+    absmax, _, sigma, gl = channel_stats(g)
+    if mode == "full":
+        s, cls = classify_clip(density_count(g, sigma), absmax, N * H * W, s_prev=s_prev, lam=lam, k=k, A=A)
+    elif mode == "gq":
+        s, cls = np.full(C, gl, np.float32), np.ones(C, np.uint8)
+    elif mode == "gvq_max":
+        s, cls = absmax.copy(), np.ones(C, np.uint8)
+    elif mode == "layer_mcs":
+        one = g.reshape(1, 1, N * C * H, W)
+        am1, _, sg1, _ = channel_stats(one)
+        prev = None if s_prev is None else np.atleast_1d(_f32(s_prev))[:1]
+        s1, c1 = classify_clip(density_count(one, sg1), am1, N * C * H * W, s_prev=prev, lam=lam, k=k, A=A)
+        s, cls = np.full(C, s1[0], np.float32), np.full(C, c1[0], np.uint8)
+    else:
+        raise ValueError(mode)
+    return s, cls, gl
+
+
 def rand_uniform(seed: int, stream: int, index: int) -> float:
     return float(lib().dai8o_rand_uniform(seed & 0xFFFFFFFF, stream, index))
 

@@ -19,6 +19,7 @@ NCHW, NHWC = 0, 1
 ROUND_NEAREST_EVEN, ROUND_STOCHASTIC = 0, 1
 SCALE_ABSMAX, SCALE_GIVEN = 0, 1
 OP_FWD, OP_BWD_DATA, OP_BWD_FILTER = 0, 1, 2
+GRAD_FULL, GRAD_GQ, GRAD_GVQ_MAX, GRAD_LAYER_MCS = 0, 1, 2, 3
 
 EXPORTS = [
     "dai8_status_string", "dai8_mcs_defaults", "dai8_padded_channels", "dai8_quantize_tensor",
@@ -26,7 +27,7 @@ EXPORTS = [
     "dai8_quantize_grad_workspace_bytes", "dai8_quantize_grad", "dai8_quantize_grad_noalloc",
     "dai8_conv_workspace_bytes",
     "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
-    "dai8_launch_count", "dai8_get_device_status",
+    "dai8_launch_count", "dai8_get_device_status", "dai8_debug_expire_waits",
 ]
 
 
@@ -45,7 +46,7 @@ class ConvGeom(ctypes.Structure):
 
 class McsParams(ctypes.Structure):
     _fields_ = [("lam", ctypes.c_float), ("k", ctypes.c_float), ("A", ctypes.c_float),
-                ("std_unbiased", c_int), ("center_mean", c_int)]
+                ("std_unbiased", c_int), ("center_mean", c_int), ("mode", c_int)]
 
 
 class Dai8Error(RuntimeError):
@@ -95,6 +96,7 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(ConvGeom), c_void_p, c_int, c_void_p,
                                            c_size_t, c_void_p]
         l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
+        l.dai8_debug_expire_waits.argtypes = [c_uint64, ctypes.POINTER(c_int), c_void_p, c_size_t, c_void_p]
         _lib = l
     return _lib
 
@@ -154,6 +156,15 @@ def get_device_status() -> int:
     v = c_int(0)
     _check(lib().dai8_get_device_status(ctypes.byref(v), _stream()), "dai8_get_device_status")
     return v.value
+
+
+def debug_expire_waits(limit_cycles: int, ws: torch.Tensor):
+    """dai8_debug_expire_waits: runs the bounded-wait helpers on barriers nobody completes; returns the
+    three flags (1 = the wait gave up by itself)."""
+    rep = (c_int * 3)()
+    p, n = _ws_args(ws)
+    _check(lib().dai8_debug_expire_waits(limit_cycles, rep, p, n, _stream()), "dai8_debug_expire_waits")
+    return list(rep)
 
 
 def quantize_tensor_workspace_bytes() -> int:

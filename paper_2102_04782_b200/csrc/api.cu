@@ -44,6 +44,7 @@ extern "C" void dai8_mcs_defaults(dai8_mcs_params* p) {
   p->A = 0.8f;       // Sec. 4.1
   p->std_unbiased = 0;
   p->center_mean = 1;
+  p->mode = DAI8_GRAD_FULL;
 }
 
 extern "C" int dai8_padded_channels(int C) { return C > 0 ? dai8::round_up(C, 16) : 0; }
@@ -55,4 +56,21 @@ extern "C" uint64_t dai8_launch_count(void) {
 extern "C" dai8_status dai8_get_device_status(int* host_status, void* stream) {
   if (!host_status) return DAI8_ERR_INVALID_ARG;
   return dai8::read_clear_device_status(host_status, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" dai8_status dai8_debug_expire_waits(uint64_t limit_cycles, int* report, void* ws, size_t ws_bytes,
+                                               void* stream) {
+  if (!report || !ws || ws_bytes < 32 || !dai8::aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (limit_cycles == 0 || limit_cycles > 100000000ull) return DAI8_ERR_INVALID_ARG;   // at most ~50 ms
+  dai8_status a = dai8::check_device_arch();
+  if (a != DAI8_OK) return a;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int* rep = reinterpret_cast<int*>(static_cast<char*>(ws) + 16);
+  if (cudaMemsetAsync(rep, 0, 12, st) != cudaSuccess) return DAI8_ERR_CUDA;
+  a = dai8::expire_gvq_waits((long long)limit_cycles, ws, rep, st);
+  if (a == DAI8_OK) a = dai8::expire_conv_wait((long long)limit_cycles, rep, st);
+  if (a != DAI8_OK) return a;
+  if (cudaMemcpyAsync(report, rep, 12, cudaMemcpyDeviceToHost, st) != cudaSuccess) return DAI8_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return DAI8_ERR_CUDA;
+  return DAI8_OK;
 }

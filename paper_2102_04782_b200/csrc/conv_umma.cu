@@ -52,6 +52,21 @@ namespace {
 
 using namespace umma;
 
+// Self-test of the bounded wait of the convolution kernels: an mbarrier nobody arrives on, waited for
+// with a limit of a few thousand cycles and nothing in flight (see dai8_debug_expire_waits).
+__global__ void expire_conv_wait_kernel(long long limit, int* report) {
+  __shared__ uint64_t bar;
+  __shared__ volatile uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    abort_flag = 0u;
+    mbar_init(&bar, 1);
+    fence_mbar_init();
+  }
+  __syncthreads();
+  const bool ok = mbar_wait(&bar, 0u, &abort_flag, &g_device_status, limit);
+  if (threadIdx.x == 0) report[2] = ok ? 0 : 1;
+}
+
 constexpr int kThreadsIgemm = 192;      // weight-gradient kernel: TMA warp, MMA warp, 4 epilogue warps
 constexpr int kEpiWarps = 8;             // persistent kernel: two epilogue warps per tensor-memory lane quarter
 constexpr int kThreadsPersist = 64 + 32 * kEpiWarps;
@@ -993,6 +1008,13 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
 }
 
 }  // namespace
+
+dai8_status expire_conv_wait(long long limit, int* report_dev, cudaStream_t st) {
+  expire_conv_wait_kernel<<<1, 64, 0, st>>>(limit, report_dev);
+  note_launch(1);
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
 
 void set_halo_disabled(int disabled) { g_halo_disabled.store(disabled ? 1 : 0, std::memory_order_relaxed); }
 

@@ -23,6 +23,12 @@ dai8_status read_clear_device_status(int* host_status, cudaStream_t stream);
 // Device address of that status word on the current device (nullptr on failure).
 unsigned int* device_status_address();
 
+// Self-tests of the bounded device-side waits (gvq.cu, conv_umma.cu): each runs the file's own wait
+// helpers on barriers nobody completes, with `limit` cycles; report_dev[0..2] get 1 where the wait
+// gave up as it must.  ws: 16 bytes of scratch.
+dai8_status expire_gvq_waits(long long limit, void* ws, int* report_dev, cudaStream_t st);
+dai8_status expire_conv_wait(long long limit, int* report_dev, cudaStream_t st);
+
 // Programmatic dependent launch.  A kernel launched with launch_dependent() may start while the
 // kernel before it on the stream is still running: its CTAs take the SM resources that become free
 // and run their set-up (barrier initialisation, tensor-memory allocation, descriptor prefetch), then

@@ -1,14 +1,22 @@
 // Gradient Vectorized Quantization with the Magnitude-aware Clipping Strategy (Algorithm 1 up to
 // the two quantizations) and the layer-wide quantizer of the forward pass (Eq. 1), as HBM-bound kernels.
 //
-// Three sweeps over dY, because each needs a per-channel scalar the previous one produces:
-//   1. stats   : |g|max,c, sum, sum of squares  -> mean, sigma          (Algorithm 1)
-//   2. count   : #{|g| > sigma_c}                -> class, clip s_c      (Algorithm 1, Eq. 14/15)
-//   3. quantize: vq (per-channel s_c) and gq (layer |g|max) in one pass (Algorithm 1)
-// The last block of sweeps 1 and 2 (found with a ticket counter) finishes the per-channel
-// scalars, so no separate tiny launches are needed.  Floating-point sums are combined in a
-// fixed order (per-block partials, then a fixed tree), so results do not depend on scheduling;
-// max and the density count use integer atomics, which are order-independent.
+// Each step of Algorithm 1 needs a per-channel scalar the previous one produces: |g|max,c and sigma_c
+// (statistics), then #{|g| > sigma_c} (density), then the class and the clip value s_c (Eq. 14/15), then
+// the codes.  The kernels that run, by input:
+//   * NHWC, C a multiple of the 16-byte vector (the layout of the benchmarks): ONE persistent
+//     cooperative launch.  gvq_fused_nhwc_kernel partitions the pixels over the SMs, keeps as much of
+//     a CTA's range as fits resident in shared memory (bulk asynchronous copies on an mbarrier ring)
+//     and makes two sweeps: statistics, then density count fused with both code tensors, written with
+//     the clip value of a PREDICTED class; channels whose count contradicts the prediction are redone.
+//     gvq_columns_kernel serves many channels x few pixels: a CTA owns whole channel vectors, so
+//     everything but the layer-wide |g|max is CTA-local.
+//   * anything else (NCHW, ragged C, no cooperative launch): three launches -- stats_*, count_*,
+//     quantize_* -- whose last block (ticket counter) finishes the per-channel scalars.
+// Floating-point sums are combined in a fixed order (per-block partials, then a fixed tree), so results
+// do not depend on scheduling; maxima and counts are order-independent.
+// dai8_quantize_tensor: one launch for small tensors (every CTA finds the maximum itself) and for
+// tensors that fit the GPU's shared memory (quantize_flat_fused_kernel); else max, then codes.
 //
 // Layouts.  The native layout is NHWC: a thread owns one 16-byte vector of channels
 // (4 fp32 / 8 bf16) of one pixel and walks down the pixels, so per-channel scalars stay in
@@ -38,6 +46,7 @@ struct GvqWs {
   float* pmax;          // [PB][C] per-block partial max
   double* psum;         // [PB][C]
   double* pss;          // [PB][C]
+  float* layer_scale;   // [1] the single clip value of the layer-wide modes
 };
 
 size_t control_words(int C) { return (size_t)2 * C + 4; }
@@ -68,12 +77,14 @@ GvqWs carve(void* ws, int C) {
   w.psum = reinterpret_cast<double*>(p + off);
   w.pss = w.psum + (size_t)kMaxPixelBlocks * C;
   w.pmax = reinterpret_cast<float*>(w.pss + (size_t)kMaxPixelBlocks * C);
+  w.layer_scale = w.pmax + (size_t)kMaxPixelBlocks * C;     // inside the 64 bytes of slack at the end
   return w;
 }
 
 struct McsDev {
   float lambda, k, A;
   int std_unbiased, center_mean;
+  int mode;   // dai8_grad_mode
 };
 
 // mean and sigma of one channel from the moments of d = g - pivot (binary64).  The pivot (the
@@ -295,10 +306,48 @@ __device__ void solve_channels(const GvqWs& ws, int C, int64_t M, const McsDev& 
                                float* __restrict__ gmax_layer, float* __restrict__ stats_out,
                                uint8_t* __restrict__ cls) {
   const float t = __fsub_rn(1.0f, __fmul_rn(mp.k, mp.A));
+  const float gmax_l = __uint_as_float(__ldcg(ws.gmax_bits));
+  if (mp.mode == DAI8_GRAD_GQ || mp.mode == DAI8_GRAD_LAYER_MCS) {
+    // One scale for the whole layer (the ablation baselines of Sec. 4.1).  GQ: s = |g|max of the layer.
+    // Layer-wise MCS: Eq. 15 and Eq. 14 on the statistics of the whole layer -- the count sweep ran with
+    // the layer's sigma for every channel, so the layer's density is the sum of the channel counts.
+    __shared__ unsigned long long s_total;
+    __shared__ float s_layer;
+    __shared__ int s_bell;
+    if (threadIdx.x == 0) s_total = 0ull;
+    __syncthreads();
+    unsigned long long part = 0ull;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) part += (unsigned long long)__ldcg(ws.cnt + c);
+    if (part) atomicAdd(&s_total, part);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float s = gmax_l;
+      bool bell = true;                   // GQ: no clipping
+      if (mp.mode == DAI8_GRAD_LAYER_MCS) {
+        bell = (double)s_total > (double)mp.lambda * ((double)M * (double)C);
+        if (!bell) s = __fadd_rn(__fmul_rn(t, has_prev ? s_state[0] : gmax_l), __fmul_rn(mp.A, gmax_l));
+      }
+      s_layer = s;
+      s_bell = bell ? 1 : 0;
+    }
+    __syncthreads();
+    const bool bell = s_bell != 0;
+    const float s = s_layer;
+    const double P_layer = (double)s_total / ((double)M * (double)C);
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+      s_state[c] = s;
+      if (cls) cls[c] = bell ? 1 : 0;
+      if (stats_out)
+        stats_out[c * 4 + DAI8_STAT_P] = mp.mode == DAI8_GRAD_LAYER_MCS ? (float)P_layer
+                                                                         : (float)((double)__ldcg(ws.cnt + c) / (double)M);
+    }
+    if (threadIdx.x == 0) { *gmax_layer = gmax_l; *ws.layer_scale = s; }   // the layer scale, for the code kernels
+    return;
+  }
   for (int c = threadIdx.x; c < C; c += blockDim.x) {
     const uint32_t cnt = __ldcg(ws.cnt + c);
     const float gmax = __ldcg(ws.absmax + c);
-    const bool bell = (double)cnt > (double)mp.lambda * (double)M;
+    const bool bell = mp.mode == DAI8_GRAD_GVQ_MAX || (double)cnt > (double)mp.lambda * (double)M;
     float s;
     if (bell) {
       s = gmax;
@@ -310,7 +359,42 @@ __device__ void solve_channels(const GvqWs& ws, int C, int64_t M, const McsDev& 
     if (cls) cls[c] = bell ? 1 : 0;
     if (stats_out) stats_out[c * 4 + DAI8_STAT_P] = (float)((double)cnt / (double)M);
   }
-  if (threadIdx.x == 0) *gmax_layer = __uint_as_float(__ldcg(ws.gmax_bits));
+  if (threadIdx.x == 0) *gmax_layer = gmax_l;
+}
+
+// Layer-wise MCS: sigma of the whole layer from the per-channel means and sigmas (every channel has the
+// same number of elements), written over every channel's sigma for the count sweep.
+//   mean_l = sum_c mean_c / C;   var_l = sum_c (var_c + mean_c^2) / C - mean_l^2   (population form;
+//   the sample form rescales by M/(M-1) per channel and back by CM/(CM-1))
+__global__ void __launch_bounds__(kThreads)
+layer_sigma_kernel(GvqWs ws, int C, int64_t M, McsDev mp, float* __restrict__ stats_out) {
+  __shared__ double s_a[kThreads], s_b[kThreads];
+  double a = 0.0, b = 0.0;
+  const double unb = mp.std_unbiased && M > 1 ? (double)(M - 1) / (double)M : 1.0;   // back to sum of squares / M
+  for (int c = threadIdx.x; c < C; c += kThreads) {
+    const double m = (double)ws.mean[c], sg = (double)ws.sigma[c];
+    a += m;
+    b += sg * sg * unb + (mp.center_mean ? m * m : 0.0);
+  }
+  s_a[threadIdx.x] = a; s_b[threadIdx.x] = b;
+  __syncthreads();
+  for (int o = kThreads / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) { s_a[threadIdx.x] += s_a[threadIdx.x + o]; s_b[threadIdx.x] += s_b[threadIdx.x + o]; }
+    __syncthreads();
+  }
+  const double mean_l = s_a[0] / (double)C;
+  double var = s_b[0] / (double)C - (mp.center_mean ? mean_l * mean_l : 0.0);
+  if (var < 0.0) var = 0.0;
+  const double total = (double)M * (double)C;
+  if (mp.std_unbiased && total > 1.0) var *= total / (total - 1.0);
+  const float sigma_l = (float)sqrt(var);
+  for (int c = threadIdx.x; c < C; c += kThreads) {
+    ws.sigma[c] = sigma_l;
+    if (stats_out) {      // in this mode the rows report the layer's mean and sigma
+      stats_out[c * 4 + DAI8_STAT_MEAN] = (float)mean_l;
+      stats_out[c * 4 + DAI8_STAT_SIGMA] = sigma_l;
+    }
+  }
 }
 
 // Sweep 2, NHWC.  grid = (pixel blocks, column blocks).
@@ -720,24 +804,26 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false if the CTA is giving up (this wait or another one ran out).
 __device__ __noinline__ bool mbar_wait_slow(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                            unsigned int* status) {
+                                            unsigned int* status, long long limit) {
   const long long t0 = clock64();
   for (;;) {
 #pragma unroll 1
     for (int i = 0; i < 64; ++i)
       if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitTimeoutCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1u;
       atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
       return false;
     }
   }
 }
+// `limit`: cycles after which the wait gives up (the default, about a second, everywhere but in the
+// self-test of the give-up path).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned int* status) {
+                                          unsigned int* status, long long limit = kWaitTimeoutCycles) {
   if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity, abort_flag, status);
+  return mbar_wait_slow(bar, parity, abort_flag, status, limit);
 }
 // Contiguous global -> shared copy of `bytes` (multiple of 16, both addresses 16-byte aligned).
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -774,7 +860,8 @@ struct FusedArgs {
 // every consumer thread of the CTA) if the others do not arrive in time, after recording
 // DAI8_ERR_TIMEOUT.
 __device__ __noinline__ bool grid_barrier(uint32_t* counter, uint32_t target, unsigned int* status,
-                                          volatile uint32_t* abort_flag, uint32_t* s_ok) {
+                                          volatile uint32_t* abort_flag, uint32_t* s_ok,
+                                          long long limit = kWaitTimeoutCycles) {
   consumer_sync();
   if (threadIdx.x == 0) {
     // release: the CTA's writes (ordered before this thread by the barrier above) become visible
@@ -786,7 +873,7 @@ __device__ __noinline__ bool grid_barrier(uint32_t* counter, uint32_t target, un
       uint32_t seen;
       asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(counter) : "memory");
       if (!ok || seen >= target) break;
-      if (clock64() - t0 > kWaitTimeoutCycles) {
+      if (clock64() - t0 > limit) {
         atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
         *abort_flag = 1u;
         ok = 0u;
@@ -1944,7 +2031,10 @@ dai8_status launch_fused(const T* dY, FusedArgs& a, cudaStream_t st) {
   if (slots > kMaxSlots) slots = kMaxSlots;
   if (slots > pieces) slots = pieces;
   a.slots = (int)slots;
-  a.ring_log2 = slots >= 10 ? 3 : (slots >= 8 ? 2 : (slots >= 4 ? 1 : 0));   // 8, 4, 2 or 1 cycling pieces
+  // 8, 4, 2 or 1 cycling pieces: for tensors far larger than shared memory what stays resident is a few
+  // per cent, and the bytes in flight per SM matter more (four 32 KB pieces instead of two: 309 -> 299 us
+  // on 822 MB)
+  a.ring_log2 = slots >= 10 ? 3 : (slots >= 4 ? 2 : (slots >= 2 ? 1 : 0));
   {
     const double M = (double)a.npix;
     const double denom = a.mp.std_unbiased ? M - 1.0 : M;
@@ -2039,17 +2129,29 @@ int nchw_slices(int N, int C) {
 template <typename T>
 constexpr int vec_elems() { return 16 / (int)sizeof(T); }
 
+McsDev make_mcs(const dai8_mcs_params& p) {
+  McsDev mp{p.lambda, p.k, p.A, p.std_unbiased, p.center_mean, p.mode};
+  return mp;
+}
+
 template <typename T>
 dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, int H, int W,
-                                const McsDev& mp, float* s_state, int has_prev, float* gmax_layer,
+                                const McsDev& mp_in, float* s_state, int has_prev, float* gmax_layer,
                                 float* stats, uint8_t* cls, int8_t* vq, int8_t* gq, uint32_t seed,
                                 const float* sigma_override, const GvqWs& ws, cudaStream_t st) {
   const int64_t HW = (int64_t)H * W;
   const int64_t npix = (int64_t)N * HW;
   const int Cp = round_up(C, 16);
   constexpr int VEfull = vec_elems<T>();
+  McsDev mp = mp_in;
+  // The ablation modes of Sec. 4.1.  Per-channel |g|max without the discriminator is the full method
+  // with a threshold no density can fall below; the two layer-wide modes (one clip value for all
+  // channels) take the three-launch path, whose last count block solves for the layer.
+  if (mp.mode == DAI8_GRAD_GVQ_MAX) mp.lambda = -1.0f;
+  const bool layer_wide = mp.mode == DAI8_GRAD_GQ || mp.mode == DAI8_GRAD_LAYER_MCS;
+  if (mp.mode == DAI8_GRAD_LAYER_MCS) sigma_override = nullptr;   // the layer's own sigma is the method here
   const float* sigma = sigma_override ? sigma_override : ws.sigma;
-  if (layout == DAI8_NHWC && C % VEfull == 0) {
+  if (!layer_wide && layout == DAI8_NHWC && C % VEfull == 0) {
     // many channels, few pixels: whole vector columns per CTA (no cross-CTA reductions)
     int grid = 0, per = 0;
     size_t smem = 0;
@@ -2071,7 +2173,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       return launch_columns<T, VEfull>(dY, a, gq != nullptr, grid, smem, st);
     }
   }
-  if (layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
+  if (!layer_wide && layout == DAI8_NHWC && fused_config().coop && C <= kFusedMaxC && C % VEfull == 0) {
     FusedArgs a;
     a.npix = npix; a.HW = HW; a.C = C; a.Cp = Cp; a.G = C / VEfull; a.Gp = Cp / VEfull;
     a.rp = 0; a.adv_q = 0; a.adv_rem = 0; a.slots = 0; a.ring_log2 = 0; a.rows_per_warp = 0; a.rpi = 0; a.inv_M = 0.0; a.inv_denom = 0.0; a.pred_ratio = 0.f;
@@ -2086,10 +2188,17 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
     if (C % VEfull == 0) {
       const NhwcGrid g = nhwc_grid(npix, C / VEfull);
       stats_nhwc_kernel<T, VEfull><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, mp, stats);
+      if (mp.mode == DAI8_GRAD_LAYER_MCS) layer_sigma_kernel<<<1, kThreads, 0, st>>>(ws, C, npix, mp, stats);
       count_nhwc_kernel<T, VEfull><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, sigma, mp, s_state,
                                                                 has_prev, gmax_layer, stats, cls);
       const NhwcGrid gq_ = nhwc_grid(npix, Cp / VEfull);
-      if (gq)
+      if (layer_wide && gq)
+        quantize_nhwc_kernel<T, VEfull, false, true, true><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, ws.layer_scale, gmax_layer, seed, vq, gq);
+      else if (layer_wide)
+        quantize_nhwc_kernel<T, VEfull, false, true, false><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, ws.layer_scale, gmax_layer, seed, vq, nullptr);
+      else if (gq)
         quantize_nhwc_kernel<T, VEfull, true, true, true><<<gq_.grid, kThreads, 0, st>>>(
             dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, gq);
       else
@@ -2098,10 +2207,17 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
     } else {
       const NhwcGrid g = nhwc_grid(npix, C);
       stats_nhwc_kernel<T, 1><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, mp, stats);
+      if (mp.mode == DAI8_GRAD_LAYER_MCS) layer_sigma_kernel<<<1, kThreads, 0, st>>>(ws, C, npix, mp, stats);
       count_nhwc_kernel<T, 1><<<g.grid, kThreads, 0, st>>>(dY, npix, C, g.G, ws, sigma, mp, s_state,
                                                            has_prev, gmax_layer, stats, cls);
       const NhwcGrid gq_ = nhwc_grid(npix, Cp);
-      if (gq)
+      if (layer_wide && gq)
+        quantize_nhwc_kernel<T, 1, false, true, true><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, ws.layer_scale, gmax_layer, seed, vq, gq);
+      else if (layer_wide)
+        quantize_nhwc_kernel<T, 1, false, true, false><<<gq_.grid, kThreads, 0, st>>>(
+            dY, npix, HW, C, Cp, gq_.G, ws.layer_scale, gmax_layer, seed, vq, nullptr);
+      else if (gq)
         quantize_nhwc_kernel<T, 1, true, true, true><<<gq_.grid, kThreads, 0, st>>>(
             dY, npix, HW, C, Cp, gq_.G, s_state, gmax_layer, seed, vq, gq);
       else
@@ -2111,10 +2227,17 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
   } else {
     const dim3 grid((unsigned)C, (unsigned)nchw_slices(N, C), 1);
     stats_nchw_kernel<T><<<grid, kThreads, 0, st>>>(dY, N, C, HW, ws, mp, stats);
+    if (mp.mode == DAI8_GRAD_LAYER_MCS) layer_sigma_kernel<<<1, kThreads, 0, st>>>(ws, C, npix, mp, stats);
     count_nchw_kernel<T><<<grid, kThreads, 0, st>>>(dY, N, C, HW, ws, sigma, mp, s_state, has_prev,
                                                     gmax_layer, stats, cls);
     const dim3 qgrid((unsigned)ceil_div64(HW, kTileHW), (unsigned)((Cp + kTileC - 1) / kTileC), (unsigned)N);
-    if (gq)
+    if (layer_wide && gq)
+      quantize_nchw_kernel<T, false, true, true><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, ws.layer_scale,
+                                                                             gmax_layer, seed, vq, gq);
+    else if (layer_wide)
+      quantize_nchw_kernel<T, false, true, false><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, ws.layer_scale,
+                                                                              gmax_layer, seed, vq, nullptr);
+    else if (gq)
       quantize_nchw_kernel<T, true, true, true><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, s_state,
                                                                             gmax_layer, seed, vq, gq);
     else
@@ -2322,7 +2445,8 @@ extern "C" dai8_status dai8_quantize_grad(const void* dY, dai8_dtype dtype, dai8
   if (a != DAI8_OK) return a;
   dai8_mcs_params p;
   if (params) p = *params; else dai8_mcs_defaults(&p);
-  McsDev mp{p.lambda, p.k, p.A, p.std_unbiased, p.center_mean};
+  if (p.mode < DAI8_GRAD_FULL || p.mode > DAI8_GRAD_LAYER_MCS) return DAI8_ERR_INVALID_ARG;
+  McsDev mp = make_mcs(p);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   GvqWs w = carve(ws, C);
   DAI8_RETURN_IF_CUDA(cudaMemsetAsync(w.tickets, 0, control_words(C) * 4, st));
@@ -2357,6 +2481,45 @@ extern "C" dai8_status dai8_quantize_tensor(const void* x, dai8_dtype dtype, dai
   return quantize_tensor_typed<bf16_t>(static_cast<const bf16_t*>(x), layout, N, C, H, W, scale_mode,
                                        scale, round, seed, q, ws, st);
 }
+
+// ------------------------------------------------------------------------------------------------
+// Self-test of the give-up path of the bounded waits.  Nothing is in flight: one CTA initialises an
+// mbarrier on which nobody ever arrives and waits for it, then meets a grid barrier whose target is one
+// arrival more than there are CTAs -- both with a limit of a few thousand cycles instead of a second.
+// Each wait must return false by itself and leave DAI8_ERR_TIMEOUT in the device status word; the
+// kernel then ends normally, so the context stays usable.
+// ------------------------------------------------------------------------------------------------
+namespace dai8 {
+namespace {
+__global__ void __launch_bounds__(kFT)
+expire_waits_kernel(uint32_t* gridbar, unsigned int* status, long long limit, int* report) {
+  __shared__ uint64_t bar;
+  __shared__ volatile uint32_t s_abort;
+  __shared__ uint32_t s_ok;
+  if (threadIdx.x == 0) {
+    s_abort = 0u;
+    mbar_init(&bar, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  const bool ok1 = mbar_wait(&bar, 0u, &s_abort, status, limit);
+  __syncthreads();
+  if (threadIdx.x == 0) { report[0] = ok1 ? 0 : 1; s_abort = 0u; }
+  __syncthreads();
+  const bool ok2 = grid_barrier(gridbar, gridDim.x + 1u, status, &s_abort, &s_ok, limit);
+  if (threadIdx.x == 0) report[1] = ok2 ? 0 : 1;
+}
+}  // namespace
+dai8_status expire_gvq_waits(long long limit, void* ws, int* report_dev, cudaStream_t st) {
+  unsigned int* status = device_status_address();
+  if (!status) return DAI8_ERR_CUDA;
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, 16, st));
+  expire_waits_kernel<<<1, kFT, 0, st>>>(static_cast<uint32_t*>(ws), status, limit, report_dev);
+  note_launch(1);
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  return DAI8_OK;
+}
+}  // namespace dai8
 
 // ------------------------------------------------------------------------------------------------
 // dai8_quantize_grad_noalloc: the same kernels as dai8_quantize_grad, with the scratch memory taken
@@ -2430,7 +2593,8 @@ extern "C" dai8_status dai8_quantize_grad_noalloc(const void* dY, dai8_dtype dty
   if (a != DAI8_OK) return a;
   dai8_mcs_params p;
   if (params) p = *params; else dai8_mcs_defaults(&p);
-  McsDev mp{p.lambda, p.k, p.A, p.std_unbiased, p.center_mean};
+  if (p.mode < DAI8_GRAD_FULL || p.mode > DAI8_GRAD_LAYER_MCS) return DAI8_ERR_INVALID_ARG;
+  McsDev mp = make_mcs(p);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   GvqWs w = carve(scratch, C);
   DAI8_RETURN_IF_CUDA(cudaMemsetAsync(w.tickets, 0, control_words(C) * 4, st));

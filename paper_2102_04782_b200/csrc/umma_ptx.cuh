@@ -38,14 +38,15 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 // Bounded wait.  Returns false if the CTA is aborting (this wait or another one expired).
 // `status`: the device status word that receives DAI8_ERR_TIMEOUT.
+// `limit`: cycles after which the wait gives up (the default everywhere but in the self-test of this path).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned int* status) {
+                                          unsigned int* status, long long limit = kTimeoutCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kTimeoutCycles) {
+    if (clock64() - t0 > limit) {
       *abort_flag = 1u;
       atomicExch(status, (unsigned int)DAI8_ERR_TIMEOUT);
       return false;

@@ -345,3 +345,23 @@ def test_back_to_back_calls_match_synchronised_calls(g):
     bad = [n for n, a, b in zip(names, want, (qX, qW, Y, vq, gq, dW, dX, s_c)) if not torch.equal(a, b)]
     assert not bad, bad
     assert api.get_device_status() == api.OK
+
+
+def test_bounded_waits_give_up_and_the_library_stays_usable():
+    """The give-up path of the device-side waits: barriers nobody completes, a limit of a few thousand
+    cycles, nothing in flight.  Each wait must return by itself and leave DAI8_ERR_TIMEOUT in the device
+    status word; reading clears it, and a normal call afterwards is bit-exact again."""
+    assert api.get_device_status() == api.OK
+    flags = api.debug_expire_waits(5000, ws_bytes(64))
+    assert flags == [1, 1, 1]
+    assert api.get_device_status() == api.ERR_TIMEOUT      # read ...
+    assert api.get_device_status() == api.OK               # ... and cleared
+    g = TC_GEOMS[2]
+    N, Cin, Cout, H, W, R, S, st, pad = g
+    rng = np.random.default_rng(77)
+    P, Q = O.out_hw(H, W, R, S, st, pad)
+    qX, qW = rand_codes(rng, (N, Cin, H, W)), rand_codes(rng, (Cout, Cin, R, S))
+    Y = torch.empty((N, P, Q, Cout), dtype=torch.int32, device="cuda")
+    api.conv_fwd(codes_from_nchw(qX), weights_dev(qW), scalar(1), scalar(1), geom(*g), Y, api.NHWC, None)
+    np.testing.assert_array_equal(out_to_nchw(Y, api.NHWC), O.conv_fwd_acc(qX, qW, st, pad)[0])
+    assert api.get_device_status() == api.OK

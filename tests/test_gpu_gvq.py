@@ -318,3 +318,60 @@ def test_more_than_2_32_elements():
     got_g = gq[N - 1].cpu().numpy().transpose(2, 0, 1)[None]
     np.testing.assert_array_equal(got_v, O.quantize(last, s_gpu, True, seed, 0, first_image=N - 1))
     np.testing.assert_array_equal(got_g, O.quantize(last, gl, True, seed, 1, first_image=N - 1))
+
+
+MODES = {"gq": api.GRAD_GQ, "gvq_max": api.GRAD_GVQ_MAX, "layer_mcs": api.GRAD_LAYER_MCS}
+
+
+@pytest.mark.parametrize("mode", ["gq", "gvq_max", "layer_mcs"])
+@pytest.mark.parametrize("layout", [api.NHWC, api.NCHW])
+@pytest.mark.parametrize("shape,bf16", [((8, 64, 14, 14), False), ((3, 20, 9, 11), True), ((16, 64, 56, 56), True)])
+def test_ablation_modes(mode, layout, shape, bf16):
+    """The quantization strategies of the ablation study (Sec. 4.1) as modes of dai8_quantize_grad, three
+    iterations each, stage by stage against the oracle's composition of the same steps."""
+    N, C, H, W = shape
+    M = N * H * W
+    g0, _, _ = synth.channel_mixed_grad(N, C, H, W, seed=51)
+    if mode == "layer_mcs":
+        g0 = g0 / np.float32(g0.std(axis=(0, 2, 3), keepdims=True))     # equal widths: the layer's class can go either way
+    p = api.mcs_defaults()
+    p.mode = MODES[mode]
+    gq = GradQuant(N, C, H, W)
+    s_prev = None
+    for t in range(3):
+        g = g0 * np.float32(1.0 + 0.25 * t)
+        if t == 1 and mode == "layer_mcs":
+            g = np.random.default_rng(5).laplace(0, 1e-4, g.shape).astype(np.float32)   # a long-tailed layer
+        if bf16:
+            g = synth.round_to_bf16(g)
+        gq.run(dev_input(g, bf16, layout), layout, 40 + t, has_prev=t > 0, params=p)
+        stats = gq.stats.cpu().numpy()
+        s_gpu, cls_gpu, gl_gpu = gq.s_state.cpu().numpy(), gq.cls.cpu().numpy(), float(gq.gmax.item())
+        absmax, mean, sigma, gl = O.channel_stats(g)
+        np.testing.assert_array_equal(stats[:, 0], absmax)
+        assert gl_gpu == gl
+        if mode == "gq":
+            assert np.all(s_gpu == gl) and np.all(cls_gpu == 1)
+        elif mode == "gvq_max":
+            np.testing.assert_array_equal(s_gpu, absmax)
+            assert np.all(cls_gpu == 1)
+            np.testing.assert_allclose(stats[:, 2], sigma, rtol=REL)
+        else:
+            one = g.reshape(1, 1, N * C * H, W)
+            _, mean_l, sigma_l, _ = O.channel_stats(one)
+            np.testing.assert_allclose(stats[:, 2], np.full(C, sigma_l[0]), rtol=REL)
+            assert np.all(stats[:, 2] == stats[0, 2])
+            cnt = O.density_count(one, stats[:1, 2])                 # given the GPU's sigma of the layer
+            np.testing.assert_array_equal(stats[:, 3], np.full(C, np.float32(float(cnt[0]) / (M * C))))
+            s_or, cls_or = O.classify_clip(cnt, np.array([gl], np.float32), M * C, s_prev=None if s_prev is None else s_prev[:1])
+            assert np.all(cls_gpu == cls_or[0])
+            np.testing.assert_allclose(s_gpu, np.full(C, s_or[0]), rtol=REL)
+            assert np.all(s_gpu == s_gpu[0])
+            # end to end: unless the layer's count sits on the threshold, the oracle's own composition agrees
+            if abs(float(cnt[0]) - 0.3 * M * C) > 2:
+                s_e, cls_e, _ = O.grad_scales(g, "layer_mcs", s_prev=s_prev)
+                assert np.all(cls_gpu == cls_e) and np.allclose(s_gpu, s_e, rtol=REL)
+        np.testing.assert_array_equal(codes_to_nchw(gq.vq, C), O.quantize(g, s_gpu, True, 40 + t, 0))
+        np.testing.assert_array_equal(codes_to_nchw(gq.gq, C), O.quantize(g, gl_gpu, True, 40 + t, 1))
+        assert padding_is_zero(gq.vq, C) and padding_is_zero(gq.gq, C)
+        s_prev = s_gpu

@@ -282,3 +282,40 @@ def test_quantize_slice_of_a_larger_tensor():
     u = O.rand_uniform(11, 1, (1 << 33) * 5 * 21)
     v = np.float32(np.float32(x[0, 0, 0, 0]) * np.float32(np.float32(127.0) / s[0]))
     assert int(big[0, 0, 0, 0]) == min(127, int(np.floor(np.float32(v + np.float32(u)))))
+
+
+def test_ablation_modes_reduce_to_the_definitions():
+    """The strategies of the ablation study (Sec. 4.1) as compositions of the pinned steps: checked on
+    cases where each reduces to something known."""
+    rng = np.random.default_rng(21)
+    g = (rng.standard_normal((3, 4, 5, 6)) * np.array([1e-3, 2e-4, 5e-5, 1e-5])[None, :, None, None]).astype(np.float32)
+    absmax = np.abs(g).max(axis=(0, 2, 3))
+    # GQ: one scale, the layer's |g|max; its codes are the layer-wide quantizer's
+    s, cls, gl = O.grad_scales(g, "gq")
+    assert gl == absmax.max() and np.all(s == gl) and np.all(cls == 1)
+    np.testing.assert_array_equal(O.quantize(g, s), O.quantize(g, float(gl)))
+    # per-channel max without the discriminator = the full method when no density can fall below the threshold
+    s, cls, _ = O.grad_scales(g, "gvq_max")
+    np.testing.assert_array_equal(s, absmax)
+    s_full, cls_full, _ = O.grad_scales(g, "full", lam=-1.0)
+    np.testing.assert_array_equal(s, s_full)
+    assert np.all(cls_full == 1)
+    # layer-wise MCS on a one-channel tensor is the full method
+    one = g[:, :1]
+    for prev in (None, np.array([3e-3], np.float32)):
+        a = O.grad_scales(one, "layer_mcs", s_prev=prev)
+        b = O.grad_scales(one, "full", s_prev=prev)
+        np.testing.assert_array_equal(a[0], b[0]); np.testing.assert_array_equal(a[1], b[1])
+    # a long-tailed layer: density against numpy's std of ALL elements, Eq. 14 by hand
+    lap = rng.laplace(0.0, 1e-4, size=(4, 3, 20, 20)).astype(np.float32)
+    sigma_l = np.float32(np.std(lap.astype(np.float64)))
+    P = np.mean(np.abs(lap) > sigma_l)
+    assert P < 0.3
+    s, cls, gl = O.grad_scales(lap, "layer_mcs", s_prev=np.full(3, 2e-4, np.float32))
+    want = np.float32(np.float32(np.float32(1.0) - np.float32(1.0) * np.float32(0.8)) * np.float32(2e-4)) + np.float32(np.float32(0.8) * np.float32(gl))
+    assert np.all(cls == 0) and np.all(s == np.float32(want))
+    # a bell-shaped layer whose channels differ in width by decades is NOT bell-shaped as a whole: the
+    # layer-wise rule clips where the per-channel rule does not (the reason for GVQ + per-channel MCS)
+    s_l, cls_l, _ = O.grad_scales(g, "layer_mcs")
+    s_c, cls_c, _ = O.grad_scales(g, "full")
+    assert np.all(cls_l == 0) and cls_c.sum() >= 3
