@@ -704,6 +704,31 @@ def run_layer_report(args):
     print(json.dumps(out))
 
 
+def run_probe(args):
+    """The two micro-measurements the kernel designs lean on, from the library's own debug entries."""
+    import torch
+    from paper_2102_04782_b200 import api
+    torch.cuda.set_device(0)
+    api.lib()
+    ws = torch.empty(64, dtype=torch.uint8, device="cuda")
+    peaks = measured_peaks()
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    mhz = 1965.0
+    mma = []
+    for rb in (128, 64, 32):
+        for n in (16, 64, 128, 256):
+            issue, done = api.debug_probe_mma(n, rb, 4096, ws)
+            mma.append({"n_cols": n, "row_bytes": rb, "issue_cycles": round(issue, 1), "complete_cycles": round(done, 1),
+                        "tops_at_max_clock": round(2 * 128 * n * 32 / done * mhz * 1e6 * sms / 1e12, 1)})
+    sr = api.debug_probe_sr(2000, ws)
+    out = {"probe": "tcgen05.mma.kind::i8 issue rate and stochastic-rounding arithmetic rate", "sms": sms,
+           "sm_max_mhz_assumed": mhz, "mma_m128_k32": mma,
+           "sr_elements_per_second": sr, "sr_equivalent_gbs_bf16_dual": round(sr * 4 / 1e9, 1),
+           "note": "tops_at_max_clock = 2*128*N*32 / complete_cycles * clock * SMs; sr_equivalent_gbs = elements/s x (2 B in + 2 B out)",
+           "int8_proxy_peak_tops": INT8_OVER_BF16 * peaks["bf16_burst"], "hbm_peak_gbs": peaks["hbm_gbs"]}
+    print(json.dumps(out))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -717,8 +742,11 @@ def main():
     ap.add_argument("--layers", default=None, choices=["conv2x", "resnet50", "mobilenetv2", "vgg16"],
                     help="print a per-layer report for a network configuration instead of the benchmark line")
     ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--probe", action="store_true", help="print the tcgen05.mma issue-rate and rounding-arithmetic micro-measurements")
     args = ap.parse_args()
-    if args.layers:
+    if args.probe:
+        run_probe(args)
+    elif args.layers:
         run_layer_report(args)
     elif args.impl == "reference":
         run_reference(args)

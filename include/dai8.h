@@ -242,6 +242,21 @@ dai8_status dai8_get_device_status(int* host_status, void* stream);
 dai8_status dai8_debug_expire_waits(uint64_t limit_cycles, int* report /* host */, void* ws,
                                     size_t ws_bytes, void* stream);
 
+/* Two micro-measurements behind the library's tiling decisions (`python bench.py --probe`).  Both
+ * synchronise `stream`; ws: 32 bytes of device scratch.
+ *   dai8_debug_probe_mma  cycles per tcgen05.mma.kind::i8 of M = 128, K = 32 and `n_cols` (16..256,
+ *       multiple of 16) accumulator columns, operands resident in shared memory in rows of `row_bytes`
+ *       (32, 64, 128), `count` (multiple of 4) instructions issued back to back on every SM:
+ *       *issue_cycles until the last issue returned, *complete_cycles until the last one finished,
+ *       both divided by count (host pointers).
+ *   dai8_debug_probe_sr   elements per second (host pointer) of the code sweep's per-element
+ *       arithmetic (index hash, two uniforms, two stochastic roundings, packing) on values held in
+ *       registers, `iters` vectors of 8 elements per thread, whole GPU. */
+dai8_status dai8_debug_probe_mma(int n_cols, int row_bytes, int count, double* issue_cycles,
+                                 double* complete_cycles, void* ws, size_t ws_bytes, void* stream);
+dai8_status dai8_debug_probe_sr(int iters, double* elements_per_second, void* ws, size_t ws_bytes,
+                                void* stream);
+
 #ifdef __cplusplus
 }
 #endif

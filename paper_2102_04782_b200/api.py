@@ -28,6 +28,7 @@ EXPORTS = [
     "dai8_conv_workspace_bytes",
     "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
     "dai8_launch_count", "dai8_get_device_status", "dai8_debug_expire_waits",
+    "dai8_debug_probe_mma", "dai8_debug_probe_sr",
 ]
 
 
@@ -97,6 +98,9 @@ def lib() -> ctypes.CDLL:
                                            c_size_t, c_void_p]
         l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
         l.dai8_debug_expire_waits.argtypes = [c_uint64, ctypes.POINTER(c_int), c_void_p, c_size_t, c_void_p]
+        dp = ctypes.POINTER(ctypes.c_double)
+        l.dai8_debug_probe_mma.argtypes = [c_int, c_int, c_int, dp, dp, c_void_p, c_size_t, c_void_p]
+        l.dai8_debug_probe_sr.argtypes = [c_int, dp, c_void_p, c_size_t, c_void_p]
         _lib = l
     return _lib
 
@@ -165,6 +169,23 @@ def debug_expire_waits(limit_cycles: int, ws: torch.Tensor):
     p, n = _ws_args(ws)
     _check(lib().dai8_debug_expire_waits(limit_cycles, rep, p, n, _stream()), "dai8_debug_expire_waits")
     return list(rep)
+
+
+def debug_probe_mma(n_cols: int, row_bytes: int, count: int, ws: torch.Tensor):
+    """dai8_debug_probe_mma: (issue, complete) cycles per tcgen05.mma.kind::i8 with operands in shared memory."""
+    a, b = ctypes.c_double(0), ctypes.c_double(0)
+    p, n = _ws_args(ws)
+    _check(lib().dai8_debug_probe_mma(n_cols, row_bytes, count, ctypes.byref(a), ctypes.byref(b), p, n, _stream()),
+           "dai8_debug_probe_mma")
+    return a.value, b.value
+
+
+def debug_probe_sr(iters: int, ws: torch.Tensor) -> float:
+    """dai8_debug_probe_sr: elements per second of the code sweep's arithmetic in registers."""
+    v = ctypes.c_double(0)
+    p, n = _ws_args(ws)
+    _check(lib().dai8_debug_probe_sr(iters, ctypes.byref(v), p, n, _stream()), "dai8_debug_probe_sr")
+    return v.value
 
 
 def quantize_tensor_workspace_bytes() -> int:

@@ -122,6 +122,7 @@ extern "C" dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const f
     return umma_fwd(A, Wp, sX, sW, pw, out, st);
   }
   if (mode == 2) return Kp ? DAI8_ERR_WORKSPACE : DAI8_ERR_UNSUPPORTED;
+  log_choice("conv_fwd: direct kernel");
   return direct_fwd(qX, qW, sX, sW, cs, out, st);
 }
 
@@ -157,6 +158,7 @@ extern "C" dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, co
   if (mode == 2) return DAI8_ERR_UNSUPPORTED;
   dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/0, st);
   if (r != DAI8_OK) return r;
+  log_choice("conv_bwd_data: direct kernel");
   return direct_bwd_data(gq, wT, gmax, sW, cs, out, st);
 }
 
@@ -192,6 +194,7 @@ extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, 
     return DAI8_ERR_UNSUPPORTED;
   } else {
     DAI8_RETURN_IF_CUDA(cudaMemsetAsync(acc, 0, dw_acc_bytes(cs), st));
+    log_choice("conv_bwd_filter: direct kernel");
     r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
   }
   if (r != DAI8_OK) return r;

@@ -584,9 +584,7 @@ dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb,
                                    (cuuint64_t)pb.P * pb.Q * pb.Nout * out_es};
     const cuuint32_t box[4] = {128, (cuuint32_t)prm.TX, (cuuint32_t)(32 / prm.TX), 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = driver_api().tiled(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, out.ptr, dims, strides, box, estr,
-                                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, out.ptr, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   {
@@ -595,9 +593,7 @@ dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb,
     const cuuint64_t strides[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.W * pb.Kc, (cuuint64_t)pb.H * pb.W * pb.Kc};
     const cuuint32_t box[4] = {(cuuint32_t)prm.kc_bytes, (cuuint32_t)prm.TX, (cuuint32_t)(prm.TY + pb.R - 1), 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
-    CUresult r = driver_api().tiled(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides, box,
-                                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
-                                    CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides, box, estr, swizzle_for(prm.kc_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   if (pb.b_mn) {
@@ -607,18 +603,14 @@ dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb,
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Brows, (cuuint64_t)pb.b_taps * pb.Brows};
     const cuuint32_t box[3] = {(cuuint32_t)prm.b_bw, 1, (cuuint32_t)prm.kc_bytes};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
-                                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.b_bw),
-                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box, estr, swizzle_for(prm.b_bw), CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   } else {
     const cuuint64_t dims[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)(pb.R * pb.S), (cuuint64_t)pb.Brows};
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.R * pb.S * pb.Kc};
     const cuuint32_t box[3] = {(cuuint32_t)prm.kc_bytes, 1, (cuuint32_t)prm.BN};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
-                                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
-                                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box, estr, swizzle_for(prm.kc_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   const int a_stage = pb.S * (prm.TY + pb.R - 1) * prm.TX * prm.kc_bytes;
@@ -631,6 +623,10 @@ dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb,
   int ctas = sm_count();
   if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
   if (ctas > num_tiles) ctas = num_tiles;
+  log_choice("igemm_halo_kernel: %d x %d patches, N=%d (%d tiles x %d), kc=%d x %d chunks, taps %dx%d, weights %s (%d pieces), A stages %d, %d accumulators, %s, %d CTAs",
+             prm.TY, prm.TX, prm.BN, prm.m_tiles, prm.n_tiles, prm.kc_bytes, prm.chunks, prm.R, prm.S,
+             prm.b_resident ? "resident" : (prm.b_mn ? "streamed in place" : "streamed"), prm.b_resident ? pb.R * pb.S * prm.chunks : prm.b_stages,
+             prm.a_stages, prm.nbuf, prm.tma_store ? "tile stores" : "register stores", ctas);
   DAI8_RETURN_IF_CUDA(launch_dependent(igemm_halo_kernel, dim3((unsigned)ctas), dim3(kHaloThreads), smem_bytes, st, mapA, mapB,
                                        mapC, prm));
   note_launch();

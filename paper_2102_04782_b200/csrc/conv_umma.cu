@@ -543,9 +543,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const cuuint64_t strides[1] = {(cuuint64_t)pb.Nout * out_es};
     const cuuint32_t box[2] = {128, 32};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = driver_api().tiled(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, out.ptr, dims, strides, box, estr,
-                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapC, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, out.ptr, dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   {
@@ -555,10 +553,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const int lower[2] = {pb.lower_w, pb.lower_h};
     const int upper[2] = {pb.lower_w + (pb.Q - 1) * pb.sw - (pb.Wi - 1), pb.lower_h + (pb.P - 1) * pb.sh - (pb.Hi - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)pb.sw, (cuuint32_t)pb.sh, 1};
-    CUresult r = driver_api().im2col(&mapA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(pb.A), dims, strides,
-                                 lower, upper, (cuuint32_t)prm.kc_bytes, (cuuint32_t)kBM, estr,
-                                 CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
-                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_im2col_cached(&mapA, const_cast<int8_t*>(pb.A), dims, strides, lower, upper, (cuuint32_t)prm.kc_bytes, (cuuint32_t)kBM, estr, swizzle_for(prm.kc_bytes));
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   if (pb.b_mn) {
@@ -568,18 +563,14 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Brows, (cuuint64_t)pb.b_taps * pb.Brows};
     const cuuint32_t box[3] = {(cuuint32_t)prm.b_bw, 1, (cuuint32_t)prm.kc_bytes};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
-                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.b_bw),
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box, estr, swizzle_for(prm.b_bw), CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   } else {
     const cuuint64_t dims[3] = {(cuuint64_t)pb.Kc, (cuuint64_t)(pb.R * pb.S), (cuuint64_t)pb.Brows};
     const cuuint64_t strides[2] = {(cuuint64_t)pb.Kc, (cuuint64_t)pb.R * pb.S * pb.Kc};
     const cuuint32_t box[3] = {(cuuint32_t)prm.kc_bytes, 1, (cuuint32_t)prm.BN};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = driver_api().tiled(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box,
-                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle_for(prm.kc_bytes),
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<int8_t*>(pb.B), dims, strides, box, estr, swizzle_for(prm.kc_bytes), CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   const size_t smem_bytes = (size_t)(prm.b_resident ? b_res : 0) + stage_out_bytes + (size_t)stages * stage_bytes + 1024;
@@ -590,6 +581,10 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   int ctas = sm_count();
   if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
   if (ctas > num_tiles) ctas = num_tiles;
+  log_choice("igemm_kmajor_kernel: im2col, N=%d (%d tiles x %d), kc=%d, %d chunks in stages of %d, taps %dx%d stride %dx%d, weights %s, %d stages, %s, %d CTAs",
+             prm.BN, prm.m_tiles, prm.n_tiles, prm.kc_bytes, total_chunks, prm.G, prm.R, prm.S, prm.sh, prm.sw,
+             prm.b_resident ? "resident" : (prm.b_mn ? "streamed in place" : "streamed"), prm.stages,
+             prm.tma_store ? "tile stores" : "register stores", ctas);
   DAI8_RETURN_IF_CUDA(launch_dependent(igemm_kmajor_kernel, dim3((unsigned)ctas), dim3(kThreadsPersist), smem_bytes, st, mapA, mapB, mapC, prm));
   note_launch();
   return DAI8_OK;
@@ -981,9 +976,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
     const cuuint64_t strides[1] = {(cuuint64_t)cs.Coutp};
     const cuuint32_t box[2] = {128, (cuuint32_t)prm.kp};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = driver_api().tiled(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box,
-                                estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_tiled_cached(&mapG, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t*>(vq), dims, strides, box, estr, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   {
@@ -992,16 +985,15 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
     const int lower[2] = {-cs.pw, -cs.ph};
     const int upper[2] = {-cs.pw + (cs.Q - 1) * cs.sw - (cs.W - 1), -cs.ph + (cs.P - 1) * cs.sh - (cs.H - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)cs.sw, (cuuint32_t)cs.sh, 1};
-    CUresult r = driver_api().im2col(&mapX, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<int8_t*>(qX), dims, strides, lower,
-                                 upper, (cuuint32_t)prm.bw, (cuuint32_t)prm.kp, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                 swizzle_for(prm.bw), CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    CUresult r = encode_im2col_cached(&mapX, const_cast<int8_t*>(qX), dims, strides, lower, upper, (cuuint32_t)prm.bw, (cuuint32_t)prm.kp, estr, swizzle_for(prm.bw));
     if (r != CUDA_SUCCESS) return DAI8_ERR_CUDA;
   }
   const size_t smem_bytes = (size_t)stages * stage_bytes + 1024;
   static std::atomic<int> attr_done[64];
   if (set_max_smem_once(attr_done, wgrad_mnmajor_kernel, kWgradSmem + 1024) != cudaSuccess) return DAI8_ERR_CUDA;
   const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
+  log_choice("wgrad_mnmajor_kernel: %d pixel slices x %d tap groups of %d x %d channel tiles of %d x %d output-channel tiles, %d pixels per stage, %d stages",
+             ksplit, ngroups, prm.tg, prm.ci_tiles, prm.nb * prm.bw, co_tiles, prm.kp, stages);
   DAI8_RETURN_IF_CUDA(launch_dependent(wgrad_mnmajor_kernel, grid, dim3(kThreadsIgemm), smem_bytes, st, mapG, mapX, prm));
   note_launch();
   return DAI8_OK;

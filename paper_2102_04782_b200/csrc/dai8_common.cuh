@@ -5,6 +5,9 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
 
 #include "../../include/dai8.h"
 
@@ -53,6 +56,21 @@ inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 bl
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// DAI8_LOG=1 in the environment: one line on stderr per call, naming the kernel chosen and its tiling.
+inline bool log_enabled() {
+  static const bool on = [] { const char* e = std::getenv("DAI8_LOG"); return e && e[0] && e[0] != '0'; }();
+  return on;
+}
+inline void log_choice(const char* fmt, ...) {
+  if (!log_enabled()) return;
+  va_list ap;
+  va_start(ap, fmt);
+  std::fputs("[dai8] ", stderr);
+  std::vfprintf(stderr, fmt, ap);
+  std::fputc('\n', stderr);
+  va_end(ap);
 }
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

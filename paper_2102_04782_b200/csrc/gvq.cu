@@ -2170,6 +2170,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       a.mp = mp; a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
       a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
       if (!a.status) return DAI8_ERR_CUDA;
+      log_choice("quantize_grad: gvq_columns_kernel, %d CTAs x %d vector columns, %lld pixels", grid, per, (long long)npix);
       return launch_columns<T, VEfull>(dY, a, gq != nullptr, grid, smem, st);
     }
   }
@@ -2182,6 +2183,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
     a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
     if (!a.status) return DAI8_ERR_CUDA;
     const bool idx32 = npix * C < ((int64_t)1 << 32);   // NCHW element indices fit 32 bits
+    log_choice("quantize_grad: gvq_fused_nhwc_kernel, C=%d, %lld pixels", C, (long long)npix);
     return launch_fused_select<T, VEfull>(dY, a, gq != nullptr, idx32, st);
   }
   if (layout == DAI8_NHWC) {
@@ -2244,6 +2246,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       quantize_nchw_kernel<T, true, true, false><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, s_state,
                                                                              gmax_layer, seed, vq, nullptr);
   }
+  log_choice("quantize_grad: three launches (statistics, count, codes), mode %d", mp.mode);
   note_launch(3);
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
   return DAI8_OK;

@@ -1,0 +1,162 @@
+// Two micro-measurements that the tiling decisions of the library lean on, as library entry points
+// so that anyone can repeat them (bench.py --probe prints both):
+//   * what one tcgen05.mma.kind::i8 of M = 128, K = 32 costs, by accumulator width N and by the width of
+//     the shared-memory rows, with both operands resident in shared memory and nothing else running:
+//     the floor under every convolution kernel here;
+//   * how many elements per second the arithmetic of the gradient quantizer's code sweep sustains in
+//     registers alone (counter hash, two uniforms, two stochastic roundings per element, Eq. 1 with
+//     stochastic rounding): the ALU floor under dai8_quantize_grad.
+#include "umma_ptx.cuh"
+
+namespace dai8 {
+namespace {
+
+using namespace umma;
+
+constexpr int kProbeSmem = 192 * 1024;
+
+// `count` MMAs issued by one elected lane from an unrolled block of four per loop iteration, the
+// operands walking through kProbeSmem bytes of shared memory.  out[0]: cycles until the last issue
+// returned, out[1]: cycles until the last MMA completed (CTA 0's numbers).
+__global__ void __launch_bounds__(128, 1)
+probe_mma_kernel(int N, int kc, int count, long long* out) {
+  extern __shared__ uint8_t raw[];
+  __shared__ uint64_t bar;
+  __shared__ uint32_t tmem_slot;
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(raw) + 1023) & ~(uintptr_t)1023);
+  for (int i = threadIdx.x; i < kProbeSmem / 4; i += blockDim.x) reinterpret_cast<uint32_t*>(smem)[i] = (uint32_t)i * 2654435761u;
+  if (threadIdx.x == 0) { mbar_init(&bar, 1); fence_mbar_init(); }
+  fence_async_smem();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tmem_alloc(&tmem_slot, 512u);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_slot;
+  if (threadIdx.x >= 32 && threadIdx.x < 64) {
+    const bool leader = elect_one();
+    const uint32_t hi = kmajor_desc_hi(kc);
+    const uint32_t idesc = idesc_i8_kmajor(N);
+    const uint32_t base_lo = kmajor_desc_lo(smem_u32(smem));
+    const uint32_t b_off = (uint32_t)(kBM * kc) >> 4;
+    const uint32_t step = (uint32_t)(kBM * kc + N * kc) >> 4;
+    const int wrap = kProbeSmem / (kBM * kc + N * kc);
+    const uint32_t kmask = (uint32_t)(kc / 32 - 1);
+    const long long t0 = clock64();
+    uint32_t a_lo = base_lo;
+    int p = 0;
+    for (int i = 0; i < count; i += 4) {
+      if (leader) {
+#pragma unroll
+        for (uint32_t u = 0; u < 4; ++u)
+          mma_i8_parts(tmem_base, a_lo + 2u * (u & kmask), a_lo + b_off + 2u * (u & kmask), hi, idesc, (i | u) ? 1u : 0u);
+      }
+      a_lo += step;
+      if (++p == wrap) { p = 0; a_lo = base_lo; }
+    }
+    const long long t1 = clock64();
+    if (leader) tc_commit(&bar);
+    int spins = 0;
+    while (!mbar_try_wait(&bar, 0u) && ++spins < 20000000) {}
+    const long long t2 = clock64();
+    if (blockIdx.x == 0 && leader) { out[0] = t1 - t0; out[1] = t2 - t0; out[2] = spins >= 20000000 ? 1 : 0; }
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, 512u);
+  }
+}
+
+// The per-element arithmetic of the code sweep on eight bf16 values held in registers: index hash,
+// two uniforms, both stochastic roundings (clamped form), packing to bytes.  `iters` vectors per thread.
+__global__ void __launch_bounds__(512)
+probe_sr_kernel(int iters, uint32_t seed, float inv1, float inv2, uint32_t* sink) {
+  const uint32_t key0 = sr_key(seed, 0u);
+  const uint32_t keyx0 = key0 ^ (key0 >> 16);
+  uint32_t idx = (blockIdx.x * blockDim.x + threadIdx.x) * 8u;
+  uint32_t acc = 0u;
+  uint32_t w[4] = {0x3A833A83u ^ threadIdx.x, 0xBA03BA83u, 0x39003A00u, 0xB9803B00u ^ blockIdx.x};
+#pragma unroll 1
+  for (int it = 0; it < iters; ++it) {
+    uint32_t ra[8], rb[8];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
+      const uint32_t h0 = sr_hash_folded(idx + 2u * j, keyx0), h1 = sr_hash_folded(idx + 2u * j + 1u, keyx0);
+      ra[2 * j] = quant_stochastic_bits(g0, inv1, sr_uniform_fast(h0));
+      ra[2 * j + 1] = quant_stochastic_bits(g1, inv1, sr_uniform_fast(h1));
+      rb[2 * j] = quant_stochastic_bits(g0, inv2, sr_uniform_fast(h0 * 0x9E3779B1u));
+      rb[2 * j + 1] = quant_stochastic_bits(g1, inv2, sr_uniform_fast(h1 * 0x9E3779B1u));
+      w[j] += 0x00010001u;                 // new values every iteration
+    }
+    acc ^= pack_codes4(ra[0], ra[1], ra[2], ra[3]) + pack_codes4(ra[4], ra[5], ra[6], ra[7]);
+    acc ^= pack_codes4(rb[0], rb[1], rb[2], rb[3]) - pack_codes4(rb[4], rb[5], rb[6], rb[7]);
+    idx += gridDim.x * blockDim.x * 8u;
+  }
+  if (acc == 0x12345u) *sink = acc;        // keeps the arithmetic alive
+}
+
+}  // namespace
+}  // namespace dai8
+
+using namespace dai8;
+
+extern "C" dai8_status dai8_debug_probe_mma(int n_cols, int row_bytes, int count, double* issue_cycles,
+                                            double* complete_cycles, void* ws, size_t ws_bytes, void* stream) {
+  if (!issue_cycles || !complete_cycles || !ws || ws_bytes < 32 || !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (n_cols < 16 || n_cols > 256 || n_cols % 16 != 0) return DAI8_ERR_INVALID_ARG;
+  if (row_bytes != 32 && row_bytes != 64 && row_bytes != 128) return DAI8_ERR_INVALID_ARG;
+  if (count < 4 || count > (1 << 20) || count % 4 != 0) return DAI8_ERR_INVALID_ARG;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, probe_mma_kernel, umma::kBM * 0 + kProbeSmem + 2048) != cudaSuccess) return DAI8_ERR_CUDA;
+  long long* out = static_cast<long long*>(ws);
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(out, 0, 24, st));
+  long long h[3] = {0, 0, 0};
+  for (int rep = 0; rep < 2; ++rep) {      // the second launch runs from a warm instruction cache
+    probe_mma_kernel<<<sm_count(), 128, kProbeSmem + 1024, st>>>(n_cols, row_bytes, count, out);
+    note_launch(1);
+  }
+  DAI8_RETURN_IF_CUDA(cudaGetLastError());
+  DAI8_RETURN_IF_CUDA(cudaMemcpyAsync(h, out, 24, cudaMemcpyDeviceToHost, st));
+  DAI8_RETURN_IF_CUDA(cudaStreamSynchronize(st));
+  if (h[2] != 0) return DAI8_ERR_TIMEOUT;
+  *issue_cycles = (double)h[0] / count;
+  *complete_cycles = (double)h[1] / count;
+  return DAI8_OK;
+}
+
+extern "C" dai8_status dai8_debug_probe_sr(int iters, double* elements_per_second, void* ws, size_t ws_bytes,
+                                           void* stream) {
+  if (!elements_per_second || !ws || ws_bytes < 32 || !aligned16(ws)) return DAI8_ERR_INVALID_ARG;
+  if (iters < 1 || iters > (1 << 20)) return DAI8_ERR_INVALID_ARG;
+  dai8_status a = check_device_arch();
+  if (a != DAI8_OK) return a;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaEvent_t e0, e1;
+  DAI8_RETURN_IF_CUDA(cudaEventCreate(&e0));
+  if (cudaEventCreate(&e1) != cudaSuccess) { cudaEventDestroy(e0); return DAI8_ERR_CUDA; }
+  const int ctas = sm_count() * 2;
+  float best = 0.f;
+  for (int rep = 0; rep < 3; ++rep) {
+    cudaEventRecord(e0, st);
+    probe_sr_kernel<<<ctas, 512, 0, st>>>(iters, 17u, 1.27e5f, 3.1e4f, static_cast<uint32_t*>(ws));
+    cudaEventRecord(e1, st);
+    note_launch(1);
+    if (cudaEventSynchronize(e1) != cudaSuccess) { cudaEventDestroy(e0); cudaEventDestroy(e1); return DAI8_ERR_CUDA; }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep == 0 || ms < best) best = ms;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  *elements_per_second = (double)ctas * 512.0 * 8.0 * iters / ((double)best * 1e-3);
+  return DAI8_OK;
+}

@@ -4,6 +4,10 @@
 
 #include <cuda.h>
 
+#include <mutex>
+#include <string>
+#include <unordered_map>
+
 #include "conv_internal.cuh"
 
 namespace dai8 {
@@ -243,6 +247,77 @@ inline const DriverApi& driver_api() {
     return a;
   }();
   return api;
+}
+
+// Tensor maps are a function of the call's arguments only (pointer, extents, box), and a training
+// loop repeats the same layer calls every step: encoded maps are kept in a small table keyed by the
+// encoder's arguments, so that a repeated call encodes nothing.
+struct MapCache {
+  std::mutex mu;
+  std::unordered_map<std::string, CUtensorMap> table;
+  CUresult get(const std::string& key, CUtensorMap* out, CUresult (*encode)(CUtensorMap*, const void*), const void* args) {
+    {
+      std::lock_guard<std::mutex> lock(mu);
+      auto it = table.find(key);
+      if (it != table.end()) { *out = it->second; return CUDA_SUCCESS; }
+    }
+    const CUresult r = encode(out, args);
+    if (r == CUDA_SUCCESS) {
+      std::lock_guard<std::mutex> lock(mu);
+      if (table.size() >= 4096) table.clear();
+      table.emplace(key, *out);
+    }
+    return r;
+  }
+};
+inline MapCache& map_cache() { static MapCache c; return c; }
+
+template <typename T>
+inline void key_add(std::string& k, const T* p, size_t n) { k.append(reinterpret_cast<const char*>(p), n * sizeof(T)); }
+
+struct TiledArgs {
+  CUtensorMapDataType dt; cuuint32_t rank; void* ptr; const cuuint64_t* dims; const cuuint64_t* strides;
+  const cuuint32_t* box; const cuuint32_t* estr; CUtensorMapSwizzle sw; CUtensorMapL2promotion l2;
+};
+inline CUresult encode_tiled_cached(CUtensorMap* out, CUtensorMapDataType dt, cuuint32_t rank, void* ptr,
+                                    const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                                    const cuuint32_t* estr, CUtensorMapSwizzle sw, CUtensorMapL2promotion l2) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::string key;
+  key.reserve(160);
+  const int tag[5] = {0, dev, (int)dt, (int)sw, (int)l2};
+  key_add(key, tag, 5); key_add(key, &rank, 1); key_add(key, &ptr, 1);
+  key_add(key, dims, rank); key_add(key, strides, rank - 1); key_add(key, box, rank); key_add(key, estr, rank);
+  TiledArgs a{dt, rank, ptr, dims, strides, box, estr, sw, l2};
+  return map_cache().get(key, out, [](CUtensorMap* m, const void* p) {
+    const TiledArgs& t = *static_cast<const TiledArgs*>(p);
+    return driver_api().tiled(m, t.dt, t.rank, t.ptr, t.dims, t.strides, t.box, t.estr, CU_TENSOR_MAP_INTERLEAVE_NONE, t.sw,
+                              t.l2, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }, &a);
+}
+struct Im2colArgs {
+  void* ptr; const cuuint64_t* dims; const cuuint64_t* strides; const int* lower; const int* upper;
+  cuuint32_t channels, pixels; const cuuint32_t* estr; CUtensorMapSwizzle sw;
+};
+// 4-D uint8 im2col map (the only form the library uses).
+inline CUresult encode_im2col_cached(CUtensorMap* out, void* ptr, const cuuint64_t* dims, const cuuint64_t* strides,
+                                     const int* lower, const int* upper, cuuint32_t channels, cuuint32_t pixels,
+                                     const cuuint32_t* estr, CUtensorMapSwizzle sw) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  std::string key;
+  key.reserve(160);
+  const int tag[3] = {1, dev, (int)sw};
+  key_add(key, tag, 3); key_add(key, &ptr, 1); key_add(key, dims, 4); key_add(key, strides, 3);
+  key_add(key, lower, 2); key_add(key, upper, 2); key_add(key, &channels, 1); key_add(key, &pixels, 1); key_add(key, estr, 4);
+  Im2colArgs a{ptr, dims, strides, lower, upper, channels, pixels, estr, sw};
+  return map_cache().get(key, out, [](CUtensorMap* m, const void* p) {
+    const Im2colArgs& t = *static_cast<const Im2colArgs*>(p);
+    return driver_api().im2col(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, t.ptr, t.dims, t.strides, t.lower, t.upper, t.channels,
+                               t.pixels, t.estr, CU_TENSOR_MAP_INTERLEAVE_NONE, t.sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  }, &a);
 }
 
 inline CUtensorMapSwizzle swizzle_for(int kc_bytes) {
