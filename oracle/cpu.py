@@ -38,7 +38,7 @@ def lib() -> ctypes.CDLL:
         _lib.dai8o_rand_bits.restype = ctypes.c_uint32
         _lib.dai8o_rand_bits.argtypes = [ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint64]
         _lib.dai8o_num_threads.restype = ctypes.c_int
-        for name in ("dai8o_conv_fwd_acc", "dai8o_conv_bwd_data_acc", "dai8o_conv_bwd_filter_acc"):
+        for name in ("dai8o_conv_fwd_acc", "dai8o_conv_bwd_data_acc", "dai8o_conv_bwd_filter_acc", "dai8o_conv3_acc"):
             getattr(_lib, name).restype = ctypes.c_int64
     return _lib
 
@@ -221,6 +221,37 @@ def conv_bwd_filter_acc(qX, qG, filter_hw, stride=1, pad=0, idx=None):
     acc = np.empty(n if n else (Cout, Cin, R, S), np.int64)
     ov = lib().dai8o_conv_bwd_filter_acc(_p(qX), _p(qG), _p(g), _p(idx) if n else None,
                                          ctypes.c_int64(n), _p(acc))
+    return acc, int(ov)
+
+
+def _t3(v):
+    return (v, v, v) if np.isscalar(v) else tuple(v)
+
+
+def out_dhw(D, H, W, T, R, S, stride, pad):
+    st, pd = _t3(stride), _t3(pad)
+    return tuple((n + 2 * p - k) // s + 1 for n, k, s, p in zip((D, H, W), (T, R, S), st, pd))
+
+
+def conv3_acc(op: str, a, b, geom, idx=None):
+    """Integer convolution with a depth dimension and channel groups (3-D convolution, Sec. 4.4; depth-wise
+    convolution, Sec. 4.2).  geom = (N, Cin, Cout, D, H, W, T, R, S, stride, pad, groups), stride / pad
+    scalars or (d, h, w).  op "fwd": a = X (N,Cin,D,H,W), b = W (Cout,Cin/groups,T,R,S) -> Y (N,Cout,Do,P,Q);
+    "bwd_data": a = G, b = W -> dX; "bwd_filter": a = X, b = G -> dW.  Returns (acc int64, n_overflow)."""
+    N, Cin, Cout, D, H, W, T, R, S, stride, pad, groups = geom
+    st, pd = _t3(stride), _t3(pad)
+    Do, P, Q = out_dhw(D, H, W, T, R, S, st, pd)
+    g = np.array([N, Cin, Cout, D, H, W, T, R, S, *st, *pd, groups], dtype=np.int32)
+    a = np.ascontiguousarray(a, dtype=np.int8)
+    b = np.ascontiguousarray(b, dtype=np.int8)
+    code = {"fwd": 0, "bwd_data": 1, "bwd_filter": 2}[op]
+    shapes = {0: (N, Cout, Do, P, Q), 1: (N, Cin, D, H, W), 2: (Cout, Cin // groups, T, R, S)}
+    want_a = {0: (N, Cin, D, H, W), 1: (N, Cout, Do, P, Q), 2: (N, Cin, D, H, W)}[code]
+    want_b = {0: (Cout, Cin // groups, T, R, S), 1: (Cout, Cin // groups, T, R, S), 2: (N, Cout, Do, P, Q)}[code]
+    assert a.shape == want_a and b.shape == want_b, (a.shape, want_a, b.shape, want_b)
+    idx, n = _idx(idx)
+    acc = np.empty(n if n else shapes[code], np.int64)
+    ov = lib().dai8o_conv3_acc(code, _p(a), _p(b), _p(g), _p(idx) if n else None, ctypes.c_int64(n), _p(acc))
     return acc, int(ov)
 
 

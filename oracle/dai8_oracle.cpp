@@ -363,6 +363,133 @@ int64_t dai8o_conv_bwd_filter_acc(const int8_t* X, const int8_t* G, const int* g
 }
 
 // ---------------------------------------------------------------------------------------------
+// The same three integer convolutions with a depth dimension and channel groups: the variants the
+// paper names beside the plain 2-D layer -- 3-D convolution, "treating depth dimension in the same
+// way as height and width" (Sec. 4.4), and depth-wise convolution (groups = channels, the
+// MobileNetV2 paragraph of Sec. 4.2).  X (N,Cin,D,H,W), W (Cout,Cin/groups,T,R,S), Y (N,Cout,Do,P,Q);
+// output channel co belongs to group co / (Cout/groups) and reads input channels
+// group*(Cin/groups) .. +Cin/groups-1.  With D = T = 1 and groups = 1 these are the functions above.
+// ---------------------------------------------------------------------------------------------
+struct Geom3 {
+  int N, Cin, Cout, D, H, W, T, R, S, stride_d, stride_h, stride_w, pad_d, pad_h, pad_w, groups;
+};
+
+static int64_t fwd3_at(const int8_t* X, const int8_t* Wt, const Geom3& g, int n, int co, int od, int p, int q) {
+  const int cpg = g.Cin / g.groups, opg = g.Cout / g.groups;
+  const int grp = co / opg;
+  int64_t acc = 0;
+  for (int cl = 0; cl < cpg; ++cl) {
+    const int ci = grp * cpg + cl;
+    for (int t = 0; t < g.T; ++t) {
+      const int d = od * g.stride_d + t - g.pad_d;
+      if (d < 0 || d >= g.D) continue;
+      for (int r = 0; r < g.R; ++r) {
+        const int h = p * g.stride_h + r - g.pad_h;
+        if (h < 0 || h >= g.H) continue;
+        for (int s = 0; s < g.S; ++s) {
+          const int w = q * g.stride_w + s - g.pad_w;
+          if (w < 0 || w >= g.W) continue;
+          acc += (int64_t)X[((((int64_t)n * g.Cin + ci) * g.D + d) * g.H + h) * g.W + w] *
+                 (int64_t)Wt[((((int64_t)co * cpg + cl) * g.T + t) * g.R + r) * g.S + s];
+        }
+      }
+    }
+  }
+  return acc;
+}
+
+static int64_t bwd_data3_at(const int8_t* G, const int8_t* Wt, const Geom3& g, int Do, int P, int Q, int n, int ci,
+                            int d, int h, int w) {
+  const int cpg = g.Cin / g.groups, opg = g.Cout / g.groups;
+  const int grp = ci / cpg, cl = ci - grp * cpg;
+  int64_t acc = 0;
+  for (int ol = 0; ol < opg; ++ol) {
+    const int co = grp * opg + ol;
+    for (int t = 0; t < g.T; ++t) {
+      const int dd = d + g.pad_d - t;
+      if (dd < 0 || dd % g.stride_d != 0 || dd / g.stride_d >= Do) continue;
+      for (int r = 0; r < g.R; ++r) {
+        const int hp = h + g.pad_h - r;
+        if (hp < 0 || hp % g.stride_h != 0 || hp / g.stride_h >= P) continue;
+        for (int s = 0; s < g.S; ++s) {
+          const int wq = w + g.pad_w - s;
+          if (wq < 0 || wq % g.stride_w != 0 || wq / g.stride_w >= Q) continue;
+          acc += (int64_t)G[((((int64_t)n * g.Cout + co) * Do + dd / g.stride_d) * P + hp / g.stride_h) * Q + wq / g.stride_w] *
+                 (int64_t)Wt[((((int64_t)co * cpg + cl) * g.T + t) * g.R + r) * g.S + s];
+        }
+      }
+    }
+  }
+  return acc;
+}
+
+static int64_t bwd_filter3_at(const int8_t* X, const int8_t* G, const Geom3& g, int Do, int P, int Q, int co, int cl,
+                              int t, int r, int s) {
+  const int cpg = g.Cin / g.groups, opg = g.Cout / g.groups;
+  const int ci = (co / opg) * cpg + cl;
+  int64_t acc = 0;
+  for (int n = 0; n < g.N; ++n)
+    for (int od = 0; od < Do; ++od) {
+      const int d = od * g.stride_d + t - g.pad_d;
+      if (d < 0 || d >= g.D) continue;
+      for (int p = 0; p < P; ++p) {
+        const int h = p * g.stride_h + r - g.pad_h;
+        if (h < 0 || h >= g.H) continue;
+        for (int q = 0; q < Q; ++q) {
+          const int w = q * g.stride_w + s - g.pad_w;
+          if (w < 0 || w >= g.W) continue;
+          acc += (int64_t)G[((((int64_t)n * g.Cout + co) * Do + od) * P + p) * Q + q] *
+                 (int64_t)X[((((int64_t)n * g.Cin + ci) * g.D + d) * g.H + h) * g.W + w];
+        }
+      }
+    }
+  return acc;
+}
+
+// op: 0 forward, 1 input gradient, 2 weight gradient.  Whole output (n_idx == 0) or the listed flat
+// indices of it; returns the number of results outside int32.
+int64_t dai8o_conv3_acc(int op, const int8_t* A, const int8_t* B, const int* geom, const int64_t* idx, int64_t n_idx,
+                        int64_t* acc) {
+  Geom3 g;
+  std::memcpy(&g, geom, sizeof(Geom3));
+  const int Do = out_extent(g.D, g.pad_d, g.T, g.stride_d);
+  const int P = out_extent(g.H, g.pad_h, g.R, g.stride_h);
+  const int Q = out_extent(g.W, g.pad_w, g.S, g.stride_w);
+  const int cpg = g.Cin / g.groups;
+  const int64_t full = op == 0 ? (int64_t)g.N * g.Cout * Do * P * Q
+                               : (op == 1 ? (int64_t)g.N * g.Cin * g.D * g.H * g.W : (int64_t)g.Cout * cpg * g.T * g.R * g.S);
+  const int64_t total = n_idx > 0 ? n_idx : full;
+  int64_t overflow = 0;
+#pragma omp parallel for schedule(dynamic, 64) reduction(+ : overflow)
+  for (int64_t i = 0; i < total; ++i) {
+    int64_t f = n_idx > 0 ? idx[i] : i;
+    int64_t a;
+    if (op == 0) {
+      const int q = (int)(f % Q); f /= Q;
+      const int p = (int)(f % P); f /= P;
+      const int od = (int)(f % Do); f /= Do;
+      const int co = (int)(f % g.Cout);
+      a = fwd3_at(A, B, g, (int)(f / g.Cout), co, od, p, q);
+    } else if (op == 1) {
+      const int w = (int)(f % g.W); f /= g.W;
+      const int h = (int)(f % g.H); f /= g.H;
+      const int d = (int)(f % g.D); f /= g.D;
+      const int ci = (int)(f % g.Cin);
+      a = bwd_data3_at(A, B, g, Do, P, Q, (int)(f / g.Cin), ci, d, h, w);
+    } else {
+      const int s = (int)(f % g.S); f /= g.S;
+      const int r = (int)(f % g.R); f /= g.R;
+      const int t = (int)(f % g.T); f /= g.T;
+      const int cl = (int)(f % cpg);
+      a = bwd_filter3_at(A, B, g, Do, P, Q, (int)(f / cpg), cl, t, r, s);
+    }
+    acc[i] = a;
+    if (a > INT32_MAX || a < INT32_MIN) ++overflow;
+  }
+  return overflow;
+}
+
+// ---------------------------------------------------------------------------------------------
 // De-quantization of an accumulator (Sec. 3.2, the vectorized de-quantization, and Algorithm 1
 // final two steps, with the scales the equations imply: s_X for G_W, s_W for G_X).
 //   out = (float)acc * ((sa / 127) * (sb / 127)), the scale product formed in binary32.

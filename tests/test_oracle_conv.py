@@ -169,3 +169,57 @@ def test_quantized_conv_approximates_float_conv():
     assert np.abs(dx - tx.grad.numpy()).max() < 0.03 * np.abs(tx.grad.numpy()).max()
     # the layer-wide scale drowns the small channels (the paper's motivation for GVQ)
     assert np.all(gq[:, 3] == 0) and np.abs(vq[:, 3]).max() == 127
+
+
+def _codes(rng, shape):
+    return rng.integers(-127, 128, size=shape, dtype=np.int64).astype(np.int8)
+
+
+@pytest.mark.parametrize("geom", [
+    # N, Cin, Cout, D, H, W, T, R, S, stride, pad, groups
+    (2, 4, 6, 5, 6, 7, 3, 3, 3, 1, 1, 1),                       # 3-D convolution, Sec. 4.4
+    (1, 3, 5, 6, 7, 5, 3, 1, 3, (2, 1, 2), (1, 0, 1), 1),        # strides and paddings that differ per axis
+    (2, 6, 6, 1, 7, 8, 1, 3, 3, 1, 1, 6),                        # depth-wise 2-D, Sec. 4.2
+    (1, 8, 8, 1, 9, 9, 1, 3, 3, 2, 1, 8),                        # depth-wise, stride 2
+    (2, 4, 8, 3, 5, 5, 2, 3, 3, 1, (0, 1, 1), 2),                # two groups with a depth tap
+])
+def test_conv3_against_torch_and_adjoint_identity(geom):
+    """The depth / group generalisation against torch's float64 convNd (exact on small integers) and
+    its autograd gradients, plus the exact integer adjoint identity <Y,G> = <X,dX> = <W,dW>."""
+    import torch
+    N, Cin, Cout, D, H, W, T, R, S, stride, pad, groups = geom
+    rng = np.random.default_rng(17)
+    st = (stride,) * 3 if np.isscalar(stride) else stride
+    pd = (pad,) * 3 if np.isscalar(pad) else pad
+    Do, P, Q = O.out_dhw(D, H, W, T, R, S, st, pd)
+    X, Wt, G = _codes(rng, (N, Cin, D, H, W)), _codes(rng, (Cout, Cin // groups, T, R, S)), _codes(rng, (N, Cout, Do, P, Q))
+    y, o1 = O.conv3_acc("fwd", X, Wt, geom)
+    dx, o2 = O.conv3_acc("bwd_data", G, Wt, geom)
+    dw, o3 = O.conv3_acc("bwd_filter", X, G, geom)
+    assert o1 == o2 == o3 == 0
+    tx = torch.tensor(X, dtype=torch.float64, requires_grad=True)
+    tw = torch.tensor(Wt, dtype=torch.float64, requires_grad=True)
+    ty = torch.nn.functional.conv3d(tx, tw, stride=st, padding=pd, groups=groups)
+    ty.backward(torch.tensor(G, dtype=torch.float64))
+    np.testing.assert_array_equal(y, ty.detach().numpy().astype(np.int64))
+    np.testing.assert_array_equal(dx, tx.grad.numpy().astype(np.int64))
+    np.testing.assert_array_equal(dw, tw.grad.numpy().astype(np.int64))
+    lhs = int((y * G.astype(np.int64)).sum())
+    assert lhs == int((dx * X.astype(np.int64)).sum()) == int((dw * Wt.astype(np.int64)).sum())
+    # sampled outputs equal the full ones
+    idx = rng.choice(y.size, 20, replace=False)
+    np.testing.assert_array_equal(O.conv3_acc("fwd", X, Wt, geom, idx=idx)[0], y.reshape(-1)[idx])
+
+
+def test_conv3_reduces_to_the_2d_functions():
+    """Depth 1, one group: the generalised loops are the 2-D ones (which have their own pins)."""
+    rng = np.random.default_rng(18)
+    X, Wt = _codes(rng, (2, 5, 9, 8)), _codes(rng, (7, 5, 3, 3))
+    P, Q = O.out_hw(9, 8, 3, 3, 2, 1)
+    G = _codes(rng, (2, 7, P, Q))
+    geom = (2, 5, 7, 1, 9, 8, 1, 3, 3, (1, 2, 2), (0, 1, 1), 1)
+    np.testing.assert_array_equal(O.conv3_acc("fwd", X[:, :, None], Wt[:, :, None], geom)[0][:, :, 0], O.conv_fwd_acc(X, Wt, 2, 1)[0])
+    np.testing.assert_array_equal(O.conv3_acc("bwd_data", G[:, :, None], Wt[:, :, None], geom)[0][:, :, 0],
+                                  O.conv_bwd_data_acc(G, Wt, (9, 8), 2, 1)[0])
+    np.testing.assert_array_equal(O.conv3_acc("bwd_filter", X[:, :, None], G[:, :, None], geom)[0][:, :, 0],
+                                  O.conv_bwd_filter_acc(X, G, (3, 3), 2, 1)[0])
