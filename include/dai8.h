@@ -218,6 +218,36 @@ dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, const float
                                  const float* s, const dai8_conv_geom* geom /* host */, void* dW,
                                  dai8_dtype out_dtype, void* ws, size_t ws_bytes, void* stream);
 
+/* ----------------------------------------------------------------------------------------------
+ * The same three convolutions with a depth dimension and channel groups: 3-D convolution, "treating
+ * depth dimension in the same way as height and width" (Sec. 4.4), and depth-wise convolution
+ * (groups = Cin = Cout; the MobileNetV2 paragraph of Sec. 4.2).  Arithmetic as above (int8 codes,
+ * wrapping int32 accumulators, de-quantization by the two scales); CUDA-core kernels for every
+ * geometry with T*R*S <= 32 taps, no workspace.
+ *   X (N,Cin,D,H,W), W (Cout,Cin/groups,T,R,S), Y (N,Cout,Do,P,Q); groups 0 or 1 = one group; with
+ *   several groups the channels per group must be 1 or a multiple of 4
+ *   codes: activations / gradients [N][D][H][W][Cp]; weights [Cout][T][R][S][Cgp], Cgp = Cin/groups
+ *   rounded up to 16 -- i.e. dai8_quantize_tensor of the (N, C, D*H, W) tensor, and of the weights
+ *   passed as an NCHW tensor with N = Cout, C = Cin/groups, H = T*R, W = S.  The gradient quantizer
+ *   takes a 5-D gradient the same way, as (N, C, Do*P, Q): its statistics run over everything but
+ *   the channel, and its random numbers follow the flat index, which is the same.
+ *   outputs: channels last, unpadded: Y [N][Do][P][Q][Cout], dX [N][D][H][W][Cin] (F32, BF16 or
+ *   I32 = raw accumulators); dW (Cout,Cin/groups,T,R,S) F32 or I32.
+ * -------------------------------------------------------------------------------------------- */
+typedef struct {
+  int N, Cin, Cout, D, H, W, T, R, S, stride_d, stride_h, stride_w, pad_d, pad_h, pad_w, groups;
+} dai8_conv3d_geom;
+
+dai8_status dai8_conv3d_fwd(const int8_t* qX, const int8_t* qW, const float* sX, const float* sW,
+                            const dai8_conv3d_geom* geom /* host */, void* Y, dai8_dtype out_dtype,
+                            void* stream);
+dai8_status dai8_conv3d_bwd_data(const int8_t* gq, const int8_t* qW, const float* gmax,
+                                 const float* sW, const dai8_conv3d_geom* geom /* host */, void* dX,
+                                 dai8_dtype out_dtype, void* stream);
+dai8_status dai8_conv3d_bwd_filter(const int8_t* qX, const int8_t* vq, const float* sX,
+                                   const float* s, const dai8_conv3d_geom* geom /* host */, void* dW,
+                                   dai8_dtype out_dtype, void* stream);
+
 /* Kernel family selection for the convolutions (process-wide, host side): 0 = automatic
  * (tensor-core kernels where the geometry allows, direct kernels otherwise), 1 = direct kernels
  * only, 2 = tensor-core kernels only (DAI8_ERR_UNSUPPORTED where they do not apply), 3 = like 2 but

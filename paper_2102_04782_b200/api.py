@@ -29,6 +29,7 @@ EXPORTS = [
     "dai8_conv_fwd", "dai8_conv_bwd_data", "dai8_conv_bwd_filter", "dai8_set_conv_backend",
     "dai8_launch_count", "dai8_get_device_status", "dai8_debug_expire_waits",
     "dai8_debug_probe_mma", "dai8_debug_probe_sr",
+    "dai8_conv3d_fwd", "dai8_conv3d_bwd_data", "dai8_conv3d_bwd_filter",
 ]
 
 
@@ -43,6 +44,16 @@ class ConvGeom(ctypes.Structure):
     @property
     def Q(self) -> int:
         return (self.W + 2 * self.pad_w - self.S) // self.stride_w + 1
+
+
+class Conv3dGeom(ctypes.Structure):
+    _fields_ = [(n, c_int) for n in ("N", "Cin", "Cout", "D", "H", "W", "T", "R", "S", "stride_d", "stride_h",
+                                     "stride_w", "pad_d", "pad_h", "pad_w", "groups")]
+
+    def out_dhw(self):
+        return ((self.D + 2 * self.pad_d - self.T) // self.stride_d + 1,
+                (self.H + 2 * self.pad_h - self.R) // self.stride_h + 1,
+                (self.W + 2 * self.pad_w - self.S) // self.stride_w + 1)
 
 
 class McsParams(ctypes.Structure):
@@ -97,6 +108,10 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(ConvGeom), c_void_p, c_int, c_void_p,
                                            c_size_t, c_void_p]
         l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
+        nd_args = [c_void_p, c_void_p, c_void_p, c_void_p, ctypes.POINTER(Conv3dGeom), c_void_p, c_int, c_void_p]
+        l.dai8_conv3d_fwd.argtypes = nd_args
+        l.dai8_conv3d_bwd_data.argtypes = nd_args
+        l.dai8_conv3d_bwd_filter.argtypes = nd_args
         l.dai8_debug_expire_waits.argtypes = [c_uint64, ctypes.POINTER(c_int), c_void_p, c_size_t, c_void_p]
         dp = ctypes.POINTER(ctypes.c_double)
         l.dai8_debug_probe_mma.argtypes = [c_int, c_int, c_int, dp, dp, c_void_p, c_size_t, c_void_p]
@@ -269,3 +284,19 @@ def conv_bwd_filter(qX, vq, sX, s, geom: ConvGeom, dW: torch.Tensor, ws) -> None
     _check(lib().dai8_conv_bwd_filter(_ptr(qX), _ptr(vq), _ptr(sX), _ptr(s), ctypes.byref(geom),
                                       _ptr(dW), _dtype_code(dW), p, n, _stream()),
            "dai8_conv_bwd_filter")
+
+
+def conv3d_fwd(qX, qW, sX, sW, geom: Conv3dGeom, Y: torch.Tensor) -> None:
+    """dai8_conv3d_fwd: codes [N][D][H][W][Cp] x [Cout][T][R][S][Cgp] -> Y [N][Do][P][Q][Cout]."""
+    _check(lib().dai8_conv3d_fwd(_ptr(qX), _ptr(qW), _ptr(sX), _ptr(sW), ctypes.byref(geom), _ptr(Y), _dtype_code(Y),
+                                 _stream()), "dai8_conv3d_fwd")
+
+
+def conv3d_bwd_data(gq, qW, gmax, sW, geom: Conv3dGeom, dX: torch.Tensor) -> None:
+    _check(lib().dai8_conv3d_bwd_data(_ptr(gq), _ptr(qW), _ptr(gmax), _ptr(sW), ctypes.byref(geom), _ptr(dX),
+                                      _dtype_code(dX), _stream()), "dai8_conv3d_bwd_data")
+
+
+def conv3d_bwd_filter(qX, vq, sX, s, geom: Conv3dGeom, dW: torch.Tensor) -> None:
+    _check(lib().dai8_conv3d_bwd_filter(_ptr(qX), _ptr(vq), _ptr(sX), _ptr(s), ctypes.byref(geom), _ptr(dW),
+                                        _dtype_code(dW), _stream()), "dai8_conv3d_bwd_filter")
