@@ -155,6 +155,10 @@ def aggregate_value(ops_per_step_per_rank, ms_per_step, world):
 # ------------------------------------------------------------------------------------------------
 # CUDA arm
 # ------------------------------------------------------------------------------------------------
+GRAPH_SEEDS = 4                 # CUDA graphs of the step, one per rounding seed, replayed in turn
+BLOCKER_CYCLES = 16_000_000     # about 8 ms of device spin in front of a step of the per-call breakdown
+
+
 class LayerBuffers:
     """Device buffers of one layer; `host` adds pinned host copies of the inputs and results."""
 
@@ -339,25 +343,52 @@ class Runner:
             self.dist.barrier()
         self.torch.cuda.synchronize()
 
-    def timed(self, steps, warmup, sampler=None):
+    def capture(self, n_graphs=GRAPH_SEEDS):
+        """The step as CUDA graphs: every entry point only enqueues work on the stream it is given
+        (no allocation, no synchronisation), so a whole step is captured once and replayed.  The seed of
+        the stochastic rounding is a by-value argument, hence one graph per seed; the replays cycle
+        through n_graphs of them.  Returns the kernel launches of one step."""
         torch, api = self.torch, self.api
-        for _ in range(max(warmup, 3)):
+        self.graphs = []
+        per_step = 0
+        for _ in range(n_graphs):
+            g = torch.cuda.CUDAGraph()
+            n0 = api.launch_count()
+            with torch.cuda.graph(g):
+                self.step()
+            per_step = api.launch_count() - n0
+            self.graphs.append(g)
+        self.barrier()
+        return per_step
+
+    def timed(self, steps, warmup, sampler=None, graph=True):
+        torch, api = self.torch, self.api
+        for _ in range(max(warmup, 3)):     # eager: first-use initialisation happens outside any capture
             self.step()
         self.barrier()
+        per_step = self.capture() if graph else 0
+        if graph:
+            for i in range(max(warmup, 3)):
+                self.graphs[i % len(self.graphs)].replay()
+            self.barrier()
         launches0 = api.launch_count()
         t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
         if sampler:
             sampler.mark_start()
         t0.record()
-        for _ in range(steps):
-            self.step()
+        for i in range(steps):
+            if graph:
+                self.graphs[i % len(self.graphs)].replay()
+            else:
+                self.step()
         t1.record()
         self.barrier()
         if sampler:
             sampler.mark_end()
         total_ms = max_over_ranks(t0.elapsed_time(t1), self.dist, self.dev)
-        launches = api.launch_count() - launches0
+        launches = per_step * steps if graph else api.launch_count() - launches0
         assert api.get_device_status() == api.OK
+        self.graphs = []
         return total_ms, launches
 
     def breakdown(self, steps):
@@ -365,7 +396,11 @@ class Runner:
         from overlapping, so this pass is not the one `value` comes from)."""
         records = []
         for _ in range(steps):
+            # the host enqueues a step of small layers more slowly than the GPU runs it; a spin of a few
+            # milliseconds in front lets the host get ahead, so the event pairs bracket device time only
+            self.torch.cuda._sleep(BLOCKER_CYCLES)
             self.step(record=records)
+            self.torch.cuda.synchronize()
         self.barrier()
         agg = {}
         for lname, cname, a, b_ in records:
@@ -492,7 +527,7 @@ def run_dai8(args):
     sampler = ClockSampler(local) if rank == 0 else None
     main = Runner(args.workload, torch, api, synth, dev, dist, world, with_host=True)
     warmup = max(args.warmup, 3)
-    total_ms, launches = main.timed(args.steps, warmup, sampler)
+    total_ms, launches = main.timed(args.steps, warmup, sampler, graph=not args.eager)
     clocks = sampler.stop() if sampler else None
     ms_per_step = total_ms / args.steps
     value = aggregate_value(main.ops_step, ms_per_step, world)
@@ -537,7 +572,7 @@ def run_dai8(args):
                 continue
             r = Runner(wl, torch, api, synth, dev, None, 1)
             steps = min(args.steps, 20)
-            t_ms, _ = r.timed(steps, 3)
+            t_ms, _ = r.timed(steps, 3, graph=not args.eager)
             s, c, _, _ = r.summarize(r.breakdown(min(steps, 5)), INT8_OVER_BF16 * peaks["bf16_burst"], peaks)
             s["workload"] = r.name
             s["ms_per_step"] = round(t_ms / steps, 4)
@@ -562,6 +597,8 @@ def run_dai8(args):
         "config": {"workload": name, "layers": len(workloads()[args.workload][1]()), "batch": batch,
                    "outputs": "Y,dX bf16 NHWC; dW fp32",
                    "l2": "inputs larger than L2 (several GB touched per step)",
+                   "launch": "eager, one library call after another" if args.eager else
+                             f"the step captured in CUDA graphs (one per rounding seed, {GRAPH_SEEDS} seeds in turn) and replayed",
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
         "clocks": clocks, "gpu_launches": int(launches),
         "e2e": {"value": round(e2e_value, 3), "unit": UNIT, "ms_per_step": round(e2e_ms, 3), "steps": e2e_steps,
@@ -739,6 +776,7 @@ def main():
                     help="configuration of the JSON line (default: VGG-16, the compute-bound one)")
     ap.add_argument("--main-only", action="store_true", help="skip the other configurations in `detail`")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--eager", action="store_true", help="time eager library calls instead of CUDA-graph replays of the step")
     ap.add_argument("--layers", default=None, choices=["conv2x", "resnet50", "mobilenetv2", "vgg16"],
                     help="print a per-layer report for a network configuration instead of the benchmark line")
     ap.add_argument("--batch", type=int, default=0)
