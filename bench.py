@@ -295,16 +295,6 @@ class ClockSampler:
                 "samples": len(inside), "window": window, "reasons": reasons}
 
 
-KERNEL_OF_CALL = {
-    "quantize_x": "quantize_tensor kernels (layer scale + codes of X)",
-    "quantize_w": "quantize_tensor kernels (layer scale + codes of W)",
-    "conv_fwd": "igemm_kmajor_kernel (forward)",
-    "quantize_grad": "gvq_fused_nhwc_kernel / gvq_columns_kernel",
-    "conv_bwd_filter": "wgrad_mnmajor_kernel + finalize_bwd_filter_kernel",
-    "conv_bwd_data": "igemm_kmajor_kernel (input gradient)",
-}
-
-
 class Runner:
     """One workload on one GPU: buffers, the step, the timed region, the per-call breakdown."""
 
@@ -314,6 +304,7 @@ class Runner:
         self.layers = fn()
         self.bufs = [LayerBuffers(L, self.batch, SEED + i, torch, api, synth, dev) for i, L in enumerate(self.layers)]
         self.step_no = 0
+        self.kernel_of = {}             # (layer, call) -> kernel family, as the library reports it
         self.ops_step = bwd_ops(self.layers, self.batch)
         self.hosts = [HostBuffers(b, torch) for b in self.bufs] if with_host else None
 
@@ -330,6 +321,7 @@ class Runner:
                 if record is not None:
                     e1 = torch.cuda.Event(enable_timing=True); e1.record()
                     record.append((b.L.name, name, e0, e1))
+                    self.kernel_of[(b.L.name, name)] = api.debug_last_kernel()
 
         for b in bufs:                      # forward pass, layer order
             run(b, b.fwd_calls(api))
@@ -502,8 +494,24 @@ class Runner:
                "conv_bwd_frac_int8_peak": round(bwd_ops_ / bwd_ms / 1e9 / int8_peak, 4),
                "gvq_effective_gbs": round(gvq["bytes"] / gvq["ms"] / 1e6, 1),
                "gvq_frac_hbm": round(gvq["bytes"] / gvq["ms"] / 1e6 / peaks["hbm_gbs"], 4)}
-        dom_name = max(by_call, key=lambda n: by_call[n]["ms"])
-        return out, calls, dom_name, by_call[dom_name]
+        # the same calls grouped by the kernel that served them: the dominant KERNEL of the step
+        by_kernel = {}
+        for key, ms in per_call_ms.items():
+            a = alg[key]
+            t = by_kernel.setdefault(self.kernel_of.get(key, key[1]), {"ms": 0.0, "bytes": 0, "ops": 0, "n": 0, "calls": set()})
+            t["ms"] += ms; t["bytes"] += a["bytes"]; t["ops"] += a.get("ops", 0); t["n"] += 1; t["calls"].add(key[1])
+        kernels = {}
+        for name, t in sorted(by_kernel.items(), key=lambda kv: -kv[1]["ms"]):
+            k = {"ms": round(t["ms"], 4), "share": round(t["ms"] / total, 4), "launch_groups": t["n"],
+                 "calls": sorted(t["calls"]), "gbs": round(t["bytes"] / t["ms"] / 1e6, 1),
+                 "frac_hbm": round(t["bytes"] / t["ms"] / 1e6 / peaks["hbm_gbs"], 4)}
+            if t["ops"]:
+                k["tops"] = round(t["ops"] / t["ms"] / 1e9, 1)
+                k["frac_int8_peak"] = round(t["ops"] / t["ms"] / 1e9 / int8_peak, 4)
+            kernels[name] = k
+        out["kernels"] = kernels
+        dom_name = max(by_kernel, key=lambda n: by_kernel[n]["ms"])
+        return out, calls, dom_name, by_kernel[dom_name]
 
 
 def run_dai8(args):
@@ -551,8 +559,8 @@ def run_dai8(args):
         achieved, peak, unit = dom["bytes"] / dom["ms"] / 1e6, peaks["hbm_gbs"], "GB/s"
     roofline = {"bound": "tensor" if tensor_bound else "hbm", "achieved": round(achieved, 2), "peak": peak,
                 "unit": unit, "frac": round(achieved / peak, 4), "traffic": None,
-                "kernel": KERNEL_OF_CALL[dom_name], "launches_per_step": dom["n"],
-                "share_of_step": summary["phases"][dom_name]["share"],
+                "kernel": dom_name, "launches_per_step": dom["n"], "calls": sorted(dom["calls"]),
+                "share_of_step": summary["kernels"][dom_name]["share"],
                 "algorithmic_ops_per_step": dom["ops"], "algorithmic_bytes_per_step": dom["bytes"],
                 "ms_per_step": round(dom["ms"], 4), "peak_source": peaks["source"],
                 "peak_kind": ("int8 = 2 x bf16 " + ("sustained" if sustained else "burst")) if unit == "TOPS" else "copy",

@@ -272,6 +272,11 @@ dai8_status dai8_get_device_status(int* host_status, void* stream);
 dai8_status dai8_debug_expire_waits(uint64_t limit_cycles, int* report /* host */, void* ws,
                                     size_t ws_bytes, void* stream);
 
+/* Name of the kernel (family) that the calling thread's most recent entry-point call launched, e.g.
+ * "igemm_halo_kernel" -- for harnesses that attribute device time to kernels.  Host only; the string is
+ * static.  "" before the first call. */
+const char* dai8_debug_last_kernel(void);
+
 /* Two micro-measurements behind the library's tiling decisions (`python bench.py --probe`).  Both
  * synchronise `stream`; ws: 32 bytes of device scratch.
  *   dai8_debug_probe_mma  cycles per tcgen05.mma.kind::i8 of M = 128, K = 32 and `n_cols` (16..256,

@@ -30,6 +30,7 @@ EXPORTS = [
     "dai8_launch_count", "dai8_get_device_status", "dai8_debug_expire_waits",
     "dai8_debug_probe_mma", "dai8_debug_probe_sr",
     "dai8_conv3d_fwd", "dai8_conv3d_bwd_data", "dai8_conv3d_bwd_filter",
+    "dai8_debug_last_kernel",
 ]
 
 
@@ -108,6 +109,8 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(ConvGeom), c_void_p, c_int, c_void_p,
                                            c_size_t, c_void_p]
         l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
+        l.dai8_debug_last_kernel.argtypes = []
+        l.dai8_debug_last_kernel.restype = ctypes.c_char_p
         nd_args = [c_void_p, c_void_p, c_void_p, c_void_p, ctypes.POINTER(Conv3dGeom), c_void_p, c_int, c_void_p]
         l.dai8_conv3d_fwd.argtypes = nd_args
         l.dai8_conv3d_bwd_data.argtypes = nd_args
@@ -300,3 +303,8 @@ def conv3d_bwd_data(gq, qW, gmax, sW, geom: Conv3dGeom, dX: torch.Tensor) -> Non
 def conv3d_bwd_filter(qX, vq, sX, s, geom: Conv3dGeom, dW: torch.Tensor) -> None:
     _check(lib().dai8_conv3d_bwd_filter(_ptr(qX), _ptr(vq), _ptr(sX), _ptr(s), ctypes.byref(geom), _ptr(dW),
                                         _dtype_code(dW), _stream()), "dai8_conv3d_bwd_filter")
+
+
+def debug_last_kernel() -> str:
+    """Name of the kernel family the calling thread's last library call launched."""
+    return lib().dai8_debug_last_kernel().decode()

@@ -58,6 +58,8 @@ extern "C" dai8_status dai8_get_device_status(int* host_status, void* stream) {
   return dai8::read_clear_device_status(host_status, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" const char* dai8_debug_last_kernel(void) { return dai8::last_kernel_slot(); }
+
 extern "C" dai8_status dai8_debug_expire_waits(uint64_t limit_cycles, int* report, void* ws, size_t ws_bytes,
                                                void* stream) {
   if (!report || !ws || ws_bytes < 32 || !dai8::aligned16(ws)) return DAI8_ERR_INVALID_ARG;

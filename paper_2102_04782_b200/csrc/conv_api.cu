@@ -119,9 +119,12 @@ extern "C" dai8_status dai8_conv_fwd(const int8_t* qX, const int8_t* qW, const f
     dai8_status r = pack_small_cin(qX, cs, Kp, A, st);
     if (r == DAI8_OK) r = pack_small_cin_weights(qW, cs, Kp, Wp, st);
     if (r != DAI8_OK) return r;
-    return umma_fwd(A, Wp, sX, sW, pw, out, st);
+    r = umma_fwd(A, Wp, sX, sW, pw, out, st);
+    note_kernel("pack_small_cin_kernel + igemm_kmajor_kernel");
+    return r;
   }
   if (mode == 2) return Kp ? DAI8_ERR_WORKSPACE : DAI8_ERR_UNSUPPORTED;
+  note_kernel("direct_fwd_kernel");
   log_choice("conv_fwd: direct kernel");
   return direct_fwd(qX, qW, sX, sW, cs, out, st);
 }
@@ -153,11 +156,14 @@ extern "C" dai8_status dai8_conv_bwd_data(const int8_t* gq, const int8_t* qW, co
     if (r == DAI8_OK) r = pack_small_cin(gq, f, Kp, A, st);
     if (r == DAI8_OK) r = pack_small_cin_weights(wT, f, Kp, Wp, st);
     if (r != DAI8_OK) return r;
-    return umma_fwd(A, Wp, gmax, sW, pw, out, st);
+    r = umma_fwd(A, Wp, gmax, sW, pw, out, st);
+    note_kernel("pack_small_cin_kernel + igemm_kmajor_kernel");
+    return r;
   }
   if (mode == 2) return DAI8_ERR_UNSUPPORTED;
   dai8_status r = repack_weights_transposed(qW, cs, wT, /*flip=*/0, st);
   if (r != DAI8_OK) return r;
+  note_kernel("direct_bwd_data_kernel");
   log_choice("conv_bwd_data: direct kernel");
   return direct_bwd_data(gq, wT, gmax, sW, cs, out, st);
 }
@@ -189,11 +195,13 @@ extern "C" dai8_status dai8_conv_bwd_filter(const int8_t* qX, const int8_t* vq, 
     r = pack_small_cin(qX, cs, Kp, A, st);
     if (r == DAI8_OK) r = umma_bwd_filter_acc(A, vq, pw, acc, &splits, st);
     if (r != DAI8_OK) return r;
+    note_kernel("pack_small_cin_kernel + wgrad_mnmajor_kernel");
     return finalize_bwd_filter(acc, splits, sX, s, pw, &cs, dW, out_dtype, st);
   } else if (mode == 2) {
     return DAI8_ERR_UNSUPPORTED;
   } else {
     DAI8_RETURN_IF_CUDA(cudaMemsetAsync(acc, 0, dw_acc_bytes(cs), st));
+    note_kernel("direct_bwd_filter_kernel");
     log_choice("conv_bwd_filter: direct kernel");
     r = direct_bwd_filter_acc(qX, vq, cs, acc, st);
   }

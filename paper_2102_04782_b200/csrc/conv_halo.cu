@@ -623,6 +623,7 @@ dai8_status launch_halo(const HaloProblem& pb, const float* sa, const float* sb,
   int ctas = sm_count();
   if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
   if (ctas > num_tiles) ctas = num_tiles;
+  note_kernel("igemm_halo_kernel");
   log_choice("igemm_halo_kernel: %d x %d patches, N=%d (%d tiles x %d), kc=%d x %d chunks, taps %dx%d, weights %s (%d pieces), A stages %d, %d accumulators, %s, %d CTAs",
              prm.TY, prm.TX, prm.BN, prm.m_tiles, prm.n_tiles, prm.kc_bytes, prm.chunks, prm.R, prm.S,
              prm.b_resident ? "resident" : (prm.b_mn ? "streamed in place" : "streamed"), prm.b_resident ? pb.R * pb.S * prm.chunks : prm.b_stages,

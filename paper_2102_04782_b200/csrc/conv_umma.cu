@@ -581,6 +581,7 @@ dai8_status launch_igemm(const IgemmProblem& pb, const float* sa, const float* s
   int ctas = sm_count();
   if (prm.b_resident && prm.n_tiles > 1) ctas = ctas >= prm.n_tiles ? ctas / prm.n_tiles * prm.n_tiles : prm.n_tiles;
   if (ctas > num_tiles) ctas = num_tiles;
+  note_kernel("igemm_kmajor_kernel");
   log_choice("igemm_kmajor_kernel: im2col, N=%d (%d tiles x %d), kc=%d, %d chunks in stages of %d, taps %dx%d stride %dx%d, weights %s, %d stages, %s, %d CTAs",
              prm.BN, prm.m_tiles, prm.n_tiles, prm.kc_bytes, total_chunks, prm.G, prm.R, prm.S, prm.sh, prm.sw,
              prm.b_resident ? "resident" : (prm.b_mn ? "streamed in place" : "streamed"), prm.stages,
@@ -992,6 +993,7 @@ dai8_status launch_wgrad(const int8_t* qX, const int8_t* vq, const ConvShape& cs
   static std::atomic<int> attr_done[64];
   if (set_max_smem_once(attr_done, wgrad_mnmajor_kernel, kWgradSmem + 1024) != cudaSuccess) return DAI8_ERR_CUDA;
   const dim3 grid((unsigned)ksplit, (unsigned)(ngroups * prm.ci_tiles), (unsigned)co_tiles);
+  note_kernel("wgrad_mnmajor_kernel");
   log_choice("wgrad_mnmajor_kernel: %d pixel slices x %d tap groups of %d x %d channel tiles of %d x %d output-channel tiles, %d pixels per stage, %d stages",
              ksplit, ngroups, prm.tg, prm.ci_tiles, prm.nb * prm.bw, co_tiles, prm.kp, stages);
   DAI8_RETURN_IF_CUDA(launch_dependent(wgrad_mnmajor_kernel, grid, dim3(kThreadsIgemm), smem_bytes, st, mapG, mapX, prm));

@@ -73,6 +73,14 @@ inline void log_choice(const char* fmt, ...) {
   va_end(ap);
 }
 
+// The kernel (family) the calling thread's last entry-point call ran on: what dai8_debug_last_kernel
+// reports, so that a timing harness can attribute device time to kernels by name.
+inline const char*& last_kernel_slot() {
+  static thread_local const char* name = "";
+  return name;
+}
+inline void note_kernel(const char* name) { last_kernel_slot() = name; }
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }

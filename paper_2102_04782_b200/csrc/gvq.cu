@@ -646,6 +646,42 @@ quantize_nchw_rows_kernel(const T* __restrict__ x, int N, int C, int Cp, int HW,
   }
 }
 
+// Eq. 1 for an NHWC tensor of at most 16 channels (the images a network's first layer reads): a thread
+// owns one pixel and writes its padded code row as one 16-byte vector.
+template <typename T, bool STOCH>
+__global__ void __launch_bounds__(kThreads)
+quantize_nhwc_c16_kernel(const T* __restrict__ x, int64_t npix, int64_t HW, int C, const float* __restrict__ scale,
+                         uint32_t seed, int8_t* __restrict__ q) {
+  const float inv = inv_scale(*scale);
+  const uint32_t key0 = sr_key(seed, 0u);
+  for (int64_t pix = (int64_t)blockIdx.x * kThreads + threadIdx.x; pix < npix; pix += (int64_t)gridDim.x * kThreads) {
+    const T* src = x + pix * C;
+    uint32_t b[16];
+    uint64_t idx = 0;
+    if (STOCH) {
+      const int64_t n = pix / HW;
+      idx = (uint64_t)n * (uint64_t)C * (uint64_t)HW + (uint64_t)(pix - n * HW);   // NCHW index of channel 0
+    }
+#pragma unroll
+    for (int c = 0; c < 16; ++c) {
+      b[c] = 0u;
+      if (c < C) {
+        const float v = to_f32(src[c]);
+        if (STOCH) {
+          const uint32_t hi = (uint32_t)(idx >> 32);
+          const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
+          b[c] = quant_stochastic_bits(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key)));
+          idx += (uint64_t)HW;
+        } else {
+          b[c] = quant_nearest_bits(v, inv);
+        }
+      }
+    }
+    *reinterpret_cast<uint4*>(q + pix * 16) = make_uint4(pack_codes4(b[0], b[1], b[2], b[3]), pack_codes4(b[4], b[5], b[6], b[7]),
+                                                         pack_codes4(b[8], b[9], b[10], b[11]), pack_codes4(b[12], b[13], b[14], b[15]));
+  }
+}
+
 // max|x| over a whole tensor (layout-free), into the bit pattern at out_bits (zeroed before).
 template <typename T, int VE>
 __global__ void __launch_bounds__(kThreads)
@@ -2170,6 +2206,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       a.mp = mp; a.s_state = s_state; a.has_prev = has_prev; a.gmax_layer = gmax_layer; a.stats_out = stats;
       a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
       if (!a.status) return DAI8_ERR_CUDA;
+      note_kernel("gvq_columns_kernel");
       log_choice("quantize_grad: gvq_columns_kernel, %d CTAs x %d vector columns, %lld pixels", grid, per, (long long)npix);
       return launch_columns<T, VEfull>(dY, a, gq != nullptr, grid, smem, st);
     }
@@ -2183,6 +2220,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
     a.cls = cls; a.seed = seed; a.q1 = vq; a.q2 = gq; a.status = device_status_address();
     if (!a.status) return DAI8_ERR_CUDA;
     const bool idx32 = npix * C < ((int64_t)1 << 32);   // NCHW element indices fit 32 bits
+    note_kernel("gvq_fused_nhwc_kernel");
     log_choice("quantize_grad: gvq_fused_nhwc_kernel, C=%d, %lld pixels", C, (long long)npix);
     return launch_fused_select<T, VEfull>(dY, a, gq != nullptr, idx32, st);
   }
@@ -2246,6 +2284,7 @@ dai8_status quantize_grad_typed(const T* dY, dai8_layout layout, int N, int C, i
       quantize_nchw_kernel<T, true, true, false><<<qgrid, kThreads, 0, st>>>(dY, C, Cp, HW, s_state,
                                                                              gmax_layer, seed, vq, nullptr);
   }
+  note_kernel("stats / count / quantize kernels (three launches)");
   log_choice("quantize_grad: three launches (statistics, count, codes), mode %d", mp.mode);
   note_launch(3);
   DAI8_RETURN_IF_CUDA(cudaGetLastError());
@@ -2310,6 +2349,141 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
   }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Weights (an NCHW tensor of N filters with few positions each) in ONE cooperative launch.  A CTA
+// copies a contiguous run of whole filters into shared memory while taking their max|x|, the CTAs
+// combine the maxima through one atomic word and meet at a grid barrier, and each CTA then writes
+// the codes of its filters, transposed to [n][hw][Cp], from shared memory: the tensor is read once,
+// and no thread stores single bytes.
+// ------------------------------------------------------------------------------------------------
+struct RowsArgs {
+  const void* x;
+  int8_t* q;
+  float* scale;          // out: max|x|
+  uint32_t* ctrl;        // [0] grid-barrier counter, [1] bit pattern of the running maximum; zeroed before the launch
+  int N, C, Cp, HW;
+  int rows_per_cta;
+  unsigned int* status;
+};
+
+constexpr int kRowsThreads = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(kRowsThreads)
+quantize_rows_fused_kernel(const RowsArgs a) {
+  extern __shared__ __align__(16) uint8_t rows_raw[];     // [rows of this CTA][C][HW] as in global memory
+  __shared__ float s_part[kRowsThreads / 32];
+  __shared__ uint32_t s_ok;
+  const int tid = threadIdx.x;
+  const int per_n = a.C * a.HW;
+  const int n0 = blockIdx.x * a.rows_per_cta;
+  const int rows = min(a.rows_per_cta, a.N - n0);
+  const int elems = rows * per_n;
+  const T* src = static_cast<const T*>(a.x) + (size_t)n0 * per_n;
+  T* raw = reinterpret_cast<T*>(rows_raw);
+  constexpr int VE = 16 / (int)sizeof(T);
+  float m = 0.f;
+  // the CTA's filters are one contiguous range; 16-byte copies when it starts on a 16-byte boundary
+  const bool vec_ok = (((size_t)n0 * per_n * sizeof(T)) & 15) == 0;
+  const int nvec = vec_ok ? elems / VE : 0;
+#pragma unroll 4
+  for (int i = tid; i < nvec; i += kRowsThreads) {
+    const uint4 r = *reinterpret_cast<const uint4*>(src + (size_t)i * VE);
+    *reinterpret_cast<uint4*>(raw + (size_t)i * VE) = r;
+    float v[VE];
+    unpack_raw(r, v, (const T*)nullptr);
+#pragma unroll
+    for (int e = 0; e < VE; ++e) m = fmaxf(m, fabsf(v[e]));
+  }
+  for (int i = nvec * VE + tid; i < elems; i += kRowsThreads) {
+    const T t = src[i];
+    raw[i] = t;
+    m = fmaxf(m, fabsf(to_f32(t)));
+  }
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  if ((tid & 31) == 0) s_part[tid >> 5] = m;
+  __syncthreads();
+  if (tid == 0) {
+    for (int w = 1; w < kRowsThreads / 32; ++w) m = fmaxf(m, s_part[w]);
+    if (m > 0.f) atomicMax(a.ctrl + 1, __float_as_uint(m));    // non-negative floats order like their bits
+    // grid barrier (bounded): release this CTA's maximum, acquire everybody's
+    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(a.ctrl) : "memory");
+    uint32_t ok = 1u;
+    const long long t0 = clock64();
+    for (;;) {
+      uint32_t seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(a.ctrl) : "memory");
+      if (seen >= gridDim.x) break;
+      if (clock64() - t0 > kWaitTimeoutCycles) {
+        atomicExch(a.status, (unsigned int)DAI8_ERR_TIMEOUT);
+        ok = 0u;
+        break;
+      }
+    }
+    s_ok = ok;
+    s_part[0] = __uint_as_float(__ldcg(a.ctrl + 1));
+  }
+  __syncthreads();
+  if (!s_ok) return;
+  const float smax = s_part[0];
+  if (blockIdx.x == 0 && tid == 0) *a.scale = smax;
+  const float inv = inv_scale(smax);
+  // a warp takes one (filter, position) at a time, a lane four consecutive channels of it: 4-byte
+  // stores, 128 contiguous bytes per warp
+  const int cw = a.Cp >> 2;
+  const int lane = tid & 31;
+  uint32_t* dst = reinterpret_cast<uint32_t*>(a.q + (size_t)n0 * a.HW * a.Cp);
+#pragma unroll 1
+  for (int pix = tid >> 5; pix < rows * a.HW; pix += kRowsThreads / 32) {
+    const int row = pix / a.HW, hw = pix - row * a.HW;
+    const T* rbase = raw + (size_t)row * per_n + hw;
+#pragma unroll 2
+    for (int w = lane; w < cw; w += 32) {
+      const int c = w << 2;
+      const T* r = rbase + (size_t)c * a.HW;
+      uint32_t b[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) b[j] = c + j < a.C ? quant_nearest_bits(to_f32(r[j * a.HW]), inv) : 0u;
+      dst[(size_t)pix * cw + w] = pack_codes4(b[0], b[1], b[2], b[3]);
+    }
+  }
+}
+
+template <typename T>
+bool rows_fused_applicable(int N, int C, int HW, size_t* smem_bytes, int* rows_per_cta) {
+  const FusedConfig& cfg = fused_config();
+  if (!cfg.coop) return false;
+  const size_t row_bytes = (size_t)C * HW * sizeof(T);
+  int64_t ctas = N < cfg.sms ? N : cfg.sms;
+  const int64_t rpc = ceil_div64(N, ctas);
+  const size_t smem = (rpc * row_bytes + 15) / 16 * 16;
+  if (smem + 1024 > cfg.smem_max) return false;
+  *smem_bytes = smem;
+  *rows_per_cta = (int)rpc;
+  return true;
+}
+
+template <typename T>
+dai8_status launch_quantize_rows_fused(const T* x, int N, int C, int Cp, int HW, size_t smem, int rows_per_cta,
+                                       float* scale, int8_t* q, void* ws, cudaStream_t st) {
+  RowsArgs a;
+  a.x = x; a.q = q; a.scale = scale; a.ctrl = static_cast<uint32_t*>(ws);
+  a.N = N; a.C = C; a.Cp = Cp; a.HW = HW; a.rows_per_cta = rows_per_cta;
+  a.status = device_status_address();
+  if (!a.status) return DAI8_ERR_CUDA;
+  auto kern = quantize_rows_fused_kernel<T>;
+  static std::atomic<int> attr_done[64];
+  if (set_max_smem_once(attr_done, kern, fused_config().smem_max - 1024) != cudaSuccess) return DAI8_ERR_CUDA;
+  DAI8_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, 16, st));
+  const int ctas = (N + rows_per_cta - 1) / rows_per_cta;
+  void* args[] = {(void*)&a};
+  DAI8_RETURN_IF_CUDA(cudaLaunchCooperativeKernel((void*)kern, dim3((unsigned)ctas), dim3(kRowsThreads), args, smem, st));
+  note_launch(1);
+  note_kernel("quantize_rows_fused_kernel");
+  log_choice("quantize_tensor: quantize_rows_fused_kernel, %d filters of %d x %d, %d CTAs", N, C, HW, ctas);
+  return DAI8_OK;
+}
+
 constexpr size_t kQuantizeTensorWsBytes = 256;
 
 // One cooperative launch: layer scale and codes of a tensor whose codes have the layout of its values.
@@ -2354,7 +2528,17 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
       // its sweeps (one read from DRAM instead of two); beyond that the two plain kernels stream faster
       total / VEfull <= (int64_t)fused_config().sms * kQtMaxSlots * kQtPieceVecs &&
       fused_config().smem_max >= (size_t)kQtMaxSlots * kQtPieceBytes + 2048)
+  {
+    note_kernel("quantize_flat_fused_kernel");
     return launch_quantize_flat_fused<T>(x, total / VEfull, scale, q, ws, st);
+  }
+  if (ws && mode == DAI8_SCALE_ABSMAX && round == DAI8_ROUND_NEAREST_EVEN && layout == DAI8_NCHW &&
+      npix * Cp > kSmallTensorElems && HW <= 64) {
+    size_t smem = 0;
+    int rpc = 0;
+    if (rows_fused_applicable<T>(N, C, (int)HW, &smem, &rpc))
+      return launch_quantize_rows_fused<T>(x, N, C, Cp, (int)HW, smem, rpc, scale, q, ws, st);
+  }
   if (npix * Cp <= kSmallTensorElems) {
     const int am = mode == DAI8_SCALE_ABSMAX ? 1 : 0, sr = round == DAI8_ROUND_STOCHASTIC ? 1 : 0;
     int small_ctas = (int)ceil_div64(npix * Cp, 4 * kSmallThreads);
@@ -2364,9 +2548,12 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
     else
       DAI8_RETURN_IF_CUDA(launch_dependent(quantize_small_kernel<T, false>, dim3((unsigned)small_ctas), dim3(kSmallThreads), 0, st, x, N, C, (int)HW, Cp, am, sr, seed, scale, q));
     note_launch(1);
+    note_kernel("quantize_small_kernel");
     DAI8_RETURN_IF_CUDA(cudaGetLastError());
     return DAI8_OK;
   }
+  note_kernel(layout == DAI8_NHWC ? "absmax_kernel + quantize_flat_nearest_kernel / quantize_nhwc_kernel"
+                                  : "absmax_kernel + quantize_nchw_kernel");
   if (mode == DAI8_SCALE_ABSMAX) {
     DAI8_RETURN_IF_CUDA(cudaMemsetAsync(scale, 0, sizeof(float), st));
     uint32_t* bits = reinterpret_cast<uint32_t*>(scale);
@@ -2385,6 +2572,12 @@ dai8_status quantize_tensor_typed(const T* x, dai8_layout layout, int N, int C, 
     const int64_t nvec = total / VEfull;      // C is a multiple of 16
     const int blocks = (int)(ceil_div64(nvec, kThreads * 4) < 2 * kMaxPixelBlocks ? ceil_div64(nvec, kThreads * 4) : 2 * kMaxPixelBlocks);
     DAI8_RETURN_IF_CUDA(launch_dependent(quantize_flat_nearest_kernel<T, VEfull>, dim3((unsigned)blocks), dim3(kThreads), 0, st, x, nvec, scale, q));
+  } else if (layout == DAI8_NHWC && Cp == 16 && C < 16) {
+    const int blocks = (int)(ceil_div64(npix, kThreads) < 8 * kMaxPixelBlocks ? ceil_div64(npix, kThreads) : 8 * kMaxPixelBlocks);
+    if (stoch)
+      quantize_nhwc_c16_kernel<T, true><<<blocks, kThreads, 0, st>>>(x, npix, HW, C, scale, seed, q);
+    else
+      quantize_nhwc_c16_kernel<T, false><<<blocks, kThreads, 0, st>>>(x, npix, HW, C, scale, seed, q);
   } else if (layout == DAI8_NHWC) {
     if (C % VEfull == 0) {
       const NhwcGrid g = nhwc_grid(npix, Cp / VEfull);

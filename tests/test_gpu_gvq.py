@@ -194,6 +194,9 @@ LARGE_TENSORS = [
     ((256, 130, 3, 3), api.NCHW),       # weights with padded code channels
     ((1024, 256, 1, 1), api.NCHW),      # pointwise weights
     ((2, 130, 31, 33), api.NCHW),       # channel tiles with a ragged tail
+    ((5, 13, 61, 67), api.NHWC),        # fewer than 16 channels: one thread per pixel
+    ((600, 27, 3, 3), api.NCHW),        # filters whose byte size is not a multiple of 16: ranges of CTAs start unaligned
+    ((300, 100, 5, 5), api.NCHW),       # 5x5 filters, several per CTA
 ]
 
 
