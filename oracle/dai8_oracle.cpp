@@ -131,12 +131,15 @@ void dai8o_classify_clip(const uint32_t* cnt, const float* absmax, int C, int64_
 }
 
 // ---------------------------------------------------------------------------------------------
-// Counter-based uniform numbers for stochastic rounding.  The paper fixes no generator; this one
-// is defined by its integer arithmetic: two rounds of a 32-bit finaliser (xor-shift 16, multiply,
-// xor-shift 13, multiply, xor-shift 16) keyed by the seed and the high half of the element index.
-// stream 0 (per-channel codes) uses the hash itself, stream 1 (layer-wide codes) the hash times an
-// odd constant.  u = top 23 bits * 2^-23, in [0, 1).
-// ---------------------------------------------------------------------------------------------
+// Counter-based uniform numbers for stochastic rounding.  The paper names the rounding mode
+// (Sec. 3) but fixes no generator; this one is defined by its integer arithmetic:
+//   key = finalise32(seed xor 0x9E3779B9 * (high half of the index + 1))       (once per 2^32 elements)
+//   x   = low half of the index * 0x9E3779B1 + key                            (mod 2^32)
+//   f   = high half xor low half of the 64-bit product x * 0x85EBCA6B         (a folded multiply)
+//   h   = f * 0xC2B2AE35 for stream 0 (per-channel codes), f * 0x2C1B3C6D for stream 1 (layer-wide codes)
+//   u   = (h >> 9) * 2^-23, in [0, 1).
+// finalise32 is a 32-bit avalanche function (xor-shift 16, multiply, xor-shift 13, multiply,
+// xor-shift 16).
 static inline uint32_t finalise32(uint32_t h) {
   h ^= h >> 16;
   h *= 0x85EBCA6Bu;
@@ -150,9 +153,10 @@ uint32_t dai8o_rand_bits(uint32_t seed, uint32_t stream, uint64_t index) {
   const uint32_t hi = (uint32_t)(index >> 32);
   const uint32_t lo = (uint32_t)index;
   const uint32_t key = finalise32(seed ^ (0x9E3779B9u * (hi + 1u)));
-  uint32_t h = finalise32(lo ^ key);
-  if (stream != 0) h *= 0x9E3779B1u;
-  return h;
+  const uint32_t x = lo * 0x9E3779B1u + key;
+  const uint64_t p = (uint64_t)x * 0x85EBCA6Bull;
+  const uint32_t f = (uint32_t)(p >> 32) ^ (uint32_t)p;
+  return f * (stream != 0 ? 0x2C1B3C6Du : 0xC2B2AE35u);
 }
 
 float dai8o_rand_uniform(uint32_t seed, uint32_t stream, uint64_t index) {

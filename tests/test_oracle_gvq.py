@@ -217,6 +217,36 @@ def test_uniform_generator():
     assert all(float(x * 2 ** 23).is_integer() for x in u[:100])
 
 
+def test_uniform_generator_pairs_and_strides():
+    """Joint behaviour, which stochastic rounding of neighbouring elements depends on: pairs at lag 1,
+    pairs one channel apart at the same pixel (lag H*W of an NCHW index), the two streams of one
+    element, and the sub-sequence a single pixel column sees (stride H*W) -- 16 x 16 chi-square
+    (255 degrees of freedom: mean 255, s.d. 22.6) and correlations."""
+    n = 1 << 18
+    for seed in (11, 12345):
+        bits0 = np.array([O.rand_bits(seed, 0, i) for i in range(n)], dtype=np.uint32)
+        bits1 = np.array([O.rand_bits(seed, 1, i) for i in range(n)], dtype=np.uint32)
+        u, v = (bits0 >> 9) * 2.0 ** -23, (bits1 >> 9) * 2.0 ** -23
+
+        def chi2(a, b):
+            h = np.histogram2d(a, b, bins=16, range=((0, 1), (0, 1)))[0]
+            e = a.size / 256
+            return ((h - e) ** 2 / e).sum()
+
+        for lag in (1, 49, 196, 3136, 12544):
+            assert chi2(u[:-lag], u[lag:]) < 255 + 5 * 22.6, lag
+            assert abs(np.corrcoef(u[:-lag], u[lag:])[0, 1]) < 4 / math.sqrt(n)
+            assert abs(np.corrcoef(u[:-lag], v[lag:])[0, 1]) < 4 / math.sqrt(n)
+        assert chi2(u, v) < 255 + 5 * 22.6
+        # low-order bits of u (they decide the rounding of values close to an integer)
+        w = (u * 4096) % 1
+        hist = np.histogram(w, bins=16, range=(0, 1))[0]
+        assert ((hist - n / 16) ** 2 / (n / 16)).sum() < 45
+        us = np.array([O.rand_uniform(seed, 0, k * 3136) for k in range(1 << 15)])
+        assert abs(np.corrcoef(us[:-1], us[1:])[0, 1]) < 4 / math.sqrt(us.size)
+        assert abs(us.mean() - 0.5) < 4 * math.sqrt(1 / 12 / us.size)
+
+
 def test_stochastic_rounding_properties():
     """SR picks floor or ceil, is unbiased, saturates at +-127 and errs by less than one step."""
     rng = np.random.default_rng(7)
