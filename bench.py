@@ -298,9 +298,12 @@ class ClockSampler:
 class Runner:
     """One workload on one GPU: buffers, the step, the timed region, the per-call breakdown."""
 
-    def __init__(self, workload, torch, api, synth, dev, dist, world, with_host=False):
+    def __init__(self, workload, torch, api, synth, dev, dist, world, with_host=False, batch=0):
         self.torch, self.api, self.dev, self.dist, self.world = torch, api, dev, dist, world
         self.name, fn, self.batch = workloads()[workload]
+        if batch:                       # a reduced batch, for profiler captures of a small case
+            self.batch = batch
+            self.name += f"_batch{batch}"
         self.layers = fn()
         self.bufs = [LayerBuffers(L, self.batch, SEED + i, torch, api, synth, dev) for i, L in enumerate(self.layers)]
         self.step_no = 0
@@ -533,7 +536,7 @@ def run_dai8(args):
     peaks = measured_peaks()
 
     sampler = ClockSampler(local) if rank == 0 else None
-    main = Runner(args.workload, torch, api, synth, dev, dist, world, with_host=True)
+    main = Runner(args.workload, torch, api, synth, dev, dist, world, with_host=True, batch=args.batch)
     warmup = max(args.warmup, 3)
     total_ms, launches = main.timed(args.steps, warmup, sampler, graph=not args.eager)
     clocks = sampler.stop() if sampler else None
@@ -787,7 +790,7 @@ def main():
     ap.add_argument("--eager", action="store_true", help="time eager library calls instead of CUDA-graph replays of the step")
     ap.add_argument("--layers", default=None, choices=["conv2x", "resnet50", "mobilenetv2", "vgg16"],
                     help="print a per-layer report for a network configuration instead of the benchmark line")
-    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--batch", type=int, default=0, help="reduced batch (profiler captures of a small case; not a benchmark result)")
     ap.add_argument("--probe", action="store_true", help="print the tcgen05.mma issue-rate and rounding-arithmetic micro-measurements")
     args = ap.parse_args()
     if args.probe:

@@ -153,10 +153,11 @@ __device__ __forceinline__ void load_vec<bf16_t, 1>(const bf16_t* p, float (&v)[
 
 // ------------------------------------------------------------------------------------------------
 // Counter-based uniform numbers for stochastic rounding (the paper names the rounding mode in
-// Sec. 3 but no generator).  A 32-bit avalanche finaliser (xor-shift 16, multiply, xor-shift 13,
-// multiply, xor-shift 16) is applied to the low half of the element's NCHW index xor a key that
-// mixes the seed with the high half.  Stream 0 uses the hash, stream 1 the hash times an odd
-// constant.  u = (top 23 bits) * 2^-23.
+// Sec. 3 but no generator).  key = avalanche32(seed xor 0x9E3779B9 * (high half of the element's NCHW
+// index + 1)), once per 2^32 elements; x = low half * 0x9E3779B1 + key; f = high half xor low half of
+// the 64-bit product x * 0x85EBCA6B; stream 0 uses f * 0xC2B2AE35, stream 1 f * 0x2C1B3C6D;
+// u = (top 23 bits) * 2^-23.  Per element that is four multiplies and ONE instruction of the
+// half-rate integer/logic pipe, which is what bounds the code sweep.
 // ------------------------------------------------------------------------------------------------
 __host__ __device__ __forceinline__ uint32_t avalanche32(uint32_t h) {
   h ^= h >> 16;
@@ -213,16 +214,14 @@ __device__ __forceinline__ uint32_t pack_codes4(uint32_t a, uint32_t b, uint32_t
 __device__ __forceinline__ float sr_uniform_fast(uint32_t h) {
   return __uint_as_float(__funnelshift_r(h, 0x7Fu, 9)) - 1.0f;
 }
-// avalanche32(idx ^ key) with the first xor-shift folded: (a ^ a>>16) for a = idx ^ key equals
-// idx ^ (idx >> 16) ^ keyx with keyx = key ^ (key >> 16).
-__device__ __forceinline__ uint32_t sr_hash_folded(uint32_t idx, uint32_t keyx) {
-  uint32_t h = idx ^ (idx >> 16) ^ keyx;
-  h *= 0x85EBCA6Bu;
-  h ^= h >> 13;
-  h *= 0xC2B2AE35u;
-  h ^= h >> 16;
-  return h;
+// The folded multiply f of an element (see above); sr_bits0 / sr_bits1 turn it into the two streams' bits.
+__device__ __forceinline__ uint32_t sr_fold(uint32_t index_lo, uint32_t key) {
+  const uint32_t x = index_lo * 0x9E3779B1u + key;
+  const uint64_t p = (uint64_t)x * 0x85EBCA6Bull;
+  return (uint32_t)(p >> 32) ^ (uint32_t)p;
 }
+__device__ __forceinline__ uint32_t sr_bits0(uint32_t f) { return f * 0xC2B2AE35u; }
+__device__ __forceinline__ uint32_t sr_bits1(uint32_t f) { return f * 0x2C1B3C6Du; }
 __device__ __forceinline__ float inv_scale(float s) { return s > 0.0f ? __fdiv_rn(127.0f, s) : 0.0f; }
 
 }  // namespace dai8

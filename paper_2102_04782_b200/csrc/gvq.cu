@@ -528,9 +528,9 @@ quantize_nhwc_kernel(const T* __restrict__ x, int64_t npix, int64_t HW, int C, i
           const uint64_t idx = idx0 + (uint64_t)e * HW;
           const uint32_t hi = (uint32_t)(idx >> 32);
           const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
-          const uint32_t h = avalanche32((uint32_t)idx ^ key);
+          const uint32_t f = sr_fold((uint32_t)idx, key), h = sr_bits0(f);
           qa[e] = quant_stochastic(v[e], inv1[e], sr_uniform(h));
-          qb[e] = DUAL ? quant_stochastic(v[e], inv2, sr_uniform(h * 0x9E3779B1u)) : 0;
+          qb[e] = DUAL ? quant_stochastic(v[e], inv2, sr_uniform(sr_bits1(f))) : 0;
         } else {
           qa[e] = quant_nearest(v[e], inv1[e]);
           qb[e] = DUAL ? quant_nearest(v[e], inv2) : 0;
@@ -581,9 +581,9 @@ quantize_nchw_kernel(const T* __restrict__ x, int C, int Cp, int64_t HW,
       if (STOCH) {
         const uint32_t hi = (uint32_t)(idx >> 32);
         const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
-        const uint32_t h = avalanche32((uint32_t)idx ^ key);
+        const uint32_t f = sr_fold((uint32_t)idx, key), h = sr_bits0(f);
         a = quant_stochastic(v, sinv[cl], sr_uniform(h));
-        if (DUAL) b = quant_stochastic(v, inv2, sr_uniform(h * 0x9E3779B1u));
+        if (DUAL) b = quant_stochastic(v, inv2, sr_uniform(sr_bits1(f)));
       } else {
         a = quant_nearest(v, sinv[cl]);
         if (DUAL) b = quant_nearest(v, inv2);
@@ -633,7 +633,7 @@ quantize_nchw_rows_kernel(const T* __restrict__ x, int N, int C, int Cp, int HW,
         const uint64_t idx = (uint64_t)n * per_n + (uint64_t)i;       // the NCHW index
         const uint32_t hi = (uint32_t)(idx >> 32);
         const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
-        code = quant_stochastic(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key)));
+        code = quant_stochastic(v, inv, sr_uniform(sr_bits0(sr_fold((uint32_t)idx, key))));
       } else {
         code = quant_nearest(v, inv);
       }
@@ -670,7 +670,7 @@ quantize_nhwc_c16_kernel(const T* __restrict__ x, int64_t npix, int64_t HW, int 
         if (STOCH) {
           const uint32_t hi = (uint32_t)(idx >> 32);
           const uint32_t key = hi == 0u ? key0 : sr_key(seed, hi);
-          b[c] = quant_stochastic_bits(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key)));
+          b[c] = quant_stochastic_bits(v, inv, sr_uniform(sr_bits0(sr_fold((uint32_t)idx, key))));
           idx += (uint64_t)HW;
         } else {
           b[c] = quant_nearest_bits(v, inv);
@@ -1283,7 +1283,6 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   // ---------------- sweep 2: density count + both sets of codes --------------------------------------
   using Idx = typename std::conditional<IDX32, uint32_t, uint64_t>::type;
   const uint32_t key0 = sr_key(a.seed, 0u);
-  const uint32_t keyx0 = key0 ^ (key0 >> 16);
   const Idx HWi = (Idx)a.HW;
   const Idx wrap = (Idx)(C - 1) * HWi;           // added to the NCHW index when n advances
   const int64_t first = p0 + rl;                 // this thread's first pixel
@@ -1298,13 +1297,13 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
   int8_t* o1 = a.q1 + first * a.Cp + c0;
   int8_t* o2 = DUAL ? a.q2 + first * a.Cp + c0 : nullptr;
   float inv1[VE];
-  auto hash_at = [&](Idx idx) -> uint32_t {
+  auto hash_at = [&](Idx idx) -> uint32_t {     // the element's folded multiply (sr_fold)
     if constexpr (IDX32) {
-      return sr_hash_folded(idx, keyx0);
+      return sr_fold(idx, key0);
     } else {
       const uint32_t hi = (uint32_t)(idx >> 32);
       const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-      return avalanche32((uint32_t)idx ^ key);
+      return sr_fold((uint32_t)idx, key);
     }
   };
   // One pixel's vector of this thread: codes with inv1 (and, if with_gq, the layer-wide ones).
@@ -1330,12 +1329,12 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
             idx += HWi;
             const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
             const uint64_t v1 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv1[2 * j])), __float_as_uint(__fmul_rn(g1, inv1[2 * j + 1])));
-            const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0, 0x7Fu, 9), __funnelshift_r(h1, 0x7Fu, 9)), minus1);
+            const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(sr_bits0(h0), 0x7Fu, 9), __funnelshift_r(sr_bits0(h1), 0x7Fu, 9)), minus1);
             f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v1, u1), magic), ra[2 * j], ra[2 * j + 1]);
             if constexpr (DUAL) {
               if (with_gq) {
-                const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0 * 0x9E3779B1u, 0x7Fu, 9),
-                                                            __funnelshift_r(h1 * 0x9E3779B1u, 0x7Fu, 9)), minus1);
+                const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(sr_bits1(h0), 0x7Fu, 9),
+                                                            __funnelshift_r(sr_bits1(h1), 0x7Fu, 9)), minus1);
                 const uint64_t v2 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv2)), __float_as_uint(__fmul_rn(g1, inv2)));
                 f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v2, u2), magic), rb2[2 * j], rb2[2 * j + 1]);
               }
@@ -1348,10 +1347,10 @@ gvq_fused_nhwc_kernel(const T* __restrict__ x, const FusedArgs a) {
         unpack_raw(raw, v, (const T*)nullptr);
 #pragma unroll
         for (int e = 0; e < VE; ++e) {
-          const uint32_t h = hash_at(idx);
+          const uint32_t f = hash_at(idx), h = sr_bits0(f);
           ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
           if constexpr (DUAL) {
-            if (with_gq) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+            if (with_gq) rb2[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(sr_bits1(f)));
           }
           idx += HWi;
         }
@@ -1574,22 +1573,22 @@ struct ColArgs {
 // the pixel-partitioned kernel for the argument).
 template <bool DUAL>
 __device__ __forceinline__ void quantize_vec8_unclipped(const uint4& raw, const float (&inv1)[8], float inv2, uint32_t idx,
-                                                        uint32_t HW, uint32_t keyx0, uint32_t (&ra)[8], uint32_t (&rb)[8]) {
+                                                        uint32_t HW, uint32_t key0, uint32_t (&ra)[8], uint32_t (&rb)[8]) {
   const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
   const uint64_t minus1 = f32x2_pack(0xBF800000u, 0xBF800000u), magic = f32x2_pack(0x4B400000u, 0x4B400000u);
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const uint32_t h0 = sr_hash_folded(idx, keyx0);
+    const uint32_t h0 = sr_fold(idx, key0);
     idx += HW;
-    const uint32_t h1 = sr_hash_folded(idx, keyx0);
+    const uint32_t h1 = sr_fold(idx, key0);
     idx += HW;
     const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
     const uint64_t v1 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv1[2 * j])), __float_as_uint(__fmul_rn(g1, inv1[2 * j + 1])));
-    const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0, 0x7Fu, 9), __funnelshift_r(h1, 0x7Fu, 9)), minus1);
+    const uint64_t u1 = f32x2_add_rn(f32x2_pack(__funnelshift_r(sr_bits0(h0), 0x7Fu, 9), __funnelshift_r(sr_bits0(h1), 0x7Fu, 9)), minus1);
     f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v1, u1), magic), ra[2 * j], ra[2 * j + 1]);
     if (DUAL) {
-      const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(h0 * 0x9E3779B1u, 0x7Fu, 9),
-                                                  __funnelshift_r(h1 * 0x9E3779B1u, 0x7Fu, 9)), minus1);
+      const uint64_t u2 = f32x2_add_rn(f32x2_pack(__funnelshift_r(sr_bits1(h0), 0x7Fu, 9),
+                                                  __funnelshift_r(sr_bits1(h1), 0x7Fu, 9)), minus1);
       const uint64_t v2 = f32x2_pack(__float_as_uint(__fmul_rn(g0, inv2)), __float_as_uint(__fmul_rn(g1, inv2)));
       f32x2_unpack(f32x2_add_rd(f32x2_add_rn(v2, u2), magic), rb[2 * j], rb[2 * j + 1]);
     }
@@ -1797,8 +1796,7 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
         cthr[j] = (__float_as_uint(l0) >> 16) | (__float_as_uint(l1) & 0xFFFF0000u);
       }
     }
-    const uint32_t keyx0 = key0 ^ (key0 >> 16);
-#pragma unroll 2
+  #pragma unroll 2
     for (int p = tid; p < npix; p += kFT) {
       const uint4 raw = mine[p];
       float v[VE];
@@ -1813,7 +1811,7 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
           const uint32_t over = bf16x2_gt_one(raw.x & 0x7FFF7FFFu, cthr[0]) | bf16x2_gt_one(raw.y & 0x7FFF7FFFu, cthr[1]) |
                                 bf16x2_gt_one(raw.z & 0x7FFF7FFFu, cthr[2]) | bf16x2_gt_one(raw.w & 0x7FFF7FFFu, cthr[3]);
           if (over == 0u) {
-            quantize_vec8_unclipped<DUAL>(raw, inv1, inv2, (uint32_t)idx, (uint32_t)a.HW, keyx0, ra, rb);
+            quantize_vec8_unclipped<DUAL>(raw, inv1, inv2, (uint32_t)idx, (uint32_t)a.HW, key0, ra, rb);
             done = true;
           }
         }
@@ -1823,9 +1821,9 @@ gvq_columns_kernel(const T* __restrict__ x, const ColArgs a) {
       for (int e = 0; e < VE; ++e) {
         const uint32_t hi = (uint32_t)(idx >> 32);
         const uint32_t key = hi == 0u ? key0 : sr_key(a.seed, hi);
-        const uint32_t h = avalanche32((uint32_t)idx ^ key);
+        const uint32_t f = sr_fold((uint32_t)idx, key), h = sr_bits0(f);
         ra[e] = quant_stochastic_bits(v[e], inv1[e], sr_uniform_fast(h));
-        if (DUAL) rb[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(h * 0x9E3779B1u));
+        if (DUAL) rb[e] = quant_stochastic_bits(v[e], inv2, sr_uniform_fast(sr_bits1(f)));
         idx += HWi;
       }
       }
@@ -2342,7 +2340,7 @@ quantize_small_kernel(const T* __restrict__ x, int N, int C, int HW, int Cp, int
       const int n = pix / HW, hw = pix - n * HW;
       const int idx = (n * C + c) * HW + hw;               // NCHW index: the generator's counter
       const float v = to_f32(x[NHWC_IN ? pix * C + c : idx]);
-      code = stochastic ? quant_stochastic(v, inv, sr_uniform(avalanche32((uint32_t)idx ^ key0)))
+      code = stochastic ? quant_stochastic(v, inv, sr_uniform(sr_bits0(sr_fold((uint32_t)idx, key0))))
                         : quant_nearest(v, inv);
     }
     q[o] = (int8_t)code;

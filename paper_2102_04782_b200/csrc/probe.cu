@@ -77,7 +77,6 @@ probe_mma_kernel(int N, int kc, int count, long long* out) {
 __global__ void __launch_bounds__(512)
 probe_sr_kernel(int iters, uint32_t seed, float inv1, float inv2, uint32_t* sink) {
   const uint32_t key0 = sr_key(seed, 0u);
-  const uint32_t keyx0 = key0 ^ (key0 >> 16);
   uint32_t idx = (blockIdx.x * blockDim.x + threadIdx.x) * 8u;
   uint32_t acc = 0u;
   uint32_t w[4] = {0x3A833A83u ^ threadIdx.x, 0xBA03BA83u, 0x39003A00u, 0xB9803B00u ^ blockIdx.x};
@@ -87,11 +86,11 @@ probe_sr_kernel(int iters, uint32_t seed, float inv1, float inv2, uint32_t* sink
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float g0 = __uint_as_float(w[j] << 16), g1 = __uint_as_float(w[j] & 0xFFFF0000u);
-      const uint32_t h0 = sr_hash_folded(idx + 2u * j, keyx0), h1 = sr_hash_folded(idx + 2u * j + 1u, keyx0);
-      ra[2 * j] = quant_stochastic_bits(g0, inv1, sr_uniform_fast(h0));
-      ra[2 * j + 1] = quant_stochastic_bits(g1, inv1, sr_uniform_fast(h1));
-      rb[2 * j] = quant_stochastic_bits(g0, inv2, sr_uniform_fast(h0 * 0x9E3779B1u));
-      rb[2 * j + 1] = quant_stochastic_bits(g1, inv2, sr_uniform_fast(h1 * 0x9E3779B1u));
+      const uint32_t f0 = sr_fold(idx + 2u * j, key0), f1 = sr_fold(idx + 2u * j + 1u, key0);
+      ra[2 * j] = quant_stochastic_bits(g0, inv1, sr_uniform_fast(sr_bits0(f0)));
+      ra[2 * j + 1] = quant_stochastic_bits(g1, inv1, sr_uniform_fast(sr_bits0(f1)));
+      rb[2 * j] = quant_stochastic_bits(g0, inv2, sr_uniform_fast(sr_bits1(f0)));
+      rb[2 * j + 1] = quant_stochastic_bits(g1, inv2, sr_uniform_fast(sr_bits1(f1)));
       w[j] += 0x00010001u;                 // new values every iteration
     }
     acc ^= pack_codes4(ra[0], ra[1], ra[2], ra[3]) + pack_codes4(ra[4], ra[5], ra[6], ra[7]);
