@@ -141,6 +141,10 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   const int b_res_bytes = prm.b_resident ? total_chunks * b_chunk_bytes : 0;
   const int chunk_pair_bytes = a_chunk_bytes + (prm.b_resident ? 0 : b_chunk_bytes);   // per chunk of a stage
   const int stage_bytes = prm.G * chunk_pair_bytes;
+  // A tile whose output rows fit one column block would leave one epilogue warp of every lane quarter
+  // idle; there the two warps take alternate TILES instead (warp group g drains accumulator g), so two
+  // tiles are in the epilogue at a time.
+  const bool by_tile = prm.tma_store ? prm.BN * prm.out_elem_bytes <= 128 : prm.BN <= 32;
   uint8_t* stage_out = smem + ((b_res_bytes + 1023) & ~1023);   // [kEpiWarps][2][4 KB] when tma_store
   uint8_t* ring = stage_out + (prm.tma_store ? kEpiWarps * 2 * kOutBlockBytes : 0);
   const int num_tiles = prm.m_tiles * prm.n_tiles;
@@ -148,7 +152,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
   if (threadIdx.x == 0) {
     abort_flag = 0u;
     for (int s = 0; s < prm.stages; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], kEpiWarps); }
+    for (int i = 0; i < 2; ++i) { mbar_init(&acc_full[i], 1); mbar_init(&acc_empty[i], by_tile ? kEpiWarps / 2 : kEpiWarps); }
     mbar_init(&b_full, 1);
     fence_mbar_init();
   }
@@ -312,8 +316,9 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
     const bool vec_ok = nhwc && (prm.Nout % (prm.out_elem_bytes == 2 ? 8 : 4)) == 0;
     const size_t plane = (size_t)prm.oH * prm.oW;
     const float scale = prm.out.dtype == DAI8_I32 ? 0.f : dequant_scale(*prm.sa, *prm.sb);
-    int tile_i = 0, n_store = 0;
-    for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++tile_i) {
+    int tile_i = by_tile ? half : 0, n_store = 0;
+    const int t_step = by_tile ? 2 : 1, c_first = by_tile ? 0 : half, c_step = by_tile ? 1 : 2;
+    for (int t = blockIdx.x + tile_i * (int)gridDim.x; t < num_tiles; t += t_step * (int)gridDim.x, tile_i += t_step) {
       const int buf = tile_i & 1;
       if (!mbar_wait(&acc_full[buf], (tile_i >> 1) & 1, &abort_flag, &g_device_status)) break;
       tc_fence_after();
@@ -335,7 +340,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
         const int cols_per_block = 128 / prm.out_elem_bytes;          // 32 (fp32, int32) or 64 (bf16)
         const int row_bytes = prm.BN * prm.out_elem_bytes;
         uint8_t* my_stage = stage_out + (size_t)(warp - 2) * 2 * kOutBlockBytes;
-        for (int blk = half; blk * 128 < row_bytes; blk += 2) {
+        for (int blk = c_first; blk * 128 < row_bytes; blk += c_step) {
           const int col = blk * cols_per_block;
           if (n0 + col >= prm.Nout) break;
           uint8_t* st = my_stage + (size_t)(n_store & 1) * kOutBlockBytes;
@@ -388,7 +393,7 @@ igemm_kmajor_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_const
           ++n_store;
         }
       } else
-      for (int cg2 = half; cg2 * 32 < prm.BN; cg2 += 2) {
+      for (int cg2 = c_first; cg2 * 32 < prm.BN; cg2 += c_step) {
         const int col = cg2 * 32;
         if (n0 + col >= prm.Nout) break;
         const bool second = col + 16 < prm.BN && n0 + col + 16 < prm.Nout;
