@@ -248,6 +248,61 @@ dai8_status dai8_conv3d_bwd_filter(const int8_t* qX, const int8_t* vq, const flo
                                    const float* s, const dai8_conv3d_geom* geom /* host */, void* dW,
                                    dai8_dtype out_dtype, void* stream);
 
+/* ----------------------------------------------------------------------------------------------
+ * Batch-sharded (data-parallel) operation: every rank holds N_local of the batch's images.  The
+ * statistics, the density count, the classes and the clip values of Algorithm 1 belong to the WHOLE
+ * batch, so the gradient quantizer is split into stages between which the caller exchanges
+ * per-channel scalars among the ranks (any collective library; none is called here):
+ *
+ *   dai8_dp_grad_pivot     pivot[C] = the channel values of the shard's first pixel
+ *        exchange          pivot: broadcast from one rank
+ *   dai8_dp_grad_moments   local |g|max[C] and sums[2][C] = sum (g - pivot_c), sum (g - pivot_c)^2 over
+ *                          the rank's pixels; pivot[C] must be the same on all ranks (e.g. pixel 0 of
+ *                          rank 0's shard, broadcast): it keeps the second moment free of cancellation
+ *        exchange          absmax: maximum over ranks; sums: sum over ranks
+ *   dai8_dp_grad_sigma     mean[C], sigma[C] (Eq. 15's sigma; flags of dai8_mcs_params) and the layer
+ *                          |g|max from the exchanged moments, M_global = pixels of the whole batch
+ *   dai8_dp_grad_count     local cnt[C] = #{|g| > sigma_c} (64-bit integers, so that any integer
+ *                          all-reduce can add them)
+ *        exchange          cnt: sum over ranks
+ *   dai8_dp_grad_solve     Eq. 15 on cnt / M_global, Eq. 11 / 14: s_state[C] in/out, cls[C] (may be NULL)
+ *   dai8_dp_grad_codes     vq (clip values s[C]) and gq (layer |g|max; may be NULL) of the rank's images,
+ *                          stochastic rounding; first_image = index of the rank's first image in the
+ *                          whole batch: the random numbers follow the element's index there, so the
+ *                          codes equal those dai8_quantize_grad writes for the same images of the
+ *                          unsharded tensor
+ *
+ * NHWC only (DAI8_ERR_UNSUPPORTED otherwise); ws: dai8_dp_grad_workspace_bytes(C) bytes, 16-byte
+ * aligned; everything else as for dai8_quantize_grad.  mode must be DAI8_GRAD_FULL in dai8_dp_grad_solve.
+ *
+ * The rest of a sharded layer step uses the ordinary entry points: dai8_absmax gives the local
+ * max|x| (exchange: maximum) for dai8_quantize_tensor with DAI8_SCALE_GIVEN; dai8_conv_bwd_filter
+ * with DAI8_I32 output gives the rank's integer partial of dW (exchange: integer sum, exact), and
+ * dai8_dequant_filter applies Eq. 7 to the sum: dW[co][...] = acc * (sX/127) * (s[co]/127), per_cout =
+ * Cin*R*S values per output channel.
+ * -------------------------------------------------------------------------------------------- */
+size_t dai8_dp_grad_workspace_bytes(int C);
+dai8_status dai8_dp_grad_pivot(const void* dY, dai8_dtype dtype, dai8_layout layout, int C, float* pivot,
+                               void* stream);
+dai8_status dai8_dp_grad_moments(const void* dY, dai8_dtype dtype, dai8_layout layout, int N_local, int C,
+                                 int H, int W, const float* pivot, float* absmax, double* sums, void* ws,
+                                 size_t ws_bytes, void* stream);
+dai8_status dai8_dp_grad_sigma(const float* absmax, const double* sums, const float* pivot, int C,
+                               int64_t M_global, const dai8_mcs_params* params /* host, may be NULL */,
+                               float* mean, float* sigma, float* gmax_layer, void* stream);
+dai8_status dai8_dp_grad_count(const void* dY, dai8_dtype dtype, dai8_layout layout, int N_local, int C, int H,
+                               int W, const float* sigma, long long* cnt, void* ws, size_t ws_bytes,
+                               void* stream);
+dai8_status dai8_dp_grad_solve(const long long* cnt, const float* absmax, int C, int64_t M_global,
+                               const dai8_mcs_params* params /* host, may be NULL */, float* s_state,
+                               int has_prev, uint8_t* cls, void* stream);
+dai8_status dai8_dp_grad_codes(const void* dY, dai8_dtype dtype, dai8_layout layout, int N_local, int C, int H,
+                               int W, int64_t first_image, const float* s, const float* gmax_layer,
+                               uint32_t seed, int8_t* vq, int8_t* gq, void* stream);
+dai8_status dai8_absmax(const void* x, dai8_dtype dtype, int64_t count, float* out, void* stream);
+dai8_status dai8_dequant_filter(const int32_t* acc, const float* sX, const float* s, int Cout,
+                                int64_t per_cout, float* dW, void* stream);
+
 /* Kernel family selection for the convolutions (process-wide, host side): 0 = automatic
  * (tensor-core kernels where the geometry allows, direct kernels otherwise), 1 = direct kernels
  * only, 2 = tensor-core kernels only (DAI8_ERR_UNSUPPORTED where they do not apply), 3 = like 2 but

@@ -31,6 +31,8 @@ EXPORTS = [
     "dai8_debug_probe_mma", "dai8_debug_probe_sr",
     "dai8_conv3d_fwd", "dai8_conv3d_bwd_data", "dai8_conv3d_bwd_filter",
     "dai8_debug_last_kernel",
+    "dai8_dp_grad_workspace_bytes", "dai8_dp_grad_pivot", "dai8_dp_grad_moments", "dai8_dp_grad_sigma", "dai8_dp_grad_count",
+    "dai8_dp_grad_solve", "dai8_dp_grad_codes", "dai8_absmax", "dai8_dequant_filter",
 ]
 
 
@@ -109,6 +111,22 @@ def lib() -> ctypes.CDLL:
                                            ctypes.POINTER(ConvGeom), c_void_p, c_int, c_void_p,
                                            c_size_t, c_void_p]
         l.dai8_get_device_status.argtypes = [ctypes.POINTER(c_int), c_void_p]
+        c_i64 = ctypes.c_int64
+        l.dai8_dp_grad_workspace_bytes.argtypes = [c_int]
+        l.dai8_dp_grad_workspace_bytes.restype = ctypes.c_size_t
+        l.dai8_dp_grad_pivot.argtypes = [c_void_p, c_int, c_int, c_int, c_void_p, c_void_p]
+        l.dai8_dp_grad_moments.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p,
+                                           c_void_p, c_void_p, ctypes.c_size_t, c_void_p]
+        l.dai8_dp_grad_sigma.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_i64, ctypes.POINTER(McsParams),
+                                         c_void_p, c_void_p, c_void_p, c_void_p]
+        l.dai8_dp_grad_count.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_void_p, c_void_p,
+                                         c_void_p, ctypes.c_size_t, c_void_p]
+        l.dai8_dp_grad_solve.argtypes = [c_void_p, c_void_p, c_int, c_i64, ctypes.POINTER(McsParams), c_void_p, c_int,
+                                         c_void_p, c_void_p]
+        l.dai8_dp_grad_codes.argtypes = [c_void_p, c_int, c_int, c_int, c_int, c_int, c_int, c_i64, c_void_p, c_void_p,
+                                         ctypes.c_uint32, c_void_p, c_void_p, c_void_p]
+        l.dai8_absmax.argtypes = [c_void_p, c_int, c_i64, c_void_p, c_void_p]
+        l.dai8_dequant_filter.argtypes = [c_void_p, c_void_p, c_void_p, c_int, c_i64, c_void_p, c_void_p]
         l.dai8_debug_last_kernel.argtypes = []
         l.dai8_debug_last_kernel.restype = ctypes.c_char_p
         nd_args = [c_void_p, c_void_p, c_void_p, c_void_p, ctypes.POINTER(Conv3dGeom), c_void_p, c_int, c_void_p]
@@ -308,3 +326,52 @@ def conv3d_bwd_filter(qX, vq, sX, s, geom: Conv3dGeom, dW: torch.Tensor) -> None
 def debug_last_kernel() -> str:
     """Name of the kernel family the calling thread's last library call launched."""
     return lib().dai8_debug_last_kernel().decode()
+
+
+# ---- batch-sharded (data-parallel) stages ---------------------------------------------------------
+def dp_grad_workspace_bytes(C: int) -> int:
+    return int(lib().dai8_dp_grad_workspace_bytes(C))
+
+
+def _pp(params):
+    return ctypes.byref(params) if params is not None else None
+
+
+def dp_grad_pivot(dY, layout, C, pivot) -> None:
+    _check(lib().dai8_dp_grad_pivot(_ptr(dY), _dtype_code(dY), layout, C, _ptr(pivot), _stream()), "dai8_dp_grad_pivot")
+
+
+def dp_grad_moments(dY, layout, N_local, C, H, W, pivot, absmax, sums, ws) -> None:
+    _check(lib().dai8_dp_grad_moments(_ptr(dY), _dtype_code(dY), layout, N_local, C, H, W, _ptr(pivot), _ptr(absmax),
+                                      _ptr(sums), _ptr(ws), ws.numel() * ws.element_size(), _stream()),
+           "dai8_dp_grad_moments")
+
+
+def dp_grad_sigma(absmax, sums, pivot, C, M_global, params, mean, sigma, gmax_layer) -> None:
+    _check(lib().dai8_dp_grad_sigma(_ptr(absmax), _ptr(sums), _ptr(pivot), C, M_global, _pp(params), _ptr(mean),
+                                    _ptr(sigma), _ptr(gmax_layer), _stream()), "dai8_dp_grad_sigma")
+
+
+def dp_grad_count(dY, layout, N_local, C, H, W, sigma, cnt, ws) -> None:
+    _check(lib().dai8_dp_grad_count(_ptr(dY), _dtype_code(dY), layout, N_local, C, H, W, _ptr(sigma), _ptr(cnt),
+                                    _ptr(ws), ws.numel() * ws.element_size(), _stream()), "dai8_dp_grad_count")
+
+
+def dp_grad_solve(cnt, absmax, C, M_global, params, s_state, has_prev, cls) -> None:
+    _check(lib().dai8_dp_grad_solve(_ptr(cnt), _ptr(absmax), C, M_global, _pp(params), _ptr(s_state), int(has_prev),
+                                    _ptr(cls), _stream()), "dai8_dp_grad_solve")
+
+
+def dp_grad_codes(dY, layout, N_local, C, H, W, first_image, s, gmax_layer, seed, vq, gq) -> None:
+    _check(lib().dai8_dp_grad_codes(_ptr(dY), _dtype_code(dY), layout, N_local, C, H, W, first_image, _ptr(s),
+                                    _ptr(gmax_layer), seed & 0xFFFFFFFF, _ptr(vq), _ptr(gq), _stream()),
+           "dai8_dp_grad_codes")
+
+
+def absmax(x, out) -> None:
+    _check(lib().dai8_absmax(_ptr(x), _dtype_code(x), x.numel(), _ptr(out), _stream()), "dai8_absmax")
+
+
+def dequant_filter(acc, sX, s, Cout, per_cout, dW) -> None:
+    _check(lib().dai8_dequant_filter(_ptr(acc), _ptr(sX), _ptr(s), Cout, per_cout, _ptr(dW), _stream()),
+           "dai8_dequant_filter")

@@ -11,7 +11,7 @@ PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 OBJ = PKG / "_build"
 LIB = PKG / "libdai8.so"
-SOURCES = ["api.cu", "gvq.cu", "conv_direct.cu", "conv_umma.cu", "conv_halo.cu", "conv_api.cu", "conv_nd.cu", "probe.cu"]
+SOURCES = ["api.cu", "gvq.cu", "conv_direct.cu", "conv_umma.cu", "conv_halo.cu", "conv_api.cu", "conv_nd.cu", "gvq_dp.cu", "probe.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--fmad=true"]
